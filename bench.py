@@ -1,0 +1,341 @@
+#!/usr/bin/env python
+"""Benchmark of the SwiftPrune pruning pass on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload llama2-7b] [--batch-seqs 16]
+
+A step is one pass of the whole hot path over one synthetic model: for every block and every
+distinct layer input, the calibration statistics are accumulated over all calibration tokens
+(sp_calib_accumulate in batches), finalised, and every layer reading that input is selected
+and written back (sp_select_nm / sp_select_unstructured).  The metric is pruned weights per
+second (all linear-layer weights of the model / step time).  With N > 1 ranks (torchrun) every
+rank prunes its own model of the same shape (independent problems, no data-path collective):
+weak scaling; the value is the total over ranks divided by the slowest rank's time.
+
+--impl reference times the CPU oracle (the plain restatement of the paper's algorithm) on the
+host cores on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "pruned_weights_per_sec"
+UNIT = "weights/s"
+# fused select + write-back: 2 B read + 2 B write per weight + 1 bit of mask
+SELECT_BYTES_PER_WEIGHT = 4.125
+CALIB_BYTES_PER_ELEMENT = 2.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama2-7b")
+    ap.add_argument("--batch-seqs", type=int, default=16,
+                    help="calibration sequences per sp_calib_accumulate call")
+    ap.add_argument("--e2e-steps", type=int, default=1)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_uuid: str | None):
+        self.samples = []
+        self.proc = None
+        self.uuid = gpu_uuid
+
+    def start(self):
+        cmd = ["nvidia-smi", "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+               "-lms", "100"]
+        if self.uuid:
+            cmd += ["-i", self.uuid]
+        try:
+            self.proc = subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.DEVNULL,
+                                         text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for s in self.samples:
+            parts = [p.strip() for p in s.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def mode_args(w):
+    if w.mode == "nm":
+        return [tuple(p) for p in w.patterns]
+    return list(w.sparsities)
+
+
+# ---------------------------------------------------------------------------- CPU oracle legs
+
+def oracle_sample(w, threads: int):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload: the selection of
+    every layer of block 0 at full size, and the calibration statistics of block 0's four
+    inputs over a subset of the sequences (scaled to all sequences).  Returns a dict with the
+    extrapolated weights/s for one whole-model pass."""
+    import torch
+    from oracle import swiftprune_oracle as so
+    from paper_2501_16376_b200 import synth
+
+    odt = so.F16 if w.dtype == "f16" else so.BF16
+    sample_seqs = max(1, min(w.n_seqs, 2))
+    t_calib = 0.0
+    stats = {}
+    for name, d_in in w.input_widths().items():
+        X = synth.gen_activations(w, 0, name, d_in, 0, sample_seqs, "cpu")
+        Xb = synth.bits_of(X)
+        st = so.new_stats(d_in)
+        t0 = time.perf_counter()
+        so.colsq_accumulate(st, Xb, odt, threads=threads)
+        t_calib += time.perf_counter() - t0
+        stats[name] = st
+    t_calib_full = t_calib * (w.n_seqs / sample_seqs)
+    arg = mode_args(w)[0]
+    t_select = 0.0
+    weights = 0
+    for layer in w.layers:
+        W = synth.bits_of(synth.gen_weight(w, 0, layer, "cpu"))
+        t0 = time.perf_counter()
+        if w.mode == "nm":
+            so.select_nm(W, odt, stats[layer.input], arg[0], arg[1], threads=threads)
+        else:
+            so.select_unstructured(W, odt, stats[layer.input], arg, threads=threads)
+        t_select += time.perf_counter() - t0
+        weights += layer.d_out * layer.d_in
+    t_block = t_calib_full + t_select
+    return {
+        "value": weights / t_block,
+        "unit": UNIT,
+        "cores": threads,
+        "kind": "oracle",
+        "sample": ("block 0 of %d: selection of all %d layers at full size (%.2f s) + statistics "
+                   "of its %d inputs over %d of %d sequences (%.2f s, scaled x%d)"
+                   % (w.blocks, len(w.layers), t_select, len(stats), sample_seqs, w.n_seqs,
+                      t_calib, w.n_seqs // sample_seqs)),
+        "block_seconds": t_block,
+        "whole_model_seconds": t_block * w.blocks,
+    }
+
+
+def reference_arm(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    from oracle import swiftprune_oracle as so
+    from paper_2501_16376_b200 import synth
+    w = synth.WORKLOADS[args.workload]
+    threads = so.max_threads()
+    so.build()
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample(synth.scaled(w, blocks=1, n_seqs=2, seq_len=64, shrink=8), threads)
+    results = [oracle_sample(w, threads) for _ in range(max(1, args.steps))]
+    best = max(results, key=lambda r: r["value"])
+    mean_block = sum(r["block_seconds"] for r in results) / len(results)
+    value = w.weights_per_block() / mean_block
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": mean_block * w.blocks * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "mode": w.mode, "mode_arg": str(mode_args(w)[0]),
+                   "note": "CPU oracle on host cores; each step is a bounded sample "
+                           "(one block) extrapolated to the whole model"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                         "sample": best["sample"]},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# ---------------------------------------------------------------------------- GPU arm
+
+def gpu_arm(args):
+    import torch
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA library has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+    from paper_2501_16376_b200 import binding as sp
+    from paper_2501_16376_b200 import pipeline, synth
+    from paper_2501_16376_b200 import sharding
+
+    w = synth.WORKLOADS[args.workload]
+    arg = mode_args(w)[0]
+    batch_tokens = args.batch_seqs * w.seq_len
+    # weak scaling: rank r prunes its own model (seed offset r)
+    mb = pipeline.allocate_model(w, device, model_seed_offset=sharding.unit_of_rank(rank, world))
+    torch.cuda.synchronize()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        pipeline.prune_model(mb, arg, batch_tokens)
+    barrier()
+
+    uuid = None
+    try:
+        uuid = "GPU-" + str(torch.cuda.get_device_properties(device).uuid)
+    except Exception:
+        pass
+    sampler = ClockSampler(uuid)
+    sampler.start()
+
+    phase_events = []
+    launches_before = sp.sp_launch_count()
+    start = torch.cuda.Event(enable_timing=True)
+    stop = torch.cuda.Event(enable_timing=True)
+    barrier()
+    start.record()
+    counts = None
+    for _ in range(args.steps):
+        counts = pipeline.prune_model(mb, arg, batch_tokens, phase_events)
+    stop.record()
+    barrier()
+    elapsed_ms = start.elapsed_time(stop)
+    launches = sp.sp_launch_count() - launches_before
+    clocks = sampler.stop()
+
+    elapsed_ms = sharding.max_over_ranks(elapsed_ms, world, device)
+    total_weights = w.total_weights() * world
+    value = total_weights * args.steps / (elapsed_ms * 1e-3)
+
+    calib_ms = sum(a.elapsed_time(b) for k, a, b, _ in phase_events if k == "calib")
+    select_ms = sum(a.elapsed_time(b) for k, a, b, _ in phase_events if k == "select")
+    x_elements = sum(w.tokens * d for d in w.input_widths().values()) * w.blocks * args.steps
+    calib_launches = counts["calib"] * args.steps
+    select_launches = counts["select"] * args.steps
+    peak, peak_kind = measured_peaks()
+    calib_gbs = CALIB_BYTES_PER_ELEMENT * x_elements / (calib_ms * 1e-3) / 1e9
+    select_gbs = SELECT_BYTES_PER_WEIGHT * w.total_weights() * args.steps / (select_ms * 1e-3) / 1e9
+    roofline = {
+        "kernel": "calib_accumulate_kernel", "bound": "hbm", "achieved": calib_gbs, "peak": peak,
+        "peak_kind": peak_kind, "unit": "GB/s", "frac": calib_gbs / peak, "traffic": None,
+        "avg_launch_ms": calib_ms / calib_launches,
+        "bytes_per_launch": CALIB_BYTES_PER_ELEMENT * x_elements / calib_launches,
+    }
+    roofline_select = {
+        "kernel": "select_nm_kernel" if w.mode == "nm" else "ewma_scan_kernel",
+        "bound": "hbm", "achieved": select_gbs, "peak": peak, "peak_kind": peak_kind,
+        "unit": "GB/s", "frac": select_gbs / peak, "frac_of_8TBs": select_gbs / 8000.0,
+        "traffic": None, "avg_launch_ms": select_ms / select_launches,
+        "bytes_per_launch": SELECT_BYTES_PER_WEIGHT * w.total_weights() * args.steps / select_launches,
+        "weights_per_sec": w.total_weights() * args.steps / (select_ms * 1e-3),
+        "note": "phase time includes one finalisation launch per layer input",
+    }
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": elapsed_ms / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "weights_dtype": w.dtype, "mode": w.mode,
+                   "mode_arg": str(arg), "blocks": w.blocks, "total_weights": w.total_weights(),
+                   "calib_tokens": w.tokens, "batch_tokens": batch_tokens,
+                   "l2": "inputs larger than L2 (every buffer is touched once per step; "
+                         "%.1f GB stream between reuses)" % (
+                             (CALIB_BYTES_PER_ELEMENT * x_elements / args.steps
+                              + 4 * w.total_weights()) / 1e9),
+                   "parallelism": "independent models per rank" if world > 1 else "single GPU"},
+        "whole_model_prune_s": {"calib": calib_ms / args.steps * 1e-3,
+                                "select_apply": select_ms / args.steps * 1e-3,
+                                "total": elapsed_ms / args.steps * 1e-3},
+        "roofline": roofline, "roofline_select": roofline_select,
+        "clocks": clocks, "gpu_launches": int(launches),
+    }
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import swiftprune_oracle as so
+        cb = oracle_sample(w, so.max_threads())
+        line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
+        line["cpu_baseline"]["whole_model_seconds"] = cb["whole_model_seconds"]
+
+    mb.close()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line))
+    return 0
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        return reference_arm(args)
+    return gpu_arm(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,211 @@
+/*
+ * swiftprune.h -- C ABI of the B200 (sm_100a) SwiftPrune pruning pass.
+ *
+ * The library implements the per-layer pruning pass of SwiftPrune
+ * (arXiv 2501.16376): calibration statistics (Algorithm 1, step 1), the
+ * Hessian-free contribution metric (Eq. 8), the EWMA running-threshold
+ * selection that replaces sorting (Algorithm 1; state rules in Table 2; the
+ * parameter la per pruning ratio in Table 3), the N:M group selection
+ * (Section 3.3) and the write-back of the pruned weights (Algorithm 1,
+ * "w_i = 0" / "c_i = w_i").
+ *
+ * General conventions
+ *   - Unless a parameter says "host", every data pointer is a DEVICE pointer to
+ *     memory owned by the caller, on the device the context was created for.
+ *     The library owns only the context (O(d_in) device memory).
+ *   - Calls enqueue work on the caller's stream (sp_stream = cudaStream_t passed
+ *     as void*; NULL = the default stream) and return without synchronising,
+ *     except sp_create, sp_destroy, sp_get_stats, sp_set_stats and
+ *     the *_host entry point, which say so.
+ *   - Arguments are validated on the host before anything is launched; a
+ *     non-SP_OK status means nothing was enqueued by that call.  No call
+ *     throws, traps or aborts.
+ *   - A weight matrix W is [n_rows, d_in] row-major 16-bit floats with leading
+ *     dimension ldw (elements, >= d_in): one row per output neuron, one column
+ *     per input channel.  Rows are pruned independently (Section 2; Algorithm 1,
+ *     "parallel calculation for each row").
+ *   - A mask is [n_rows, ceil(d_in/32)] uint32, row-major, no padding between
+ *     rows; bit j of word k of a row is the keep flag of column 32k+j
+ *     (1 = kept, 0 = pruned; bits past d_in are 0).
+ *   - Pruned weights are written as +0 (bit pattern 0x0000); kept weights are
+ *     copied bit for bit.
+ *   - Fast paths need 16-byte aligned base pointers and leading dimensions
+ *     that are multiples of 8 elements; anything else is handled by slower
+ *     element-wise paths with identical results.
+ *   - One context belongs to one layer input of width d_in; layers that read
+ *     the same input (q/k/v; gate/up) share it.  A context must not be used
+ *     from two streams at once.
+ */
+#ifndef SWIFTPRUNE_H_
+#define SWIFTPRUNE_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sp_ctx sp_ctx; /* opaque, library-owned */
+typedef void *sp_stream;      /* a cudaStream_t */
+
+typedef enum {
+    SP_OK = 0,
+    SP_ERR_INVALID_ARG = 1, /* null pointer, negative size, unknown enum value */
+    SP_ERR_SHAPE = 2,       /* ld < d_in, d_in % M != 0, size over a stated maximum */
+    SP_ERR_DTYPE = 3,
+    SP_ERR_STATE = 4,       /* selection or scoring before any calibration data */
+    SP_ERR_DEGENERATE = 5,  /* S == 0 or non-finite statistics (sp_get_stats reports it) */
+    SP_ERR_CUDA = 6,        /* a CUDA runtime call failed; see sp_last_cuda_error */
+    SP_ERR_NOMEM = 7
+} sp_status;
+
+typedef enum { SP_F16 = 0, SP_BF16 = 1 } sp_dtype;
+
+/* How the EWMA selection treats Algorithm 1's step "S = S - w_i^2" (Table 2, row S). */
+typedef enum {
+    SP_S_FROZEN = 0,    /* S keeps its initial value; rows are scanned in parallel */
+    SP_S_LITERAL_W2 = 1 /* the printed update, evaluated sequentially along each row */
+} sp_s_update;
+
+/* Parameters of Algorithm 1 (alpha, beta: Table 2; la: Table 3). */
+typedef struct {
+    float alpha;
+    float beta;
+    float la;
+    int s_update; /* an sp_s_update */
+} sp_ewma_params;
+
+/* Entries of the optional device counter block passed to the selection calls. */
+enum { SP_COUNTER_KEPT = 0, SP_COUNTER_S_HAZARD = 1, SP_NUM_COUNTERS = 2 };
+
+/* ------------------------------------------------------------------ context */
+
+/*
+ * Creates the context for one layer input of d_in channels on CUDA device
+ * `device` (1 <= d_in <= 2^20).  Allocates its device memory (statistics,
+ * per-channel factors, partial sums) and synchronises with that device once.
+ * The statistics start empty.
+ */
+sp_status sp_create(sp_ctx **out, int64_t d_in, int device);
+
+/* Frees the context (synchronises with its device first).  NULL is allowed. */
+sp_status sp_destroy(sp_ctx *ctx);
+
+/* ------------------------------------------------------------------ calibration (Algorithm 1, step 1) */
+
+/* Forgets all accumulated statistics. */
+sp_status sp_calib_reset(sp_ctx *ctx, sp_stream stream);
+
+/*
+ * Adds one batch of calibration activations: for every channel q,
+ *     colsq[q] += sum_t X[t, q]^2.
+ * colsq[q] is the "x_q^2" of Eq. 8, i.e. the q-th diagonal entry of X X^T
+ * (Section 2: H = 2 X X^T), and S = sum_q colsq[q] is Algorithm 1's step 1.
+ * X is [n_tokens, d_in] row-major of `dtype` with leading dimension ldx
+ * (elements).  n_tokens == 0 is a no-op.  Squares are exact in fp32; sums of
+ * at most 8 squares are formed in fp32 and then accumulated in fp64.  The
+ * result does not depend on run-to-run scheduling (no floating-point atomics).
+ */
+sp_status sp_calib_accumulate(sp_ctx *ctx, const void *X, sp_dtype dtype, int64_t n_tokens,
+                              int64_t ldx, sp_stream stream);
+
+/*
+ * Reads the statistics back to HOST buffers (any may be NULL) and synchronises
+ * the stream: colsq_host[d_in] (fp64), *S_host, factor_host[d_in] (the fp32
+ * per-channel factor c_q = 1/(2(1 - colsq[q]/S)) of Eq. 8), *n_tokens_host.
+ * Returns SP_ERR_DEGENERATE if S is zero or not finite, SP_ERR_STATE if no
+ * token has been accumulated.
+ */
+sp_status sp_get_stats(sp_ctx *ctx, double *colsq_host, double *S_host, float *factor_host,
+                       int64_t *n_tokens_host, sp_stream stream);
+
+/*
+ * Replaces the statistics by colsq_host[d_in] (HOST, fp64) and a token count
+ * (> 0), e.g. to resume from saved statistics.  Synchronises the stream.
+ */
+sp_status sp_set_stats(sp_ctx *ctx, const double *colsq_host, int64_t n_tokens, sp_stream stream);
+
+/* ------------------------------------------------------------------ metric (Eq. 8) */
+
+/*
+ * Finalises the statistics (S and the per-channel factor c_q) if new batches
+ * arrived since the last finalisation, and, if scores_out is not NULL, writes
+ *     L[r, q] = (w[r,q] * w[r,q]) * c_q ,   c_q = 0.5 / (1 - colsq[q] / S)
+ * as fp32 [n_rows, d_in] (dense, leading dimension d_in), which is Eq. 8 with S
+ * at its initial value.  All operations are IEEE binary32 with one rounding
+ * each, in exactly this order: u = colsq32/S32, den = 1-u, c = 0.5/den,
+ * w2 = w*w (exact), L = w2*c.  W may be NULL when scores_out is NULL
+ * (finalise only).  The selection calls finalise implicitly.
+ */
+sp_status sp_score(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows, int64_t ldw,
+                   float *scores_out, sp_stream stream);
+
+/* ------------------------------------------------------------------ selection */
+
+/* Table 3: la for a pruning ratio in (0, 1).  The five listed ratios (0.5 .. 0.9)
+ * return the printed values; other ratios are interpolated linearly between, or
+ * extrapolated from, the nearest two (the paper gives no values there). */
+sp_status sp_la_for_sparsity(float sparsity, float *la_out);
+
+/*
+ * Algorithm 1 (EWMA running threshold) on every row of W, fused with the
+ * write-back.  Along each row, for i = 0 .. d_in-1:
+ *     L_i as in sp_score;  est starts at L_0, dev at 0 (Table 2);
+ *     prune w_i  iff  L_i < est - la * dev      (state before the update);
+ *     est <- (1-alpha) est + alpha L_i;  dev <- (1-beta) dev + beta |est - L_i|
+ *     (dev uses the updated est, as Algorithm 1 orders the two steps).
+ * Column 0 of every row is therefore never pruned.
+ *   sparsity   nominal pruning ratio; la = sp_la_for_sparsity(sparsity),
+ *              alpha = beta = 0.125 (Section 4.2), S frozen.  The achieved ratio
+ *              is only approximately the nominal one.
+ *   mask_out   nullable; mask as described above.
+ *   W_out      nullable; pruned copy of W with leading dimension ldo; may alias W
+ *              exactly (same pointer, same ld) for in-place pruning.
+ *   counters   nullable; SP_NUM_COUNTERS device uint64 the call ADDS to:
+ *              [SP_COUNTER_KEPT] kept weights, [SP_COUNTER_S_HAZARD] rows in which
+ *              Algorithm 1's "S = S - w_i^2" could have changed S in binary32
+ *              (when 0, SP_S_FROZEN and SP_S_LITERAL_W2 give identical results).
+ * The frozen-S path evaluates the two recurrences as warp-level affine scans in
+ * fp32; results differ from a sequential fp32 evaluation by re-association only.
+ */
+sp_status sp_select_unstructured(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
+                                 int64_t ldw, float sparsity, uint32_t *mask_out, void *W_out,
+                                 int64_t ldo, unsigned long long *counters, sp_stream stream);
+
+/* Same with explicit parameters (0 < alpha, beta <= 1; la finite). */
+sp_status sp_select_unstructured_ex(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
+                                    int64_t ldw, const sp_ewma_params *params /* host */,
+                                    uint32_t *mask_out, void *W_out, int64_t ldo,
+                                    unsigned long long *counters, sp_stream stream);
+
+/*
+ * Section 3.3: N:M selection fused with the write-back.  Every row is cut into
+ * contiguous groups of M columns starting at column 0; in each group the N
+ * weights with the largest L (as in sp_score) are kept and the M-N smallest are
+ * pruned; among equal scores the lower column is pruned first; a NaN score
+ * ranks above every number.  M is 4 or 8, 0 < N < M, d_in % M == 0
+ * (else SP_ERR_SHAPE).  2:4 keeps two of every four.
+ */
+sp_status sp_select_nm(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows, int64_t ldw,
+                       int N, int M, uint32_t *mask_out, void *W_out, int64_t ldo,
+                       sp_stream stream);
+
+/*
+ * Algorithm 1's write-back on its own: W_out = W where the mask bit is 1, +0
+ * elsewhere.  W_out may alias W exactly.  Needs no context.
+ */
+sp_status sp_apply_mask(const void *W, sp_dtype dtype, int64_t n_rows, int64_t n_cols, int64_t ldw,
+                        const uint32_t *mask, void *W_out, int64_t ldo, sp_stream stream);
+
+/* ------------------------------------------------------------------ diagnostics */
+
+const char *sp_status_string(sp_status status);
+/* Text of the last CUDA error this thread saw inside the library ("" if none). */
+const char *sp_last_cuda_error(void);
+/* Kernels launched by the library since it was loaded (all threads). */
+uint64_t sp_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SWIFTPRUNE_H_ */

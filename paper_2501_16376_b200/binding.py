@@ -1,0 +1,251 @@
+"""Thin ctypes binding of libswiftprune.so: same names as the C ABI, argument marshalling only.
+
+Every step of the pruning pass runs in the library's CUDA kernels.  PyTorch tensors are used
+for device memory and streams; this module reads their ``data_ptr()``, shape and stride and
+passes them through.  If the compiled library is missing the import fails: there is no
+fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libswiftprune.so")
+
+SP_OK = 0
+SP_ERR_INVALID_ARG, SP_ERR_SHAPE, SP_ERR_DTYPE, SP_ERR_STATE = 1, 2, 3, 4
+SP_ERR_DEGENERATE, SP_ERR_CUDA, SP_ERR_NOMEM = 5, 6, 7
+SP_F16, SP_BF16 = 0, 1
+SP_S_FROZEN, SP_S_LITERAL_W2 = 0, 1
+SP_COUNTER_KEPT, SP_COUNTER_S_HAZARD, SP_NUM_COUNTERS = 0, 1, 2
+
+#: every symbol include/swiftprune.h declares
+EXPORTS = (
+    "sp_create", "sp_destroy", "sp_calib_reset", "sp_calib_accumulate", "sp_get_stats",
+    "sp_set_stats", "sp_score", "sp_la_for_sparsity", "sp_select_unstructured",
+    "sp_select_unstructured_ex", "sp_select_nm", "sp_apply_mask", "sp_status_string",
+    "sp_last_cuda_error", "sp_launch_count",
+)
+
+
+class SpError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(what)
+
+
+class EwmaParams(ctypes.Structure):
+    _fields_ = [("alpha", ctypes.c_float), ("beta", ctypes.c_float), ("la", ctypes.c_float),
+                ("s_update", ctypes.c_int)]
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            "libswiftprune.so is not built (%s); run `python -m paper_2501_16376_b200.build`. "
+            "There is no CPU fallback." % LIB_PATH)
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i64, ci, f32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_float
+    lib.sp_create.argtypes = [ctypes.POINTER(vp), i64, ci]
+    lib.sp_destroy.argtypes = [vp]
+    lib.sp_calib_reset.argtypes = [vp, vp]
+    lib.sp_calib_accumulate.argtypes = [vp, vp, ci, i64, i64, vp]
+    lib.sp_get_stats.argtypes = [vp, vp, vp, vp, ctypes.POINTER(i64), vp]
+    lib.sp_set_stats.argtypes = [vp, vp, i64, vp]
+    lib.sp_score.argtypes = [vp, vp, ci, i64, i64, vp, vp]
+    lib.sp_la_for_sparsity.argtypes = [f32, ctypes.POINTER(f32)]
+    lib.sp_select_unstructured.argtypes = [vp, vp, ci, i64, i64, f32, vp, vp, i64, vp, vp]
+    lib.sp_select_unstructured_ex.argtypes = [vp, vp, ci, i64, i64, ctypes.POINTER(EwmaParams),
+                                              vp, vp, i64, vp, vp]
+    lib.sp_select_nm.argtypes = [vp, vp, ci, i64, i64, ci, ci, vp, vp, i64, vp]
+    lib.sp_apply_mask.argtypes = [vp, ci, i64, i64, i64, vp, vp, i64, vp]
+    lib.sp_status_string.argtypes = [ci]
+    lib.sp_status_string.restype = ctypes.c_char_p
+    lib.sp_last_cuda_error.restype = ctypes.c_char_p
+    lib.sp_launch_count.restype = ctypes.c_uint64
+    for name in EXPORTS:
+        fn = getattr(lib, name)
+        if fn.restype is ctypes.c_int and name not in ("sp_status_string",):
+            fn.restype = ci
+    return lib
+
+
+lib = _load()
+
+
+def _check(status: int):
+    if status != SP_OK:
+        msg = lib.sp_status_string(status).decode()
+        if status in (SP_ERR_CUDA, SP_ERR_NOMEM):
+            msg += " [" + lib.sp_last_cuda_error().decode() + "]"
+        raise SpError(status, msg)
+
+
+def _dtype_of(t: torch.Tensor) -> int:
+    if t.dtype == torch.float16:
+        return SP_F16
+    if t.dtype == torch.bfloat16:
+        return SP_BF16
+    raise SpError(SP_ERR_DTYPE, "expected a float16 or bfloat16 tensor, got %s" % t.dtype)
+
+
+def _matrix(t: torch.Tensor, what: str):
+    if t.dim() != 2 or (t.shape[1] > 1 and t.stride(1) != 1):
+        raise SpError(SP_ERR_SHAPE, "%s must be 2-D with unit stride along its rows" % what)
+    if not t.is_cuda:
+        raise SpError(SP_ERR_INVALID_ARG, "%s must be a CUDA tensor" % what)
+    ld = t.stride(0) if t.shape[0] > 1 else max(t.stride(0), t.shape[1])
+    return t.data_ptr(), t.shape[0], t.shape[1], ld
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def sp_launch_count() -> int:
+    return int(lib.sp_launch_count())
+
+
+def sp_la_for_sparsity(sparsity: float) -> float:
+    out = ctypes.c_float()
+    _check(lib.sp_la_for_sparsity(sparsity, ctypes.byref(out)))
+    return out.value
+
+
+class Context:
+    """Owns one ``sp_ctx`` (one layer input of ``d_in`` channels)."""
+
+    def __init__(self, d_in: int, device: int | None = None):
+        if device is None:
+            device = torch.cuda.current_device()
+        self.d_in = int(d_in)
+        self.device = int(device)
+        h = ctypes.c_void_p()
+        _check(lib.sp_create(ctypes.byref(h), self.d_in, self.device))
+        self._h = h
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib.sp_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    # -- calibration ---------------------------------------------------------
+    def sp_calib_reset(self, stream=None):
+        _check(lib.sp_calib_reset(self._h, _stream(stream)))
+
+    def sp_calib_accumulate(self, X: torch.Tensor, stream=None):
+        ptr, T, n, ld = _matrix(X, "X")
+        if n != self.d_in:
+            raise SpError(SP_ERR_SHAPE, "X has %d channels, context has %d" % (n, self.d_in))
+        _check(lib.sp_calib_accumulate(self._h, ptr, _dtype_of(X), T, ld, _stream(stream)))
+
+    def sp_get_stats(self, stream=None):
+        """Returns (colsq fp64 [d_in], S, factor fp32 [d_in], n_tokens) as CPU tensors/numbers."""
+        colsq = torch.empty(self.d_in, dtype=torch.float64)
+        factor = torch.empty(self.d_in, dtype=torch.float32)
+        S = ctypes.c_double()
+        ntok = ctypes.c_int64()
+        _check(lib.sp_get_stats(self._h, colsq.data_ptr(), ctypes.addressof(S), factor.data_ptr(),
+                                ctypes.byref(ntok), _stream(stream)))
+        return colsq, S.value, factor, ntok.value
+
+    def sp_set_stats(self, colsq: torch.Tensor, n_tokens: int, stream=None):
+        colsq = colsq.detach().to("cpu", torch.float64).contiguous()
+        if colsq.numel() != self.d_in:
+            raise SpError(SP_ERR_SHAPE, "colsq must have d_in entries")
+        _check(lib.sp_set_stats(self._h, colsq.data_ptr(), int(n_tokens), _stream(stream)))
+
+    # -- metric --------------------------------------------------------------
+    def sp_score(self, W: torch.Tensor | None = None, want_scores: bool = True, stream=None):
+        """Finalises the statistics; with W, returns the fp32 score matrix L (Eq. 8)."""
+        if W is None or not want_scores:
+            _check(lib.sp_score(self._h, None, SP_F16, 0, self.d_in, None, _stream(stream)))
+            return None
+        ptr, R, n, ld = _matrix(W, "W")
+        self._check_width(n)
+        scores = torch.empty(R, n, dtype=torch.float32, device=W.device)
+        _check(lib.sp_score(self._h, ptr, _dtype_of(W), R, ld, scores.data_ptr(), _stream(stream)))
+        return scores
+
+    def _check_width(self, n):
+        if n != self.d_in:
+            raise SpError(SP_ERR_SHAPE, "W has %d columns, context has %d" % (n, self.d_in))
+
+    def _outputs(self, W, mask, W_out, want_mask, inplace):
+        R, n = W.shape
+        if mask is None and want_mask:
+            mask = torch.empty(R, (n + 31) // 32, dtype=torch.int32, device=W.device)
+        if inplace:
+            W_out = W
+        elif W_out is None:
+            W_out = torch.empty_like(W)
+        return mask, W_out
+
+    # -- selection -----------------------------------------------------------
+    def sp_select_unstructured(self, W, sparsity=None, *, params: EwmaParams | None = None,
+                               mask=None, W_out=None, inplace=False, want_mask=True,
+                               counters=None, stream=None):
+        """Algorithm 1 on every row of W.  Returns (mask int32 [R, ceil(n/32)], W_out)."""
+        ptr, R, n, ld = _matrix(W, "W")
+        self._check_width(n)
+        mask, W_out = self._outputs(W, mask, W_out, want_mask, inplace)
+        optr, _, _, ldo = _matrix(W_out, "W_out")
+        if params is not None:
+            _check(lib.sp_select_unstructured_ex(self._h, ptr, _dtype_of(W), R, ld,
+                                                 ctypes.byref(params), _ptr(mask), optr, ldo,
+                                                 _ptr(counters), _stream(stream)))
+        else:
+            _check(lib.sp_select_unstructured(self._h, ptr, _dtype_of(W), R, ld, float(sparsity),
+                                              _ptr(mask), optr, ldo, _ptr(counters),
+                                              _stream(stream)))
+        return mask, W_out
+
+    def sp_select_nm(self, W, N: int, M: int, *, mask=None, W_out=None, inplace=False,
+                     want_mask=True, stream=None):
+        """N:M selection (keep N of every M).  Returns (mask, W_out)."""
+        ptr, R, n, ld = _matrix(W, "W")
+        self._check_width(n)
+        mask, W_out = self._outputs(W, mask, W_out, want_mask, inplace)
+        optr, _, _, ldo = _matrix(W_out, "W_out")
+        _check(lib.sp_select_nm(self._h, ptr, _dtype_of(W), R, ld, int(N), int(M), _ptr(mask),
+                                optr, ldo, _stream(stream)))
+        return mask, W_out
+
+
+def sp_apply_mask(W: torch.Tensor, mask: torch.Tensor, W_out: torch.Tensor | None = None,
+                  stream=None) -> torch.Tensor:
+    ptr, R, n, ld = _matrix(W, "W")
+    if W_out is None:
+        W_out = torch.empty_like(W)
+    optr, _, _, ldo = _matrix(W_out, "W_out")
+    if mask.dim() != 2 or tuple(mask.shape) != (R, (n + 31) // 32) or not mask.is_contiguous():
+        raise SpError(SP_ERR_SHAPE, "mask must be contiguous [rows, ceil(cols/32)]")
+    _check(lib.sp_apply_mask(ptr, _dtype_of(W), R, n, ld, mask.data_ptr(), optr, ldo,
+                             _stream(stream)))
+    return W_out
+
+
+def new_counters(device=None) -> torch.Tensor:
+    """Zeroed device counter block for the selection calls (int64 view of the uint64 pair)."""
+    return torch.zeros(SP_NUM_COUNTERS, dtype=torch.int64, device=device or "cuda")

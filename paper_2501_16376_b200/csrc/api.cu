@@ -1,0 +1,318 @@
+// C ABI of the library: argument validation on the host, context management, dispatch to
+// the kernel launchers.  Nothing here synchronises unless the header says so.
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "sp_internal.h"
+
+namespace sp {
+
+static thread_local char g_cuda_error[256] = "";
+static std::atomic<uint64_t> g_launches{0};
+
+sp_status cuda_fail(cudaError_t e) {
+    snprintf(g_cuda_error, sizeof g_cuda_error, "%s: %s", cudaGetErrorName(e),
+             cudaGetErrorString(e));
+    return e == cudaErrorMemoryAllocation ? SP_ERR_NOMEM : SP_ERR_CUDA;
+}
+
+void count_launch(int n) { g_launches.fetch_add(static_cast<uint64_t>(n)); }
+
+// Makes the context's device current for the scope of one call.
+class DeviceGuard {
+   public:
+    explicit DeviceGuard(int device) {
+        if (cudaGetDevice(&prev_) != cudaSuccess) prev_ = -1;
+        if (prev_ != device) {
+            err_ = cudaSetDevice(device);
+            switched_ = err_ == cudaSuccess;
+        }
+    }
+    ~DeviceGuard() {
+        if (switched_ && prev_ >= 0) cudaSetDevice(prev_);
+    }
+    cudaError_t error() const { return err_; }
+
+   private:
+    int prev_ = -1;
+    bool switched_ = false;
+    cudaError_t err_ = cudaSuccess;
+};
+
+static bool valid_dtype(sp_dtype d) { return d == SP_F16 || d == SP_BF16; }
+
+static sp_status ensure_finalized(sp_ctx *ctx, cudaStream_t stream) {
+    if (ctx->n_tokens <= 0) return SP_ERR_STATE;
+    if (!ctx->dirty) return SP_OK;
+    return launch_finalize(ctx, stream);
+}
+
+static sp_status check_matrix_args(const sp_ctx *ctx, const void *W, sp_dtype dtype,
+                                   int64_t n_rows, int64_t ldw, const void *W_out, int64_t ldo) {
+    if (ctx == nullptr || W == nullptr) return SP_ERR_INVALID_ARG;
+    if (!valid_dtype(dtype)) return SP_ERR_DTYPE;
+    if (n_rows < 0) return SP_ERR_INVALID_ARG;
+    if (ldw < ctx->d_in) return SP_ERR_SHAPE;
+    if (W_out != nullptr) {
+        if (ldo < ctx->d_in) return SP_ERR_SHAPE;
+        if (W_out == W && ldo != ldw) return SP_ERR_SHAPE;
+    }
+    return SP_OK;
+}
+
+}  // namespace sp
+
+using namespace sp;
+
+extern "C" {
+
+sp_status sp_create(sp_ctx **out, int64_t d_in, int device) {
+    if (out == nullptr) return SP_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (d_in < 1 || d_in > kMaxDin) return SP_ERR_SHAPE;
+    int count = 0;
+    cudaError_t e = cudaGetDeviceCount(&count);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (device < 0 || device >= count) return SP_ERR_INVALID_ARG;
+    DeviceGuard guard(device);
+    if (guard.error() != cudaSuccess) return cuda_fail(guard.error());
+
+    sp_ctx *ctx = new (std::nothrow) sp_ctx();
+    if (ctx == nullptr) return SP_ERR_NOMEM;
+    ctx->device = device;
+    ctx->d_in = d_in;
+    ctx->n_pad = (d_in + kStripChannels - 1) / kStripChannels * kStripChannels;
+    ctx->strips = static_cast<int>(ctx->n_pad / kStripChannels);
+    ctx->n_tokens = 0;
+    ctx->slabs_valid = 0;
+    ctx->dirty = false;
+    e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
+    if (e != cudaSuccess) { delete ctx; return cuda_fail(e); }
+    ctx->calib_blocks_per_sm = calib_query_blocks_per_sm();
+
+    const size_t np = static_cast<size_t>(ctx->n_pad);
+    void *ptrs[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+    const size_t sizes[5] = {sizeof(double) * np * kMaxSlabs, sizeof(double) * np,
+                             sizeof(double) * static_cast<size_t>(ctx->strips), sizeof(float) * np,
+                             sizeof(DeviceScalars)};
+    for (int i = 0; i < 5; ++i) {
+        e = cudaMalloc(&ptrs[i], sizes[i]);
+        if (e == cudaSuccess) e = cudaMemset(ptrs[i], 0, sizes[i]);
+        if (e != cudaSuccess) {
+            for (int j = 0; j <= i; ++j) cudaFree(ptrs[j]);
+            delete ctx;
+            return cuda_fail(e);
+        }
+    }
+    ctx->partial = static_cast<double *>(ptrs[0]);
+    ctx->colsq = static_cast<double *>(ptrs[1]);
+    ctx->strip_sum = static_cast<double *>(ptrs[2]);
+    ctx->factor = static_cast<float *>(ptrs[3]);
+    ctx->scalars = static_cast<DeviceScalars *>(ptrs[4]);
+    e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) { sp_destroy(ctx); return cuda_fail(e); }
+    *out = ctx;
+    return SP_OK;
+}
+
+sp_status sp_destroy(sp_ctx *ctx) {
+    if (ctx == nullptr) return SP_OK;
+    DeviceGuard guard(ctx->device);
+    cudaDeviceSynchronize();
+    cudaFree(ctx->partial);
+    cudaFree(ctx->colsq);
+    cudaFree(ctx->strip_sum);
+    cudaFree(ctx->factor);
+    cudaFree(ctx->scalars);
+    delete ctx;
+    return SP_OK;
+}
+
+sp_status sp_calib_reset(sp_ctx *ctx, sp_stream stream) {
+    (void)stream;  // the partial sums are overwritten, not cleared, by the next batch
+    if (ctx == nullptr) return SP_ERR_INVALID_ARG;
+    ctx->n_tokens = 0;
+    ctx->slabs_valid = 0;
+    ctx->dirty = false;
+    return SP_OK;
+}
+
+sp_status sp_calib_accumulate(sp_ctx *ctx, const void *X, sp_dtype dtype, int64_t n_tokens,
+                              int64_t ldx, sp_stream stream) {
+    if (ctx == nullptr) return SP_ERR_INVALID_ARG;
+    if (!valid_dtype(dtype)) return SP_ERR_DTYPE;
+    if (n_tokens < 0) return SP_ERR_INVALID_ARG;
+    if (n_tokens == 0) return SP_OK;
+    if (X == nullptr) return SP_ERR_INVALID_ARG;
+    if (ldx < ctx->d_in) return SP_ERR_SHAPE;
+    DeviceGuard guard(ctx->device);
+    if (guard.error() != cudaSuccess) return cuda_fail(guard.error());
+    return launch_calib_accumulate(ctx, X, dtype, n_tokens, ldx, static_cast<cudaStream_t>(stream));
+}
+
+sp_status sp_get_stats(sp_ctx *ctx, double *colsq_host, double *S_host, float *factor_host,
+                       int64_t *n_tokens_host, sp_stream stream) {
+    if (ctx == nullptr) return SP_ERR_INVALID_ARG;
+    if (n_tokens_host != nullptr) *n_tokens_host = ctx->n_tokens;
+    if (ctx->n_tokens <= 0) return SP_ERR_STATE;
+    DeviceGuard guard(ctx->device);
+    if (guard.error() != cudaSuccess) return cuda_fail(guard.error());
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    sp_status st = ensure_finalized(ctx, s);
+    if (st != SP_OK) return st;
+    DeviceScalars sc;
+    cudaError_t e = cudaMemcpyAsync(&sc, ctx->scalars, sizeof sc, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess && colsq_host != nullptr)
+        e = cudaMemcpyAsync(colsq_host, ctx->colsq, sizeof(double) * ctx->d_in,
+                            cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess && factor_host != nullptr)
+        e = cudaMemcpyAsync(factor_host, ctx->factor, sizeof(float) * ctx->d_in,
+                            cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (S_host != nullptr) *S_host = sc.S;
+    return (sc.flags & kFlagDegenerate) ? SP_ERR_DEGENERATE : SP_OK;
+}
+
+sp_status sp_set_stats(sp_ctx *ctx, const double *colsq_host, int64_t n_tokens, sp_stream stream) {
+    if (ctx == nullptr || colsq_host == nullptr || n_tokens <= 0) return SP_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (guard.error() != cudaSuccess) return cuda_fail(guard.error());
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // The statistics become slab row 0 of the partial sums; the padding stays zero.
+    cudaError_t e = cudaMemsetAsync(ctx->partial, 0, sizeof(double) * ctx->n_pad, s);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(ctx->partial, colsq_host, sizeof(double) * ctx->d_in,
+                            cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    ctx->n_tokens = n_tokens;
+    ctx->slabs_valid = 1;
+    ctx->dirty = true;
+    return SP_OK;
+}
+
+sp_status sp_score(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows, int64_t ldw,
+                   float *scores_out, sp_stream stream) {
+    if (ctx == nullptr) return SP_ERR_INVALID_ARG;
+    if (scores_out != nullptr) {
+        sp_status st = check_matrix_args(ctx, W, dtype, n_rows, ldw, nullptr, 0);
+        if (st != SP_OK) return st;
+    }
+    if (ctx->n_tokens <= 0) return SP_ERR_STATE;
+    DeviceGuard guard(ctx->device);
+    if (guard.error() != cudaSuccess) return cuda_fail(guard.error());
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    sp_status st = ensure_finalized(ctx, s);
+    if (st != SP_OK || scores_out == nullptr) return st;
+    return launch_score(ctx, W, dtype, n_rows, ldw, scores_out, s);
+}
+
+sp_status sp_la_for_sparsity(float sparsity, float *la_out) {
+    if (la_out == nullptr || !(sparsity > 0.0f) || !(sparsity < 1.0f)) return SP_ERR_INVALID_ARG;
+    // Table 3: pruning ratio (%) -> la.
+    static const double pct[5] = {50.0, 60.0, 70.0, 80.0, 90.0};
+    static const double la[5] = {0.5, 0.2, -0.2, -0.9, -1.5};
+    const double x = static_cast<double>(sparsity) * 100.0;
+    for (int i = 0; i < 5; ++i) {
+        if (std::fabs(x - pct[i]) < 1e-4) {
+            *la_out = static_cast<float>(la[i]);
+            return SP_OK;
+        }
+    }
+    int i = 0;
+    if (x >= pct[4]) {
+        i = 3;
+    } else {
+        while (i < 3 && x >= pct[i + 1]) ++i;
+    }
+    const double t = (x - pct[i]) / (pct[i + 1] - pct[i]);
+    *la_out = static_cast<float>(la[i] + t * (la[i + 1] - la[i]));
+    return SP_OK;
+}
+
+sp_status sp_select_unstructured_ex(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
+                                    int64_t ldw, const sp_ewma_params *params, uint32_t *mask_out,
+                                    void *W_out, int64_t ldo, unsigned long long *counters,
+                                    sp_stream stream) {
+    sp_status st = check_matrix_args(ctx, W, dtype, n_rows, ldw, W_out, ldo);
+    if (st != SP_OK) return st;
+    if (params == nullptr) return SP_ERR_INVALID_ARG;
+    if (!(params->alpha > 0.0f) || !(params->alpha <= 1.0f) || !(params->beta > 0.0f) ||
+        !(params->beta <= 1.0f) || !std::isfinite(params->la))
+        return SP_ERR_INVALID_ARG;
+    if (params->s_update != SP_S_FROZEN && params->s_update != SP_S_LITERAL_W2)
+        return SP_ERR_INVALID_ARG;
+    if (ctx->n_tokens <= 0) return SP_ERR_STATE;
+    DeviceGuard guard(ctx->device);
+    if (guard.error() != cudaSuccess) return cuda_fail(guard.error());
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    st = ensure_finalized(ctx, s);
+    if (st != SP_OK) return st;
+    return launch_select_ewma(ctx, W, dtype, n_rows, ldw, *params, mask_out, W_out, ldo, counters, s);
+}
+
+sp_status sp_select_unstructured(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
+                                 int64_t ldw, float sparsity, uint32_t *mask_out, void *W_out,
+                                 int64_t ldo, unsigned long long *counters, sp_stream stream) {
+    sp_ewma_params p;
+    p.alpha = 0.125f;  // Section 4.2
+    p.beta = 0.125f;
+    p.s_update = SP_S_FROZEN;
+    sp_status st = sp_la_for_sparsity(sparsity, &p.la);
+    if (st != SP_OK) return st;
+    return sp_select_unstructured_ex(ctx, W, dtype, n_rows, ldw, &p, mask_out, W_out, ldo, counters,
+                                     stream);
+}
+
+sp_status sp_select_nm(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows, int64_t ldw,
+                       int N, int M, uint32_t *mask_out, void *W_out, int64_t ldo,
+                       sp_stream stream) {
+    sp_status st = check_matrix_args(ctx, W, dtype, n_rows, ldw, W_out, ldo);
+    if (st != SP_OK) return st;
+    if (M != 4 && M != 8) return SP_ERR_INVALID_ARG;
+    if (N <= 0 || N >= M) return SP_ERR_INVALID_ARG;
+    if (ctx->d_in % M != 0) return SP_ERR_SHAPE;
+    if (ctx->n_tokens <= 0) return SP_ERR_STATE;
+    DeviceGuard guard(ctx->device);
+    if (guard.error() != cudaSuccess) return cuda_fail(guard.error());
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    st = ensure_finalized(ctx, s);
+    if (st != SP_OK) return st;
+    return launch_select_nm(ctx, W, dtype, n_rows, ldw, N, M, mask_out, W_out, ldo, s);
+}
+
+sp_status sp_apply_mask(const void *W, sp_dtype dtype, int64_t n_rows, int64_t n_cols, int64_t ldw,
+                        const uint32_t *mask, void *W_out, int64_t ldo, sp_stream stream) {
+    if (W == nullptr || mask == nullptr || W_out == nullptr) return SP_ERR_INVALID_ARG;
+    if (!valid_dtype(dtype)) return SP_ERR_DTYPE;
+    if (n_rows < 0 || n_cols < 0) return SP_ERR_INVALID_ARG;
+    if (ldw < n_cols || ldo < n_cols) return SP_ERR_SHAPE;
+    if (W_out == W && ldo != ldw) return SP_ERR_SHAPE;
+    return launch_apply_mask(W, dtype, n_rows, n_cols, ldw, mask, W_out, ldo,
+                             static_cast<cudaStream_t>(stream));
+}
+
+const char *sp_status_string(sp_status status) {
+    switch (status) {
+        case SP_OK: return "ok";
+        case SP_ERR_INVALID_ARG: return "invalid argument";
+        case SP_ERR_SHAPE: return "invalid shape or leading dimension";
+        case SP_ERR_DTYPE: return "unsupported dtype";
+        case SP_ERR_STATE: return "no calibration statistics accumulated";
+        case SP_ERR_DEGENERATE: return "degenerate calibration statistics (S is zero or not finite)";
+        case SP_ERR_CUDA: return "CUDA runtime error";
+        case SP_ERR_NOMEM: return "out of memory";
+    }
+    return "unknown status";
+}
+
+const char *sp_last_cuda_error(void) { return g_cuda_error; }
+
+uint64_t sp_launch_count(void) { return g_launches.load(); }
+
+}  // extern "C"

@@ -1,0 +1,207 @@
+// Calibration statistics (Algorithm 1, step 1): streaming column sums of squares over the
+// tokens x d_in activations, and the finalisation that turns them into S and the
+// per-channel factor of Eq. 8.
+//
+// Layout of the work: the channel axis is cut into strips of 256 channels (one warp-wide
+// 16-byte load per activation row), the token axis into slabs.  One CTA owns one
+// (strip, slab) cell; its 8 warps take rows slab_begin + warp, + 8, ... and keep 8 rows in
+// flight per lane.  Squares are exact in fp32; the sum of the 8 in-flight squares is formed in
+// fp32 and added to an fp64 accumulator.  The CTA adds its 256 sums to row `slab` of the
+// partial-sum array, which no other CTA touches: there are no floating-point atomics, so the
+// statistics are reproducible bit for bit for a given sequence of batches.
+#include "sp_device.cuh"
+#include "sp_internal.h"
+
+namespace sp {
+
+constexpr int kCalibThreads = 256;
+constexpr int kCalibWarps = kCalibThreads / 32;
+constexpr int kRowsInFlight = 8;
+
+template <bool BF16, bool VEC>
+__global__ void __launch_bounds__(kCalibThreads)
+calib_accumulate_kernel(const uint16_t *__restrict__ X, int64_t ldx, int64_t n_tokens, int64_t n,
+                        int64_t rows_per_slab, double *__restrict__ partial, int64_t n_pad,
+                        int first_fresh_slab) {
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int strip = blockIdx.x;
+    const int slab = blockIdx.y;
+    const int64_t col = static_cast<int64_t>(strip) * kStripChannels + lane * 8;
+    const int64_t row_begin = static_cast<int64_t>(slab) * rows_per_slab;
+    const int64_t row_end = min(n_tokens, row_begin + rows_per_slab);
+
+    double acc[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j] = 0.0;
+
+    for (int64_t r = row_begin + warp; r < row_end; r += kCalibWarps * kRowsInFlight) {
+        uint32_t v[kRowsInFlight][4];
+#pragma unroll
+        for (int u = 0; u < kRowsInFlight; ++u) {
+            const int64_t rr = r + static_cast<int64_t>(u) * kCalibWarps;
+            if (rr < row_end) {
+                load8<VEC, true>(X + rr * ldx, col, n, v[u]);
+            } else {
+                v[u][0] = v[u][1] = v[u][2] = v[u][3] = 0u;
+            }
+        }
+        float s[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) s[j] = 0.0f;
+#pragma unroll
+        for (int u = 0; u < kRowsInFlight; ++u) {
+            float x[8];
+            unpack8<BF16>(v[u], x);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) s[j] = fmaf(x[j], x[j], s[j]);
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[j] += static_cast<double>(s[j]);
+    }
+
+    // Combine the 8 warps in a fixed order, then add to this cell's row of `partial`.
+    __shared__ double sm[kCalibWarps][kStripChannels];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) sm[warp][lane * 8 + j] = acc[j];
+    __syncthreads();
+    const int t = threadIdx.x;
+    const int64_t ch = static_cast<int64_t>(strip) * kStripChannels + t;
+    if (ch < n) {
+        double sum = 0.0;
+#pragma unroll
+        for (int w = 0; w < kCalibWarps; ++w) sum += sm[w][t];
+        double *dst = partial + static_cast<int64_t>(slab) * n_pad + ch;
+        if (slab >= first_fresh_slab)
+            *dst = sum;
+        else
+            *dst += sum;
+    }
+}
+
+// Finalisation.  CTA `strip` sums its 256 channels over the valid slab rows (ascending slab
+// order), writes colsq and its strip total; the last CTA to arrive adds the strip totals in
+// ascending order to S and writes the per-channel factor for every channel:
+//     u = colsq32 / S32 ;  den = 1 - u ;  c = 0.5 / den          (binary32, round to nearest)
+// No CTA waits for another one (the last arrival does the tail), so the kernel cannot hang.
+__global__ void __launch_bounds__(kStripChannels)
+finalize_kernel(const double *__restrict__ partial, int slabs_valid, int64_t n, int64_t n_pad,
+                int strips, double *__restrict__ colsq, double *__restrict__ strip_sum,
+                float *__restrict__ factor, DeviceScalars *__restrict__ scalars) {
+    __shared__ double red[kStripChannels];
+    __shared__ bool is_last;
+    const int t = threadIdx.x;
+    const int64_t ch = static_cast<int64_t>(blockIdx.x) * kStripChannels + t;
+    double v = 0.0;
+    if (ch < n) {
+        for (int s = 0; s < slabs_valid; ++s) v += partial[static_cast<int64_t>(s) * n_pad + ch];
+    }
+    colsq[ch] = v;  // ch < n_pad always; padding gets 0
+    red[t] = v;
+    __syncthreads();
+    for (int half = kStripChannels / 2; half > 0; half >>= 1) {
+        if (t < half) red[t] += red[t + half];
+        __syncthreads();
+    }
+    if (t == 0) {
+        strip_sum[blockIdx.x] = red[0];
+        __threadfence();
+        unsigned int ticket = atomicAdd(&scalars->ticket, 1u);
+        is_last = (ticket == static_cast<unsigned int>(strips) - 1u);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+
+    __shared__ double S_sh;
+    if (t == 0) {
+        double S = 0.0;
+        for (int s = 0; s < strips; ++s) S += __ldcg(strip_sum + s);
+        const float S32 = static_cast<float>(S);
+        int flags = 0;
+        if (!(S > 0.0) || isinf(S) || isnan(S) || isinf(S32)) flags |= kFlagDegenerate;
+        // "S - w^2" leaves S unchanged in binary32 whenever w^2 is below a quarter of the
+        // spacing of floats at S: 2^(e-25) for S in [2^e, 2^(e+1)).
+        float hazard = 0.0f;
+        if (!flags) {
+            const int e = static_cast<int>((__float_as_uint(S32) >> 23) & 0xffu);
+            hazard = e > 25 ? __uint_as_float(static_cast<uint32_t>(e - 25) << 23) : 0.0f;
+        }
+        scalars->S = S;
+        scalars->S32 = S32;
+        scalars->hazard_w2 = hazard;
+        scalars->flags = flags;
+        scalars->ticket = 0u;
+        S_sh = S;
+    }
+    __syncthreads();
+    const float S32 = static_cast<float>(S_sh);
+    for (int64_t q = t; q < n_pad; q += kStripChannels) {
+        float c = 0.0f;
+        if (q < n) {
+            const float x2 = static_cast<float>(__ldcg(colsq + q));
+            const float u = __fdiv_rn(x2, S32);
+            const float den = __fsub_rn(1.0f, u);
+            c = __fdiv_rn(0.5f, den);
+        }
+        factor[q] = c;
+    }
+}
+
+template <bool BF16, bool VEC>
+static int query_blocks_per_sm() {
+    int blocks = 0;
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+        &blocks, calib_accumulate_kernel<BF16, VEC>, kCalibThreads, 0);
+    if (e != cudaSuccess || blocks < 1) blocks = 1;
+    return blocks;
+}
+
+int calib_query_blocks_per_sm() { return query_blocks_per_sm<false, true>(); }
+
+sp_status launch_calib_accumulate(sp_ctx *ctx, const void *X, sp_dtype dtype, int64_t n_tokens,
+                                  int64_t ldx, cudaStream_t stream) {
+    const int64_t n = ctx->d_in;
+    // One resident wave: strips x slabs CTAs fill the GPU once, every CTA gets the same rows.
+    const int64_t resident = static_cast<int64_t>(ctx->sm_count) * ctx->calib_blocks_per_sm;
+    int64_t slabs = resident / ctx->strips;
+    if (slabs < 1) slabs = 1;
+    if (slabs > kMaxSlabs) slabs = kMaxSlabs;
+    const int64_t min_rows = kCalibWarps * kRowsInFlight;  // at least one full step per warp
+    int64_t max_slabs_by_rows = (n_tokens + min_rows - 1) / min_rows;
+    if (slabs > max_slabs_by_rows) slabs = max_slabs_by_rows;
+    int64_t rows_per_slab = (n_tokens + slabs - 1) / slabs;
+    rows_per_slab = (rows_per_slab + kCalibWarps - 1) / kCalibWarps * kCalibWarps;
+    slabs = (n_tokens + rows_per_slab - 1) / rows_per_slab;
+
+    const bool vec = aligned16(X) && (ldx % 8 == 0) && (n % 8 == 0);
+    const bool bf16 = dtype == SP_BF16;
+    dim3 grid(static_cast<unsigned>(ctx->strips), static_cast<unsigned>(slabs));
+    const uint16_t *Xp = static_cast<const uint16_t *>(X);
+#define SP_LAUNCH(B, V)                                                                       \
+    calib_accumulate_kernel<B, V><<<grid, kCalibThreads, 0, stream>>>(                        \
+        Xp, ldx, n_tokens, n, rows_per_slab, ctx->partial, ctx->n_pad, ctx->slabs_valid)
+    if (bf16) {
+        if (vec) SP_LAUNCH(true, true); else SP_LAUNCH(true, false);
+    } else {
+        if (vec) SP_LAUNCH(false, true); else SP_LAUNCH(false, false);
+    }
+#undef SP_LAUNCH
+    sp_status st = check_launch();
+    if (st != SP_OK) return st;
+    if (slabs > ctx->slabs_valid) ctx->slabs_valid = static_cast<int>(slabs);
+    ctx->n_tokens += n_tokens;
+    ctx->dirty = true;
+    return SP_OK;
+}
+
+sp_status launch_finalize(sp_ctx *ctx, cudaStream_t stream) {
+    finalize_kernel<<<ctx->strips, kStripChannels, 0, stream>>>(
+        ctx->partial, ctx->slabs_valid, ctx->d_in, ctx->n_pad, ctx->strips, ctx->colsq,
+        ctx->strip_sum, ctx->factor, ctx->scalars);
+    sp_status st = check_launch();
+    if (st == SP_OK) ctx->dirty = false;
+    return st;
+}
+
+}  // namespace sp

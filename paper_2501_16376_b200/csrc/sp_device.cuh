@@ -1,0 +1,109 @@
+// Device-side helpers: 16-bit float decoding, 8-element vector access with ragged tails,
+// mask-word assembly.  Every kernel of the library views a row as chunks of 8 consecutive
+// elements (16 bytes) owned by one lane; a warp covers a 256-element tile.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace sp {
+
+constexpr unsigned kFullWarp = 0xffffffffu;
+
+// Two packed 16-bit floats -> two fp32 values (exact).
+template <bool BF16>
+__device__ __forceinline__ float2 unpack2(uint32_t u) {
+    if constexpr (BF16) {
+        return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u));
+    } else {
+        __half2 h = *reinterpret_cast<__half2 *>(&u);
+        return __half22float2(h);
+    }
+}
+
+template <bool BF16>
+__device__ __forceinline__ void unpack8(const uint32_t (&p)[4], float (&w)[8]) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        float2 f = unpack2<BF16>(p[k]);
+        w[2 * k] = f.x;
+        w[2 * k + 1] = f.y;
+    }
+}
+
+// Loads elements [col, col+8) of a row into four packed words; elements at or past n read
+// as zero.  VEC: 16-byte access (requires 16-byte aligned row start, n % 8 == 0, col % 8 == 0).
+// STREAM: the data is read once (bypass L1, evict-first behaviour).
+template <bool VEC, bool STREAM>
+__device__ __forceinline__ void load8(const uint16_t *__restrict__ row, int64_t col, int64_t n,
+                                      uint32_t (&p)[4]) {
+    if constexpr (VEC) {
+        if (col < n) {
+            const uint4 *src = reinterpret_cast<const uint4 *>(row + col);
+            uint4 v = STREAM ? __ldcs(src) : __ldg(src);
+            p[0] = v.x; p[1] = v.y; p[2] = v.z; p[3] = v.w;
+        } else {
+            p[0] = p[1] = p[2] = p[3] = 0u;
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            uint32_t lo = 0, hi = 0;
+            if (col + 2 * k < n) lo = row[col + 2 * k];
+            if (col + 2 * k + 1 < n) hi = row[col + 2 * k + 1];
+            p[k] = lo | (hi << 16);
+        }
+    }
+}
+
+template <bool VEC>
+__device__ __forceinline__ void store8(uint16_t *__restrict__ row, int64_t col, int64_t n,
+                                       const uint32_t (&p)[4]) {
+    if constexpr (VEC) {
+        if (col < n) {
+            uint4 v = make_uint4(p[0], p[1], p[2], p[3]);
+            __stcs(reinterpret_cast<uint4 *>(row + col), v);
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            if (col + 2 * k < n) row[col + 2 * k] = static_cast<uint16_t>(p[k] & 0xffffu);
+            if (col + 2 * k + 1 < n) row[col + 2 * k + 1] = static_cast<uint16_t>(p[k] >> 16);
+        }
+    }
+}
+
+// Eight per-channel factors for columns [col, col+8); the factor array is padded with zeros
+// to a multiple of 256 entries, so the 16-byte loads never leave it.
+__device__ __forceinline__ void load_factor8(const float *__restrict__ factor, int64_t col,
+                                             float (&c)[8]) {
+    const float4 *src = reinterpret_cast<const float4 *>(factor + col);
+    float4 a = __ldg(src);
+    float4 b = __ldg(src + 1);
+    c[0] = a.x; c[1] = a.y; c[2] = a.z; c[3] = a.w;
+    c[4] = b.x; c[5] = b.y; c[6] = b.z; c[7] = b.w;
+}
+
+// Zeroes the 16-bit halves of the packed words whose keep bit (bit j of `keep`, j = element
+// index within the chunk) is clear.
+__device__ __forceinline__ void zero_pruned(uint32_t (&p)[4], uint32_t keep) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        uint32_t m = ((keep >> (2 * k)) & 1u ? 0x0000ffffu : 0u) |
+                     ((keep >> (2 * k + 1)) & 1u ? 0xffff0000u : 0u);
+        p[k] &= m;
+    }
+}
+
+// Each lane holds the 8 keep bits of its chunk.  Returns, in lanes with (lane & 3) == 0, the
+// 32-bit mask word covering the chunks of lanes lane .. lane+3.
+__device__ __forceinline__ uint32_t gather_mask_word(uint32_t keep8, int lane) {
+    uint32_t v = keep8 << (8 * (lane & 3));
+    v |= __shfl_xor_sync(kFullWarp, v, 1);
+    v |= __shfl_xor_sync(kFullWarp, v, 2);
+    return v;
+}
+
+}  // namespace sp

@@ -1,0 +1,97 @@
+// Internal declarations shared by the translation units of the library.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "swiftprune.h"
+
+namespace sp {
+
+constexpr int kStripChannels = 256;  // channels covered by one warp-wide 16-byte load
+constexpr int kMaxSlabs = 128;       // token slabs that own a row of partial sums
+constexpr int kTile = 256;           // weights per warp tile (32 lanes x 8)
+constexpr int64_t kMaxDin = 1 << 20;
+
+// Status word written by the finalisation kernel.
+constexpr int kFlagDegenerate = 1;
+
+// Scalars produced by finalisation; lives in device memory inside the context.
+struct DeviceScalars {
+    double S;             // sum_q colsq[q]
+    float S32;            // (float)S
+    float hazard_w2;      // a weight with w^2 >= this could change S in "S - w^2" (binary32)
+    int flags;            // kFlag*
+    unsigned int ticket;  // arrival counter of the finalisation kernel (returns to 0)
+};
+
+// Powers of (1-alpha) and (1-beta) that the scan kernel needs, computed on the host in
+// fp64 and rounded once.
+struct ScanConstants {
+    float alpha, beta, la;
+    float a, b;            // 1-alpha, 1-beta (rounded in fp32 like the definition)
+    float a_pow[8];        // a^(j+1)
+    float b_pow[8];
+    float a_lane[32];      // a^(8*lane)
+    float b_lane[32];
+    float a_step[5];       // a^(8*2^k)
+    float b_step[5];
+};
+
+}  // namespace sp
+
+struct sp_ctx {
+    int device;
+    int sm_count;
+    int64_t d_in;
+    int64_t n_pad;             // d_in rounded up to a multiple of kStripChannels
+    int strips;                // n_pad / kStripChannels
+    int64_t n_tokens;          // host-side count
+    int slabs_valid;           // slab rows of `partial` that hold data
+    bool dirty;                // batches arrived since the last finalisation
+    int calib_blocks_per_sm;   // measured occupancy of the accumulation kernel
+    double *partial;           // [kMaxSlabs][n_pad] fp64 partial column sums
+    double *colsq;             // [n_pad]
+    double *strip_sum;         // [strips]
+    float *factor;             // [n_pad] c_q, zero in the padding
+    sp::DeviceScalars *scalars;
+};
+
+namespace sp {
+
+// Thread-local CUDA error text and the global launch counter (api.cu).
+sp_status cuda_fail(cudaError_t e);
+void count_launch(int n = 1);
+inline sp_status check_launch() {
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e);
+    count_launch();
+    return SP_OK;
+}
+
+// calib.cu
+int calib_query_blocks_per_sm();
+sp_status launch_calib_accumulate(sp_ctx *ctx, const void *X, sp_dtype dtype, int64_t n_tokens,
+                                  int64_t ldx, cudaStream_t stream);
+sp_status launch_finalize(sp_ctx *ctx, cudaStream_t stream);
+
+// elementwise.cu
+sp_status launch_score(const sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
+                       int64_t ldw, float *scores, cudaStream_t stream);
+sp_status launch_apply_mask(const void *W, sp_dtype dtype, int64_t n_rows, int64_t n_cols,
+                            int64_t ldw, const uint32_t *mask, void *W_out, int64_t ldo,
+                            cudaStream_t stream);
+
+// select_nm.cu
+sp_status launch_select_nm(const sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
+                           int64_t ldw, int N, int M, uint32_t *mask, void *W_out, int64_t ldo,
+                           cudaStream_t stream);
+
+// select_ewma.cu
+sp_status launch_select_ewma(const sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
+                             int64_t ldw, const sp_ewma_params &p, uint32_t *mask, void *W_out,
+                             int64_t ldo, unsigned long long *counters, cudaStream_t stream);
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace sp

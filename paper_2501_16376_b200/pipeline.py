@@ -1,0 +1,119 @@
+"""Whole-model driver: walks the linear layers of a synthetic model and issues the library's
+calls for each (calibration batches -> selection fused with write-back).  Pure call sequencing
+and buffer bookkeeping; all arithmetic happens inside the CUDA library.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+
+import torch
+
+from . import binding as sp
+from . import synth
+
+
+@dataclass
+class ModelBuffers:
+    """Device-resident tensors of one synthetic model (one rank's unit of work)."""
+    workload: synth.Workload
+    device: torch.device
+    weights: list = field(default_factory=list)   # [block][layer] -> W
+    outputs: list = field(default_factory=list)   # [block][layer] -> W_out
+    masks: list = field(default_factory=list)     # [block][layer] -> mask
+    acts: dict = field(default_factory=dict)      # input name -> X [tokens, d_in] (shared by blocks)
+    ctxs: dict = field(default_factory=dict)      # input name -> Context
+
+    def close(self):
+        for c in self.ctxs.values():
+            c.close()
+        self.ctxs.clear()
+
+
+def allocate_model(w: synth.Workload, device, model_seed_offset: int = 0,
+                   distinct_acts: bool = True) -> ModelBuffers:
+    """Generates all weights of the workload and one set of calibration activations (the
+    activations of block 0, reused for every block: 128 x 2048 tokens for every block of a
+    7B-shaped model would not fit in device memory at once)."""
+    device = torch.device(device)
+    wl = w if model_seed_offset == 0 else synth.Workload(
+        **{**w.__dict__, "seed": w.seed + model_seed_offset})
+    mb = ModelBuffers(wl, device)
+    for b in range(wl.blocks):
+        ws, outs, ms = [], [], []
+        for layer in wl.layers:
+            W = synth.gen_weight(wl, b, layer, device)
+            ws.append(W)
+            outs.append(torch.empty_like(W))
+            ms.append(torch.empty(layer.d_out, (layer.d_in + 31) // 32, dtype=torch.int32,
+                                  device=device))
+        mb.weights.append(ws)
+        mb.outputs.append(outs)
+        mb.masks.append(ms)
+    by_width = {}
+    for name, d_in in wl.input_widths().items():
+        if not distinct_acts and d_in in by_width:
+            mb.acts[name] = by_width[d_in]
+        else:
+            X = torch.empty(wl.tokens, d_in, dtype=wl.torch_dtype, device=device)
+            step = max(1, min(8, wl.n_seqs))
+            for s in range(0, wl.n_seqs, step):
+                k = min(step, wl.n_seqs - s)
+                synth.gen_activations(wl, 0, name, d_in, s, k, device,
+                                      out=X[s * wl.seq_len:(s + k) * wl.seq_len])
+            mb.acts[name] = X
+            by_width[d_in] = X
+        mb.ctxs[name] = sp.Context(d_in, device.index if device.index is not None
+                                   else torch.cuda.current_device())
+    return mb
+
+
+def calibrate_input(ctx: sp.Context, X: torch.Tensor, batch_tokens: int, stream=None) -> int:
+    """Streams X through sp_calib_accumulate in batches; returns the number of launches."""
+    ctx.sp_calib_reset(stream)
+    T = X.shape[0]
+    launches = 0
+    for t0 in range(0, T, batch_tokens):
+        ctx.sp_calib_accumulate(X[t0:min(T, t0 + batch_tokens)], stream)
+        launches += 1
+    return launches
+
+
+def select_layer(ctx: sp.Context, w: synth.Workload, W, mask, W_out, mode_arg, stream=None):
+    """One selection call: mode_arg is a sparsity (unstructured) or an (N, M) pair."""
+    if w.mode == "nm":
+        N, M = mode_arg
+        ctx.sp_select_nm(W, N, M, mask=mask, W_out=W_out, stream=stream)
+    else:
+        ctx.sp_select_unstructured(W, mode_arg, mask=mask, W_out=W_out, stream=stream)
+
+
+def prune_model(mb: ModelBuffers, mode_arg, batch_tokens: int, phase_events=None, stream=None):
+    """One pass of the whole hot path over the model: for every block and every distinct layer
+    input, accumulate the calibration statistics, then select + write back every layer that
+    reads this input.  phase_events, if given, is a list that receives (kind, start, end)
+    CUDA-event triples for the calibration and selection phases.  Returns launch counts."""
+    w = mb.workload
+    n_calib = n_select = n_final = 0
+    for b in range(w.blocks):
+        for name, d_in in w.input_widths().items():
+            ctx = mb.ctxs[name]
+            if phase_events is not None:
+                e0 = torch.cuda.Event(enable_timing=True)
+                e1 = torch.cuda.Event(enable_timing=True)
+                e2 = torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+            n_calib += calibrate_input(ctx, mb.acts[name], batch_tokens, stream)
+            if phase_events is not None:
+                e1.record(stream)
+            n_final += 1
+            for li, layer in enumerate(w.layers):
+                if layer.input != name:
+                    continue
+                select_layer(ctx, w, mb.weights[b][li], mb.masks[b][li], mb.outputs[b][li],
+                             mode_arg, stream)
+                n_select += 1
+            if phase_events is not None:
+                e2.record(stream)
+                phase_events.append(("calib", e0, e1, d_in))
+                phase_events.append(("select", e1, e2, d_in))
+    return {"calib": n_calib, "finalize": n_final, "select": n_select}

@@ -1,0 +1,400 @@
+"""GPU parity: the CUDA library, called through its C ABI binding, against the CPU oracle on
+the same seeded inputs, element by element."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import swiftprune_oracle as so
+from tests import parity as P
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def sp():
+    from paper_2501_16376_b200 import binding
+    return binding
+
+
+def _gen(seed, shape, dtype, std=1.0, device="cuda"):
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    return (torch.randn(shape, generator=g, device=device, dtype=torch.float32) * std).to(dtype)
+
+
+def _activations(seed, T, n, dtype, outliers=4):
+    X = _gen(seed, (T, n), torch.float32)
+    idx = torch.randperm(n, generator=torch.Generator().manual_seed(seed))[:min(outliers, n)]
+    X[:, idx.cuda()] *= 20.0
+    return X.to(dtype)
+
+
+# ------------------------------------------------------------------ statistics
+
+@pytest.mark.parametrize("T,n,dtype,ld_extra", [
+    (2048, 512, torch.float16, 0),      # the small single-layer case
+    (1000, 520, torch.float16, 0),      # ragged strip (520 = 2*256 + 8), ragged rows
+    (77, 1030, torch.float16, 0),       # d_in not a multiple of 8: element-wise path
+    (3000, 1024, torch.bfloat16, 0),
+    (513, 768, torch.float16, 8),       # strided rows, still 16-byte aligned
+    (513, 768, torch.bfloat16, 3),      # strided rows, misaligned: element-wise path
+    (5, 8, torch.float16, 0),           # fewer rows than one warp step
+    (1, 1, torch.float16, 0),
+    (16384, 4096, torch.float16, 0),    # one batch of a LLaMA-7B-width input (134 MB)
+])
+def test_calib_statistics_match_oracle(sp, T, n, dtype, ld_extra):
+    X_full = _activations(T * 31 + n, T, n + ld_extra, dtype)
+    X = X_full[:, :n]
+    with sp.Context(n) as ctx:
+        ctx.sp_calib_accumulate(X)
+        colsq, S, factor, ntok = ctx.sp_get_stats()
+    st = P.oracle_stats([X], n)
+    assert ntok == T
+    assert P.rel_err(colsq.numpy(), st.colsq) <= P.SCORE_RTOL
+    assert abs(S - st.S) <= P.SCORE_RTOL * st.S
+    if n > 1:
+        assert P.rel_err(factor.numpy(), st.channel_factor32()) <= P.SCORE_RTOL
+    # tighter than the contract: fp32 partial sums of 8 squares, fp64 beyond
+    assert P.rel_err(colsq.numpy(), st.colsq) <= 1e-6
+
+
+def test_calib_accumulates_over_batches_resets_and_is_deterministic(sp):
+    n = 1536
+    batches = [_activations(100 + i, T, n, torch.float16) for i, T in enumerate([700, 64, 2048, 1])]
+    with sp.Context(n) as ctx:
+        for X in batches:
+            ctx.sp_calib_accumulate(X)
+        colsq, S, factor, ntok = ctx.sp_get_stats()
+        st = P.oracle_stats(batches, n)
+        assert ntok == sum(b.shape[0] for b in batches)
+        assert P.rel_err(colsq.numpy(), st.colsq) <= 1e-6
+        # same batches again after a reset: bit-identical (no floating-point atomics)
+        ctx.sp_calib_reset()
+        for X in batches:
+            ctx.sp_calib_accumulate(X)
+        colsq2, S2, factor2, _ = ctx.sp_get_stats()
+        assert torch.equal(colsq, colsq2) and S == S2 and torch.equal(factor, factor2)
+        # reset really forgets
+        ctx.sp_calib_reset()
+        ctx.sp_calib_accumulate(batches[1])
+        colsq3, _, _, ntok3 = ctx.sp_get_stats()
+        assert ntok3 == 64
+        assert P.rel_err(colsq3.numpy(), P.oracle_stats([batches[1]], n).colsq) <= 1e-6
+        # an empty batch is a no-op
+        ctx.sp_calib_accumulate(batches[1][:0])
+        assert ctx.sp_get_stats()[3] == 64
+
+
+def test_set_stats_round_trip_and_factor_is_bit_exact(sp):
+    n = 1000
+    rng = np.random.default_rng(3)
+    colsq = rng.uniform(0.5, 2.0, n) * 1e4
+    colsq[[3, 500]] *= 400.0
+    with sp.Context(n) as ctx:
+        ctx.sp_set_stats(torch.from_numpy(colsq), 123)
+        got, S, factor, ntok = ctx.sp_get_stats()
+    st = so.Stats(colsq.copy(), 123)
+    assert np.array_equal(got.numpy(), colsq) and ntok == 123
+    assert abs(S - st.S) <= 1e-12 * st.S
+    assert np.array_equal(factor.numpy(), st.channel_factor32())
+
+
+# ------------------------------------------------------------------ scores
+
+@pytest.mark.parametrize("R,n,dtype", [(64, 512, torch.float16), (33, 520, torch.bfloat16),
+                                       (7, 1030, torch.float16)])
+def test_scores_match_oracle(sp, R, n, dtype):
+    W = _gen(R + n, (R, n), dtype, 0.02)
+    X = _activations(n, 512, n, dtype)
+    with sp.Context(n) as ctx:
+        ctx.sp_calib_accumulate(X)
+        L = ctx.sp_score(W).cpu().numpy()
+        colsq, _, _, _ = ctx.sp_get_stats()
+    st = P.oracle_stats([X], n)
+    want = so.score_f32(P.bits(W), P.odtype(W), st)
+    assert P.rel_err(L, want) <= P.SCORE_RTOL
+    # with the library's own statistics handed to the oracle the scores are bit-identical
+    st_gpu = so.Stats(colsq.numpy().copy(), 512)
+    assert np.array_equal(L, so.score_f32(P.bits(W), P.odtype(W), st_gpu))
+
+
+# ------------------------------------------------------------------ N:M selection
+
+def _ctx_with_stats(sp, X_batches, n):
+    ctx = sp.Context(n)
+    for X in X_batches:
+        ctx.sp_calib_accumulate(X)
+    return ctx
+
+
+@pytest.mark.parametrize("R,n,dtype,N,M", [
+    (512, 512, torch.float16, 2, 4),
+    (300, 520, torch.float16, 2, 4),      # ragged last tile
+    (300, 520, torch.bfloat16, 4, 8),
+    (64, 1028, torch.float16, 2, 4),      # d_in % 8 == 4: element-wise path, half-filled chunk
+    (129, 2048, torch.bfloat16, 2, 4),    # bf16: many equal scores inside groups
+    (40, 1024, torch.float16, 1, 4),
+    (40, 1024, torch.float16, 3, 4),
+    (40, 1024, torch.float16, 2, 8),
+    (40, 1024, torch.float16, 6, 8),
+    (1, 8, torch.float16, 4, 8),
+    (3, 4, torch.float16, 2, 4),
+])
+def test_nm_selection_matches_oracle(sp, R, n, dtype, N, M):
+    W = _gen(R * 7 + n, (R, n), dtype, 0.02)
+    X = _activations(n + 1, 1024, n, dtype)
+    with _ctx_with_stats(sp, [X], n) as ctx:
+        mask, out = ctx.sp_select_nm(W, N, M)
+        colsq = ctx.sp_get_stats()[0]
+        # (a) against the oracle fed with the oracle's own statistics: tolerance rule
+        st = P.oracle_stats([X], n)
+        sel = so.select_nm(P.bits(W), P.odtype(W), st, N, M, want_trace=True)
+        P.check_selection(mask, out, W, sel, P.nm_allowed_flips(sel, n, M))
+        # (b) against the oracle fed with the library's statistics: bit-exact
+        sel2 = so.select_nm(P.bits(W), P.odtype(W), so.Stats(colsq.numpy().copy(), 1), N, M)
+        P.check_selection(mask, out, W, sel2, None, strict=True)
+    keep = so.unpack_mask(P.mask_np(mask), n)
+    assert (keep.reshape(R, n // M, M).sum(-1) == N).all()
+
+
+def test_nm_ties_follow_the_lower_column_rule(sp):
+    # few distinct magnitudes and uniform statistics: ties in almost every group
+    R, n = 64, 512
+    g = torch.Generator(device="cuda").manual_seed(5)
+    vals = torch.tensor([0.01, 0.02, 0.02, 0.03], device="cuda")
+    W = vals[torch.randint(0, 4, (R, n), generator=g, device="cuda")]
+    W = (W * (torch.randint(0, 2, (R, n), generator=g, device="cuda") * 2 - 1)).to(torch.float16)
+    colsq = np.full(n, 1000.0)
+    with sp.Context(n) as ctx:
+        ctx.sp_set_stats(torch.from_numpy(colsq), 10)
+        for N, M in ((2, 4), (4, 8)):
+            mask, out = ctx.sp_select_nm(W, N, M)
+            sel = so.select_nm(P.bits(W), so.F16, so.Stats(colsq.copy(), 10), N, M)
+            P.check_selection(mask, out, W, sel, None, strict=True)
+
+
+def test_nm_in_place_strided_and_mask_only(sp):
+    R, n = 96, 768
+    big = _gen(9, (R, n + 16), torch.float16, 0.02)
+    big_before = big.clone()
+    W = big[:, 8:8 + n]                      # ld = n + 16, 16-byte aligned start
+    W_ref = W.clone()
+    X = _activations(10, 512, n, torch.float16)
+    with _ctx_with_stats(sp, [X], n) as ctx:
+        colsq = ctx.sp_get_stats()[0]
+        sel = so.select_nm(P.bits(W_ref), so.F16, so.Stats(colsq.numpy().copy(), 1), 2, 4)
+        mask, out = ctx.sp_select_nm(W, 2, 4, inplace=True)
+        assert out.data_ptr() == W.data_ptr()
+        P.check_selection(mask, W, W_ref, sel, None, strict=True)
+        # the columns outside the view are untouched
+        assert torch.equal(big[:, :8], big_before[:, :8])
+        assert torch.equal(big[:, n + 8:], big_before[:, n + 8:])
+        # idempotent: selecting again on the pruned matrix reproduces the mask
+        mask2, _ = ctx.sp_select_nm(W, 2, 4)
+        assert torch.equal(mask, mask2)
+
+
+# ------------------------------------------------------------------ EWMA selection
+
+def _ewma_params(sp, la, alpha=0.125, beta=0.125, s_update=0):
+    return sp.EwmaParams(alpha, beta, la, s_update)
+
+
+@pytest.mark.parametrize("R,n,dtype,sparsity", [
+    (512, 512, torch.float16, 0.5),       # the small single-layer case
+    (300, 520, torch.float16, 0.6),       # ragged last tile
+    (64, 1030, torch.float16, 0.7),       # element-wise path
+    (200, 4096, torch.bfloat16, 0.5),
+    (200, 4096, torch.bfloat16, 0.8),
+    (50, 11008, torch.float16, 0.5),      # long rows: 43 tiles
+    (3, 8, torch.float16, 0.5),
+    (2, 1, torch.float16, 0.5),
+])
+def test_ewma_selection_matches_oracle(sp, R, n, dtype, sparsity):
+    W = _gen(R * 3 + n, (R, n), dtype, 0.02)
+    X = _activations(n + 2, 2048, n, dtype)
+    counters = sp.new_counters()
+    with _ctx_with_stats(sp, [X], n) as ctx:
+        mask, out = ctx.sp_select_unstructured(W, sparsity, counters=counters)
+        colsq = ctx.sp_get_stats()[0]
+    st = so.Stats(colsq.numpy().copy(), 1)    # isolate the selection from the statistics
+    sel = so.select_unstructured(P.bits(W), P.odtype(W), st, sparsity, want_trace=True,
+                                 s_update=so.S_LITERAL_W2)
+    # tiny matrices: the 1e-6 fraction allows no flip at all
+    P.check_selection(mask, out, W, sel, P.ewma_allowed_flips(sel))
+    keep = so.unpack_mask(P.mask_np(mask), n)
+    assert keep[:, 0].all()                   # column 0 is never pruned
+    assert int(counters[sp.SP_COUNTER_KEPT]) == int(keep.sum())
+    # at calibration scale "S - w^2" cannot change S in fp32: no hazard rows
+    assert int(counters[sp.SP_COUNTER_S_HAZARD]) == 0
+    # also against the oracle's own statistics, under the tolerance rule
+    st_o = P.oracle_stats([X], n)
+    sel_o = so.select_unstructured(P.bits(W), P.odtype(W), st_o, sparsity, want_trace=True)
+    P.check_selection(mask, out, W, sel_o, P.ewma_allowed_flips(sel_o))
+
+
+@pytest.mark.parametrize("alpha,beta,la", [(0.125, 0.125, 4.0), (0.5, 0.25, 0.5),
+                                           (0.03125, 0.0625, -0.2), (1.0, 1.0, 0.5)])
+def test_ewma_other_parameters(sp, alpha, beta, la):
+    R, n = 128, 2048
+    W = _gen(77, (R, n), torch.float16, 0.02)
+    X = _activations(78, 1024, n, torch.float16)
+    with _ctx_with_stats(sp, [X], n) as ctx:
+        mask, out = ctx.sp_select_unstructured(W, params=_ewma_params(sp, la, alpha, beta))
+        colsq = ctx.sp_get_stats()[0]
+    st = so.Stats(colsq.numpy().copy(), 1)
+    sel = so.select_ewma(P.bits(W), so.F16, st, la, alpha, beta, s_update=so.S_FROZEN,
+                         want_trace=True)
+    P.check_selection(mask, out, W, sel, P.ewma_allowed_flips(sel))
+
+
+def test_ewma_literal_S_update_is_bit_exact_and_hazard_counter_fires(sp):
+    # Tiny statistics: S is comparable to sum w^2, so Algorithm 1's "S = S - w_i^2" matters.
+    R, n = 96, 640
+    W = _gen(21, (R, n), torch.float16, 0.02)
+    colsq = np.random.default_rng(4).uniform(1.0, 2.0, n) * 1e-4
+    with sp.Context(n) as ctx:
+        ctx.sp_set_stats(torch.from_numpy(colsq), 10)
+        st = so.Stats(colsq.copy(), 10)
+        lit = so.select_ewma(P.bits(W), so.F16, st, 0.5, s_update=so.S_LITERAL_W2)
+        fro = so.select_ewma(P.bits(W), so.F16, st, 0.5, s_update=so.S_FROZEN, want_trace=True)
+        assert not np.array_equal(lit.mask, fro.mask)          # the two readings differ here
+        counters = sp.new_counters()
+        mask, out = ctx.sp_select_unstructured(
+            W, params=_ewma_params(sp, 0.5, s_update=sp.SP_S_LITERAL_W2), counters=counters)
+        P.check_selection(mask, out, W, lit, None, strict=True)  # sequential kernel: bit-exact
+        assert int(counters[sp.SP_COUNTER_KEPT]) == int(lit.keep_bool(n).sum())
+        counters.zero_()
+        mask_f, out_f = ctx.sp_select_unstructured(W, params=_ewma_params(sp, 0.5),
+                                                   counters=counters)
+        P.check_selection(mask_f, out_f, W, fro, P.ewma_allowed_flips(fro))
+        assert int(counters[sp.SP_COUNTER_S_HAZARD]) == R      # every row is flagged
+
+
+def test_ewma_literal_equals_frozen_at_calibration_scale(sp):
+    R, n = 64, 1024
+    W = _gen(31, (R, n), torch.bfloat16, 0.02)
+    X = _activations(32, 4096, n, torch.bfloat16)
+    with _ctx_with_stats(sp, [X], n) as ctx:
+        a, _ = ctx.sp_select_unstructured(W, params=_ewma_params(sp, 0.5, s_update=1))
+        colsq = ctx.sp_get_stats()[0]
+    sel = so.select_ewma(P.bits(W), so.BF16, so.Stats(colsq.numpy().copy(), 1), 0.5,
+                         s_update=so.S_LITERAL_W2)
+    assert np.array_equal(P.mask_np(a), sel.mask)
+
+
+def test_ewma_in_place_and_determinism(sp):
+    R, n = 128, 1536
+    W = _gen(41, (R, n), torch.float16, 0.02)
+    W_ref = W.clone()
+    X = _activations(42, 1024, n, torch.float16)
+    with _ctx_with_stats(sp, [X], n) as ctx:
+        m1, o1 = ctx.sp_select_unstructured(W, 0.5)
+        m2, o2 = ctx.sp_select_unstructured(W, 0.5)
+        assert torch.equal(m1, m2) and torch.equal(o1.view(torch.int16), o2.view(torch.int16))
+        m3, o3 = ctx.sp_select_unstructured(W, 0.5, inplace=True)
+        assert o3.data_ptr() == W.data_ptr()
+        assert torch.equal(m1, m3) and torch.equal(W.view(torch.int16), o1.view(torch.int16))
+        assert not torch.equal(W, W_ref)
+
+
+# ------------------------------------------------------------------ write-back
+
+@pytest.mark.parametrize("R,n,dtype", [(100, 520, torch.float16), (17, 1030, torch.bfloat16),
+                                       (1, 1, torch.float16), (64, 4096, torch.float16)])
+def test_apply_mask_matches_oracle(sp, R, n, dtype):
+    W = _gen(R + 3 * n, (R, n), dtype, 0.02)
+    g = torch.Generator().manual_seed(R)
+    keep = torch.rand(R, n, generator=g) < 0.5
+    words = (n + 31) // 32
+    packed = np.zeros((R, words * 32), dtype=np.uint8)
+    packed[:, :n] = keep.numpy()
+    mask = np.packbits(packed, axis=1, bitorder="little").view(np.uint32)
+    mask_t = torch.from_numpy(mask.view(np.int32)).cuda()
+    out = sp.sp_apply_mask(W, mask_t)
+    assert np.array_equal(P.bits(out), so.apply_mask(P.bits(W), mask))
+    # in place
+    W2 = W.clone()
+    sp.sp_apply_mask(W2, mask_t, W2)
+    assert torch.equal(W2.view(torch.int16), out.view(torch.int16))
+
+
+# ------------------------------------------------------------------ edge cases and errors
+
+def test_empty_inputs_are_no_ops(sp):
+    n = 256
+    X = _activations(1, 64, n, torch.float16)
+    with _ctx_with_stats(sp, [X], n) as ctx:
+        W0 = torch.empty(0, n, dtype=torch.float16, device="cuda")
+        m, o = ctx.sp_select_nm(W0, 2, 4)
+        assert m.shape == (0, 8) and o.shape == (0, n)
+        m, o = ctx.sp_select_unstructured(W0, 0.5)
+        assert m.shape == (0, 8)
+        assert ctx.sp_score(W0).shape == (0, n)
+
+
+def test_error_statuses(sp):
+    n = 64
+    W = _gen(1, (8, n), torch.float16, 0.02)
+    with sp.Context(n) as ctx:
+        with pytest.raises(sp.SpError) as e:                      # nothing calibrated yet
+            ctx.sp_select_nm(W, 2, 4)
+        assert e.value.status == sp.SP_ERR_STATE
+        with pytest.raises(sp.SpError) as e:
+            ctx.sp_get_stats()
+        assert e.value.status == sp.SP_ERR_STATE
+        ctx.sp_calib_accumulate(_activations(2, 32, n, torch.float16))
+        with pytest.raises(sp.SpError) as e:
+            ctx.sp_select_nm(W, 4, 4)
+        assert e.value.status == sp.SP_ERR_INVALID_ARG
+        with pytest.raises(sp.SpError) as e:
+            ctx.sp_select_nm(W, 2, 5)
+        assert e.value.status == sp.SP_ERR_INVALID_ARG
+        with pytest.raises(sp.SpError) as e:
+            ctx.sp_select_unstructured(W, 1.5)
+        assert e.value.status == sp.SP_ERR_INVALID_ARG
+        with pytest.raises(sp.SpError) as e:
+            ctx.sp_select_unstructured(W, params=_ewma_params(sp, 0.5, alpha=0.0))
+        assert e.value.status == sp.SP_ERR_INVALID_ARG
+        with pytest.raises(sp.SpError) as e:
+            ctx.sp_calib_accumulate(_activations(2, 32, n + 8, torch.float16))
+        assert e.value.status == sp.SP_ERR_SHAPE
+        with pytest.raises(sp.SpError) as e:
+            ctx.sp_select_nm(W.float(), 2, 4)
+        assert e.value.status == sp.SP_ERR_DTYPE
+    with sp.Context(60) as ctx:                                    # 60 % 8 != 0
+        ctx.sp_calib_accumulate(_activations(3, 32, 60, torch.float16))
+        with pytest.raises(sp.SpError) as e:
+            ctx.sp_select_nm(_gen(1, (4, 60), torch.float16), 4, 8)
+        assert e.value.status == sp.SP_ERR_SHAPE
+    with pytest.raises(sp.SpError) as e:
+        sp.Context(0)
+    assert e.value.status == sp.SP_ERR_SHAPE
+
+
+def test_degenerate_statistics_are_reported_not_faulted(sp):
+    n = 128
+    W = _gen(1, (8, n), torch.float16, 0.02)
+    with sp.Context(n) as ctx:
+        ctx.sp_calib_accumulate(torch.zeros(64, n, dtype=torch.float16, device="cuda"))
+        with pytest.raises(sp.SpError) as e:
+            ctx.sp_get_stats()
+        assert e.value.status == sp.SP_ERR_DEGENERATE
+        ctx.sp_select_nm(W, 2, 4)               # still runs; results are unspecified
+        torch.cuda.synchronize()
+    # a single live channel gives an infinite factor there and ordinary ones elsewhere
+    with sp.Context(n) as ctx:
+        X = torch.zeros(64, n, dtype=torch.float16, device="cuda")
+        X[:, 5] = 1.0
+        ctx.sp_calib_accumulate(X)
+        factor = ctx.sp_get_stats()[2]
+        assert torch.isinf(factor[5]) and (factor[:5] == 0.5).all()
+
+
+def test_launch_counter_counts_kernels(sp):
+    n = 256
+    before = sp.sp_launch_count()
+    with sp.Context(n) as ctx:
+        ctx.sp_calib_accumulate(_activations(1, 64, n, torch.float16))   # 1
+        ctx.sp_select_nm(_gen(1, (8, n), torch.float16, 0.02), 2, 4)      # finalise + select
+    assert sp.sp_launch_count() - before == 3

@@ -47,6 +47,10 @@ def parse_args():
     ap.add_argument("--batch-seqs", type=int, default=16,
                     help="calibration sequences per sp_calib_accumulate call")
     ap.add_argument("--e2e-steps", type=int, default=1)
+    ap.add_argument("--blocks", type=int, default=0,
+                    help="profiling aid: prune only the first BLOCKS blocks (0 = the whole model)")
+    ap.add_argument("--mode-index", type=int, default=0,
+                    help="which of the workload's sparsities / N:M patterns to run")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
 
@@ -228,7 +232,9 @@ def gpu_arm(args):
     from paper_2501_16376_b200 import sharding
 
     w = synth.WORKLOADS[args.workload]
-    arg = mode_args(w)[0]
+    if args.blocks > 0:
+        w = synth.Workload(**{**w.__dict__, "blocks": min(args.blocks, w.blocks)})
+    arg = mode_args(w)[args.mode_index]
     batch_tokens = args.batch_seqs * w.seq_len
     # weak scaling: rank r prunes its own model (seed offset r)
     mb = pipeline.allocate_model(w, device, model_seed_offset=sharding.unit_of_rank(rank, world))

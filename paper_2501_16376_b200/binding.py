@@ -13,7 +13,8 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libswiftprune.so")
+#: the compiled library; SWIFTPRUNE_LIBRARY may point at another build of the same ABI
+LIB_PATH = os.environ.get("SWIFTPRUNE_LIBRARY") or os.path.join(_HERE, "libswiftprune.so")
 
 SP_OK = 0
 SP_ERR_INVALID_ARG, SP_ERR_SHAPE, SP_ERR_DTYPE, SP_ERR_STATE = 1, 2, 3, 4

@@ -53,9 +53,10 @@ static sp_status ensure_finalized(sp_ctx *ctx, cudaStream_t stream) {
 
 static sp_status check_matrix_args(const sp_ctx *ctx, const void *W, sp_dtype dtype,
                                    int64_t n_rows, int64_t ldw, const void *W_out, int64_t ldo) {
-    if (ctx == nullptr || W == nullptr) return SP_ERR_INVALID_ARG;
+    if (ctx == nullptr) return SP_ERR_INVALID_ARG;
     if (!valid_dtype(dtype)) return SP_ERR_DTYPE;
     if (n_rows < 0) return SP_ERR_INVALID_ARG;
+    if (W == nullptr && n_rows != 0) return SP_ERR_INVALID_ARG;  // an empty matrix has no address
     if (ldw < ctx->d_in) return SP_ERR_SHAPE;
     if (W_out != nullptr) {
         if (ldo < ctx->d_in) return SP_ERR_SHAPE;
@@ -288,9 +289,10 @@ sp_status sp_select_nm(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_row
 
 sp_status sp_apply_mask(const void *W, sp_dtype dtype, int64_t n_rows, int64_t n_cols, int64_t ldw,
                         const uint32_t *mask, void *W_out, int64_t ldo, sp_stream stream) {
-    if (W == nullptr || mask == nullptr || W_out == nullptr) return SP_ERR_INVALID_ARG;
     if (!valid_dtype(dtype)) return SP_ERR_DTYPE;
     if (n_rows < 0 || n_cols < 0) return SP_ERR_INVALID_ARG;
+    if ((W == nullptr || mask == nullptr || W_out == nullptr) && n_rows * n_cols != 0)
+        return SP_ERR_INVALID_ARG;
     if (ldw < n_cols || ldo < n_cols) return SP_ERR_SHAPE;
     if (W_out == W && ldo != ldw) return SP_ERR_SHAPE;
     return launch_apply_mask(W, dtype, n_rows, n_cols, ldw, mask, W_out, ldo,

@@ -120,17 +120,20 @@ ewma_scan_kernel(const uint16_t *__restrict__ W, int64_t ldw, int64_t n_rows, in
 #pragma unroll
         for (int j = 0; j < 8; ++j) d[j] = fmaf(sc.b_pow[j], dev_in, d[j]);
 
-        // decisions against the state before each element's update
-        uint32_t keep8 = 0;
-        {
-            const float thr0 = fmaf(neg_la, dev_in, est_in);
-            keep8 |= (L[0] < thr0) ? 0u : 1u;
-        }
+        // decisions against the state before each element's update: element j is pruned iff
+        // L_j - (est_{j-1} - la*dev_{j-1}) is negative.  The difference of two floats has the
+        // exact sign (it is never rounded to zero, equal operands give +0, a NaN result is the
+        // positive canonical NaN), so the prune flag is its sign bit; a byte permute with sign
+        // replication turns two of them into the half-word mask of a packed pair.
+        float diff[8];
+        diff[0] = L[0] - fmaf(neg_la, dev_in, est_in);
 #pragma unroll
-        for (int j = 1; j < 8; ++j) {
-            const float thr = fmaf(neg_la, d[j - 1], e[j - 1]);
-            keep8 |= ((L[j] < thr) ? 0u : 1u) << j;
-        }
+        for (int j = 1; j < 8; ++j) diff[j] = L[j] - fmaf(neg_la, d[j - 1], e[j - 1]);
+        uint32_t pm[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            pm[k] = prmt(__float_as_uint(diff[2 * k]), __float_as_uint(diff[2 * k + 1]), 0xffbbu);
+        uint32_t keep8 = ~halfmasks_to_bits(pm) & 0xffu;
         const int64_t left = n - col;
         if (left < 8) keep8 &= left > 0 ? ((1u << left) - 1u) : 0u;
         kept += __popc(keep8);
@@ -139,7 +142,8 @@ ewma_scan_kernel(const uint16_t *__restrict__ W, int64_t ldw, int64_t n_rows, in
         carry_d = __shfl_sync(kFullWarp, d[7], 31);
 
         if (orow != nullptr) {
-            zero_pruned(p, keep8);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) p[k] &= ~pm[k];
             store8<VEC>(orow, col, n, p);
         }
         const uint32_t word = gather_mask_word(keep8, lane);

@@ -1,92 +1,126 @@
 // N:M selection (Section 3.3) fused with score, mask emission and write-back.
 //
-// One lane owns 8 consecutive weights of a row (one 16-byte load), i.e. two groups of four or
-// one group of eight; a group never straddles lanes, so the selection needs no cross-lane
-// traffic.  Scores are L = (w*w)*c_q in binary32 (Eq. 8).  Within a group an element's rank
-// is the number of elements that order before it (smaller score, or equal score and lower
-// column); the M-N lowest ranks are pruned.  Scores are non-negative, so they are compared
-// through their bit patterns as unsigned integers, which also puts NaN above every number.
-// Each warp processes kNmTilesPerWarp tiles with all loads issued first.
+// Work layout.  The column axis is cut into strips of 256 columns; a warp owns one strip and a
+// slab of consecutive rows, a lane owns 8 consecutive columns of the strip (one 16-byte access
+// per row), i.e. two groups of four or one group of eight: a group never straddles lanes, so
+// the selection needs no cross-lane traffic.  The 8 per-channel factors c_q of the lane's
+// columns are loaded once and stay in registers for the whole slab, and several rows are kept
+// in flight per lane.
+//
+// Selection.  Scores are L = (w*w)*c_q in binary32 (Eq. 8); they are non-negative, so they are
+// compared through their bit patterns as unsigned integers, which also ranks NaN above every
+// number.  Element i orders before element j when L_i < L_j, or L_i == L_j and i < j; an
+// element is kept when at least M-N elements of its group order before it.  The counts of all
+// 8 elements of a lane live in the bytes of two registers, biased so that a byte's top bit is
+// the keep flag; a byte permute with sign replication turns those bits into the 16-bit masks
+// that zero the pruned weights, and a two-way dot product packs them into the 8 mask bits.
 #include "sp_device.cuh"
 #include "sp_internal.h"
 
 namespace sp {
 
+// Tuning knobs (compile-time): rows kept in flight per lane, resident CTAs per SM asked of ptxas.
+#ifndef SP_NM_ROWS_IN_FLIGHT
+#define SP_NM_ROWS_IN_FLIGHT 4
+#endif
+#ifndef SP_NM_MIN_BLOCKS
+#define SP_NM_MIN_BLOCKS 4
+#endif
 constexpr int kNmThreads = 256;
 constexpr int kNmWarps = kNmThreads / 32;
-constexpr int kNmTilesPerWarp = 4;
+constexpr int kNmRowsInFlight = SP_NM_ROWS_IN_FLIGHT;
 
-// keep bits (bit e = element e of the group is kept) of one group of M scores.
+// Ranks of one lane's 8 scores, one byte per element (elements 0..3 in ra, 4..7 in rb).
+// A byte holds  bias + (number of elements of the group that order before this element)  with
+// bias = 0x80 - (M - N), so its top bit is set exactly when the element is kept.  For a pair
+// i < j the constant part counts "i orders before j"; when key_i > key_j the count moves from
+// j's byte to i's byte.  No byte can overflow or borrow: the counts stay within 0..M-1.
 template <int M>
-__device__ __forceinline__ uint32_t nm_keep_bits(const uint32_t *key, int prune_count) {
-    int rank[M];
+__device__ __forceinline__ void nm_rank_bytes(const uint32_t (&key)[8], uint32_t bias_bytes,
+                                              uint32_t &ra, uint32_t &rb) {
+    // constant part: byte j receives one count per i < j inside its group
+    ra = bias_bytes + 0x03020100u;
+    rb = bias_bytes + (M == 4 ? 0x03020100u : 0x07060504u);
 #pragma unroll
-    for (int i = 0; i < M; ++i) rank[i] = 0;
+    for (int i = 0; i < 4; ++i) {
 #pragma unroll
-    for (int i = 0; i < M; ++i) {
-#pragma unroll
-        for (int j = i + 1; j < M; ++j) {
-            const int gt = key[i] > key[j] ? 1 : 0;  // j orders before i
-            rank[i] += gt;
-            rank[j] += 1 - gt;                        // i orders before j (ties: lower column)
+        for (int j = i + 1; j < 4; ++j) {
+            const uint32_t move = (1u << (8 * i)) - (1u << (8 * j));
+            if (key[i] > key[j]) ra += move;
+            if (key[4 + i] > key[4 + j]) rb += move;
         }
     }
-    uint32_t keep = 0;
+    if constexpr (M == 8) {
 #pragma unroll
-    for (int i = 0; i < M; ++i) keep |= (rank[i] >= prune_count ? 1u : 0u) << i;
-    return keep;
+        for (int i = 0; i < 4; ++i) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (key[i] > key[4 + j]) {
+                    ra += 1u << (8 * i);
+                    rb -= 1u << (8 * j);
+                }
+            }
+        }
+    }
 }
 
 template <bool BF16, bool VEC, int M>
-__global__ void __launch_bounds__(kNmThreads)
-select_nm_kernel(const uint16_t *__restrict__ W, int64_t ldw, int64_t n, int tiles_per_row,
-                 int64_t total_tiles, const float *__restrict__ factor, int prune_count,
+__global__ void __launch_bounds__(kNmThreads, SP_NM_MIN_BLOCKS)
+select_nm_kernel(const uint16_t *__restrict__ W, int64_t ldw, int64_t n_rows, int64_t n,
+                 int rows_per_warp, const float *__restrict__ factor, int prune_count,
                  uint32_t *__restrict__ mask, int64_t mask_words, uint16_t *__restrict__ W_out,
                  int64_t ldo) {
     const int lane = threadIdx.x & 31;
-    const int64_t first_tile =
-        (static_cast<int64_t>(blockIdx.x) * kNmWarps + (threadIdx.x >> 5)) * kNmTilesPerWarp;
+    const int64_t col = static_cast<int64_t>(blockIdx.x) * kStripChannels + lane * 8;
+    const int64_t slab = static_cast<int64_t>(blockIdx.y) * kNmWarps + (threadIdx.x >> 5);
+    const int64_t row_begin = slab * rows_per_warp;
+    const int64_t row_end = min(n_rows, row_begin + rows_per_warp);
+    if (row_begin >= row_end) return;  // warp-uniform
 
-    uint32_t p[kNmTilesPerWarp][4];
-    int64_t row[kNmTilesPerWarp], col[kNmTilesPerWarp];
+    float c[8];
+    load_factor8(factor, col, c);  // zero past d_in
+    const int64_t left = n - col;
+    const uint32_t valid = left >= 8 ? 0xffu : (left > 0 ? (1u << left) - 1u : 0u);
+    uint32_t *mdst = mask != nullptr ? mask + (col >> 5) : nullptr;
+    const uint32_t bias_bytes = static_cast<uint32_t>(0x80 - prune_count) * 0x01010101u;
+
+    for (int64_t r0 = row_begin; r0 < row_end; r0 += kNmRowsInFlight) {
+        uint32_t p[kNmRowsInFlight][4];
 #pragma unroll
-    for (int u = 0; u < kNmTilesPerWarp; ++u) {
-        const int64_t tile = first_tile + u;
-        row[u] = tile / tiles_per_row;
-        col[u] = (tile - row[u] * tiles_per_row) * kTile + lane * 8;
-        if (tile < total_tiles) {
-            load8<VEC, true>(W + row[u] * ldw, col[u], n, p[u]);
-        } else {
-            p[u][0] = p[u][1] = p[u][2] = p[u][3] = 0u;
+        for (int u = 0; u < kNmRowsInFlight; ++u) {
+            if (r0 + u < row_end) {
+                load8<VEC, true>(W + (r0 + u) * ldw, col, n, p[u]);
+            } else {
+                p[u][0] = p[u][1] = p[u][2] = p[u][3] = 0u;
+            }
         }
-    }
 #pragma unroll
-    for (int u = 0; u < kNmTilesPerWarp; ++u) {
-        if (first_tile + u >= total_tiles) break;  // warp-uniform
-        uint32_t keep8 = 0;
-        if (col[u] < n) {
-            float w[8], c[8];
+        for (int u = 0; u < kNmRowsInFlight; ++u) {
+            const int64_t r = r0 + u;
+            if (r >= row_end) break;  // warp-uniform
+            float w[8];
             unpack8<BF16>(p[u], w);
-            load_factor8(factor, col[u], c);
             uint32_t key[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j)
                 key[j] = __float_as_uint(__fmul_rn(__fmul_rn(w[j], w[j]), c[j]));
-            if constexpr (M == 4) {
-                keep8 = nm_keep_bits<4>(key, prune_count) | (nm_keep_bits<4>(key + 4, prune_count) << 4);
-            } else {
-                keep8 = nm_keep_bits<8>(key, prune_count);
-            }
-            const int64_t left = n - col[u];
-            if (left < 8) keep8 &= (1u << left) - 1u;
+            uint32_t ra, rb;
+            nm_rank_bytes<M>(key, bias_bytes, ra, rb);
+            // half-word masks from the top bit of each rank byte (sign replication)
+            uint32_t m[4];
+            m[0] = prmt(ra, 0u, 0x9988u);
+            m[1] = prmt(ra, 0u, 0xbbaau);
+            m[2] = prmt(rb, 0u, 0x9988u);
+            m[3] = prmt(rb, 0u, 0xbbaau);
+            const uint32_t keep8 = halfmasks_to_bits(m) & valid;
             if (W_out != nullptr) {
-                zero_pruned(p[u], keep8);
-                store8<VEC>(W_out + row[u] * ldo, col[u], n, p[u]);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) p[u][k] &= m[k];
+                store8<VEC>(W_out + r * ldo, col, n, p[u]);
             }
+            const uint32_t word = gather_mask_word(keep8, lane);
+            if (mdst != nullptr && (lane & 3) == 0 && left > 0) mdst[r * mask_words] = word;
         }
-        const uint32_t word = gather_mask_word(keep8, lane);
-        if (mask != nullptr && (lane & 3) == 0 && col[u] < n)
-            mask[row[u] * mask_words + (col[u] >> 5)] = word;
     }
 }
 
@@ -94,25 +128,36 @@ sp_status launch_select_nm(const sp_ctx *ctx, const void *W, sp_dtype dtype, int
                            int64_t ldw, int N, int M, uint32_t *mask, void *W_out, int64_t ldo,
                            cudaStream_t stream) {
     const int64_t n = ctx->d_in;
-    const int tiles_per_row = static_cast<int>((n + kTile - 1) / kTile);
-    const int64_t total_tiles = n_rows * tiles_per_row;
-    if (total_tiles == 0) return SP_OK;
-    const int64_t tiles_per_block = static_cast<int64_t>(kNmWarps) * kNmTilesPerWarp;
-    const int64_t blocks = (total_tiles + tiles_per_block - 1) / tiles_per_block;
-    if (blocks > 0x7fffffffLL) return SP_ERR_SHAPE;
+    if (n_rows == 0) return SP_OK;
+    const int strips = ctx->strips;
+    // Enough warps to fill the GPU a few times over, at least two steps of rows per warp.
+    const int64_t target_warps = static_cast<int64_t>(ctx->sm_count) * 64;
+    int64_t rows_per_warp = (n_rows * strips + target_warps - 1) / target_warps;
+    rows_per_warp = (rows_per_warp + kNmRowsInFlight - 1) / kNmRowsInFlight * kNmRowsInFlight;
+    if (rows_per_warp < 2 * kNmRowsInFlight) rows_per_warp = 2 * kNmRowsInFlight;
+    const int64_t max_grid_y = 65535;
+    if ((n_rows + rows_per_warp * kNmWarps - 1) / (rows_per_warp * kNmWarps) > max_grid_y) {
+        // keep gridDim.y legal for very tall matrices by giving each warp more rows
+        rows_per_warp = (n_rows + max_grid_y * kNmWarps - 1) / (max_grid_y * kNmWarps);
+        rows_per_warp = (rows_per_warp + kNmRowsInFlight - 1) / kNmRowsInFlight * kNmRowsInFlight;
+    }
+    if (rows_per_warp > 0x7fffffffLL) return SP_ERR_SHAPE;
+    const int64_t slabs = (n_rows + rows_per_warp - 1) / rows_per_warp;
+    const dim3 grid(static_cast<unsigned>(strips),
+                    static_cast<unsigned>((slabs + kNmWarps - 1) / kNmWarps));
     const bool vec = aligned16(W) && ldw % 8 == 0 && n % 8 == 0 &&
                      (W_out == nullptr || (aligned16(W_out) && ldo % 8 == 0));
     const uint16_t *Wp = static_cast<const uint16_t *>(W);
     uint16_t *Op = static_cast<uint16_t *>(W_out);
     const int64_t words = (n + 31) / 32;
     const int prune_count = M - N;
-    const unsigned grid = static_cast<unsigned>(blocks);
+    const int rpw = static_cast<int>(rows_per_warp);
 #define SP_LAUNCH(B, V, MM)                                                                  \
     select_nm_kernel<B, V, MM><<<grid, kNmThreads, 0, stream>>>(                              \
-        Wp, ldw, n, tiles_per_row, total_tiles, ctx->factor, prune_count, mask, words, Op, ldo)
+        Wp, ldw, n_rows, n, rpw, ctx->factor, prune_count, mask, words, Op, ldo)
 #define SP_LAUNCH_M(B, V)                                                                     \
     do {                                                                                      \
-        if (M == 4) SP_LAUNCH(B, V, 4); else SP_LAUNCH(B, V, 8);                              \
+        if (M == 8) SP_LAUNCH(B, V, 8); else SP_LAUNCH(B, V, 4);                              \
     } while (0)
     if (dtype == SP_BF16) {
         if (vec) SP_LAUNCH_M(true, true); else SP_LAUNCH_M(true, false);

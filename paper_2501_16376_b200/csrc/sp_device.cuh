@@ -97,6 +97,26 @@ __device__ __forceinline__ void zero_pruned(uint32_t (&p)[4], uint32_t keep) {
     }
 }
 
+// prmt.b32 in its generic mode: result byte k is byte (sel nibble k & 7) of the pair {a, b};
+// when bit 3 of the nibble is set the byte's sign bit is replicated over the whole byte.
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+
+// Four half-word masks m[k] (each 16-bit half is 0xffff or 0, element 2k in the low half) ->
+// the 8-bit pattern with bit e set where element e's half is 0xffff.  Uses the signed
+// two-way dot product: a half of 0xffff is -1, and the weights are -(1 << e).
+__device__ __forceinline__ uint32_t halfmasks_to_bits(const uint32_t (&m)[4]) {
+    int acc = 0;
+    acc = __dp2a_lo(static_cast<int>(m[0]), 0x0000feff, acc);  // weights -1, -2
+    acc = __dp2a_lo(static_cast<int>(m[1]), 0x0000f8fc, acc);  // -4, -8
+    acc = __dp2a_lo(static_cast<int>(m[2]), 0x0000e0f0, acc);  // -16, -32
+    acc = __dp2a_lo(static_cast<int>(m[3]), 0x000080c0, acc);  // -64, -128
+    return static_cast<uint32_t>(acc);
+}
+
 // Each lane holds the 8 keep bits of its chunk.  Returns, in lanes with (lane & 3) == 0, the
 // 32-bit mask word covering the chunks of lanes lane .. lane+3.
 __device__ __forceinline__ uint32_t gather_mask_word(uint32_t keep8, int lane) {

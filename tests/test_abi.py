@@ -66,6 +66,7 @@ def test_status_strings_and_null_arguments(lib_path):
     assert lib.sp_destroy(None) == binding.SP_OK
     assert lib.sp_calib_reset(None, None) == binding.SP_ERR_INVALID_ARG
     assert lib.sp_apply_mask(None, 0, 1, 1, 1, None, None, 1, None) == binding.SP_ERR_INVALID_ARG
+    assert lib.sp_apply_mask(None, 0, 0, 8, 8, None, None, 8, None) == binding.SP_OK
     assert lib.sp_select_nm(None, None, 0, 1, 1, 2, 4, None, None, 1, None) == \
         binding.SP_ERR_INVALID_ARG
 

@@ -331,6 +331,8 @@ def test_empty_inputs_are_no_ops(sp):
         m, o = ctx.sp_select_unstructured(W0, 0.5)
         assert m.shape == (0, 8)
         assert ctx.sp_score(W0).shape == (0, n)
+    empty_mask = torch.empty(0, 8, dtype=torch.int32, device="cuda")
+    assert sp.sp_apply_mask(W0, empty_mask).shape == (0, n)
 
 
 def test_error_statuses(sp):

@@ -125,6 +125,30 @@ sp_status sp_get_stats(sp_ctx *ctx, double *colsq_host, double *S_host, float *f
  */
 sp_status sp_set_stats(sp_ctx *ctx, const double *colsq_host, int64_t n_tokens, sp_stream stream);
 
+/*
+ * One-shot statistics without any allocation (the paper has no counterpart: this exists for
+ * callers, not for the method).  Some programs must not allocate device memory while they
+ * run: code executing inside a framework that owns the whole memory pool, a service that has
+ * handed all remaining memory to its caches, a real-time loop that cannot afford the implicit
+ * device-wide synchronisation of cudaMalloc/cudaFree.  sp_create allocates, so such callers
+ * cannot use a context.  This call computes, for ONE batch X [n_tokens, d_in] (n_tokens >= 1),
+ * what sp_calib_accumulate + finalisation compute, on the CURRENT device, and copies the
+ * results into the caller's DEVICE buffers (each may be NULL): colsq_out[d_in] (fp64),
+ * factor_out[d_in] (fp32 c_q of Eq. 8), S_out[1] (fp64).  Its working memory is a fixed array
+ * inside the library image (about 4.4 MB per GPU, held until the process exits), hence:
+ *   - d_in must be <= 16384, else SP_ERR_SHAPE and nothing is enqueued;
+ *   - it calls no cudaMalloc/cudaFree and no allocating library routine;
+ *   - all calls on one device share that array: calls whose GPU work may overlap (different
+ *     streams, different threads) race and give wrong results - keep them on one stream or
+ *     order them with events.  Nothing is kept between calls;
+ *   - the first call on each device looks up the array's device address (a host-side,
+ *     synchronous runtime query); make that first call before starting any stream capture.
+ * Results agree with the context path to rounding (the token slabs may be cut differently).
+ */
+sp_status sp_calib_stats_noalloc(const void *X, sp_dtype dtype, int64_t n_tokens, int64_t d_in,
+                                 int64_t ldx, double *colsq_out, float *factor_out, double *S_out,
+                                 sp_stream stream);
+
 /* ------------------------------------------------------------------ metric (Eq. 8) */
 
 /*

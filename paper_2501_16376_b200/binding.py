@@ -26,7 +26,7 @@ SP_COUNTER_KEPT, SP_COUNTER_S_HAZARD, SP_NUM_COUNTERS = 0, 1, 2
 #: every symbol include/swiftprune.h declares
 EXPORTS = (
     "sp_create", "sp_destroy", "sp_calib_reset", "sp_calib_accumulate", "sp_get_stats",
-    "sp_set_stats", "sp_score", "sp_la_for_sparsity", "sp_select_unstructured",
+    "sp_set_stats", "sp_calib_stats_noalloc", "sp_score", "sp_la_for_sparsity", "sp_select_unstructured",
     "sp_select_unstructured_ex", "sp_select_nm", "sp_apply_mask", "sp_status_string",
     "sp_last_cuda_error", "sp_launch_count",
 )
@@ -57,6 +57,7 @@ def _load() -> ctypes.CDLL:
     lib.sp_get_stats.argtypes = [vp, vp, vp, vp, ctypes.POINTER(i64), vp]
     lib.sp_set_stats.argtypes = [vp, vp, i64, vp]
     lib.sp_score.argtypes = [vp, vp, ci, i64, i64, vp, vp]
+    lib.sp_calib_stats_noalloc.argtypes = [vp, ci, i64, i64, i64, vp, vp, vp, vp]
     lib.sp_la_for_sparsity.argtypes = [f32, ctypes.POINTER(f32)]
     lib.sp_select_unstructured.argtypes = [vp, vp, ci, i64, i64, f32, vp, vp, i64, vp, vp]
     lib.sp_select_unstructured_ex.argtypes = [vp, vp, ci, i64, i64, ctypes.POINTER(EwmaParams),
@@ -245,6 +246,25 @@ def sp_apply_mask(W: torch.Tensor, mask: torch.Tensor, W_out: torch.Tensor | Non
     _check(lib.sp_apply_mask(ptr, _dtype_of(W), R, n, ld, mask.data_ptr(), optr, ldo,
                              _stream(stream)))
     return W_out
+
+
+def sp_calib_stats_noalloc(X: torch.Tensor, colsq_out: torch.Tensor | None = None,
+                           factor_out: torch.Tensor | None = None,
+                           S_out: torch.Tensor | None = None, stream=None):
+    """One-shot statistics of a single batch for callers that cannot allocate device memory:
+    the library uses a fixed internal array instead of a context (d_in <= 16384).  The outputs
+    are device tensors the caller already owns (fp64 [d_in], fp32 [d_in], fp64 [1]); this
+    wrapper allocates nothing either.  Calls on one device must not overlap on the GPU."""
+    ptr, T, n, ld = _matrix(X, "X")
+    for t, dt, numel in ((colsq_out, torch.float64, n), (factor_out, torch.float32, n),
+                         (S_out, torch.float64, 1)):
+        if t is not None and (t.dtype != dt or t.numel() < numel or not t.is_cuda
+                              or not t.is_contiguous()):
+            raise SpError(SP_ERR_INVALID_ARG, "output buffers must be contiguous CUDA tensors "
+                                              "of the documented type and size")
+    with torch.cuda.device(X.device):
+        _check(lib.sp_calib_stats_noalloc(ptr, _dtype_of(X), T, n, ld, _ptr(colsq_out),
+                                          _ptr(factor_out), _ptr(S_out), _stream(stream)))
 
 
 def new_counters(device=None) -> torch.Tensor:

@@ -197,6 +197,20 @@ sp_status sp_set_stats(sp_ctx *ctx, const double *colsq_host, int64_t n_tokens, 
     return SP_OK;
 }
 
+sp_status sp_calib_stats_noalloc(const void *X, sp_dtype dtype, int64_t n_tokens, int64_t d_in,
+                                 int64_t ldx, double *colsq_out, float *factor_out, double *S_out,
+                                 sp_stream stream) {
+    if (!valid_dtype(dtype)) return SP_ERR_DTYPE;
+    if (X == nullptr || n_tokens < 1) return SP_ERR_INVALID_ARG;
+    if (d_in < 1 || d_in > calib_static_max_d_in()) return SP_ERR_SHAPE;
+    if (ldx < d_in) return SP_ERR_SHAPE;
+    int device = -1;
+    cudaError_t e = cudaGetDevice(&device);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return launch_calib_stats_static(device, X, dtype, n_tokens, d_in, ldx, colsq_out, factor_out,
+                                     S_out, static_cast<cudaStream_t>(stream));
+}
+
 sp_status sp_score(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows, int64_t ldw,
                    float *scores_out, sp_stream stream) {
     if (ctx == nullptr) return SP_ERR_INVALID_ARG;

@@ -9,6 +9,8 @@
 // fp32 and added to an fp64 accumulator.  The CTA adds its 256 sums to row `slab` of the
 // partial-sum array, which no other CTA touches: there are no floating-point atomics, so the
 // statistics are reproducible bit for bit for a given sequence of batches.
+#include <mutex>
+
 #include "sp_device.cuh"
 #include "sp_internal.h"
 
@@ -202,6 +204,123 @@ sp_status launch_finalize(sp_ctx *ctx, cudaStream_t stream) {
     sp_status st = check_launch();
     if (st == SP_OK) ctx->dirty = false;
     return st;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free one-shot statistics.
+//
+// Same two kernels as above, but every byte of working memory comes from one file-scope device
+// array instead of a context obtained with cudaMalloc.  The array is part of the library image:
+// each GPU that loads the library carries it (about 4.4 MB) until the process exits.  All calls
+// on a device share it, so two calls whose work overlaps on the GPU would overwrite each other's
+// partial sums; nothing in it needs to survive from one call to the next.
+constexpr int64_t kStaticMaxDin = 16384;
+constexpr int64_t kStaticPartialDoubles = int64_t(1) << 19;  // 4 MiB of partial sums
+
+struct StaticScratch {
+    double partial[kStaticPartialDoubles];
+    double colsq[kStaticMaxDin];
+    double strip_sum[kStaticMaxDin / kStripChannels];
+    float factor[kStaticMaxDin];
+    DeviceScalars scalars;
+};
+
+static __device__ __align__(256) unsigned char g_static_scratch[sizeof(StaticScratch)];
+
+constexpr int kMaxDevices = 64;
+struct StaticDeviceState {
+    StaticScratch *scratch = nullptr;  // device address of g_static_scratch on this device
+    int sm_count = 0;
+    int blocks_per_sm = 0;
+};
+static StaticDeviceState g_static_state[kMaxDevices];
+static std::mutex g_static_mutex;
+
+// In host code `g_static_scratch` is only a handle for the runtime, not an address the GPU can
+// use; the address on the current device has to be asked for.  Done once per device.
+static sp_status static_setup(int device, StaticDeviceState **out) {
+    if (device < 0 || device >= kMaxDevices) return SP_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    StaticDeviceState &st = g_static_state[device];
+    if (st.scratch == nullptr) {
+        void *ptr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess) return cuda_fail(e);
+        int sms = 0;
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+        if (e != cudaSuccess) return cuda_fail(e);
+        st.sm_count = sms;
+        st.blocks_per_sm = calib_query_blocks_per_sm();
+        st.scratch = static_cast<StaticScratch *>(ptr);
+    }
+    *out = &st;
+    return SP_OK;
+}
+
+int64_t calib_static_max_d_in() { return kStaticMaxDin; }
+
+sp_status launch_calib_stats_static(int device, const void *X, sp_dtype dtype, int64_t n_tokens,
+                                    int64_t d_in, int64_t ldx, double *colsq_out,
+                                    float *factor_out, double *S_out, cudaStream_t stream) {
+    StaticDeviceState *st = nullptr;
+    sp_status status = static_setup(device, &st);
+    if (status != SP_OK) return status;
+    StaticScratch *sc = st->scratch;
+
+    const int64_t n = d_in;
+    const int64_t n_pad = (n + kStripChannels - 1) / kStripChannels * kStripChannels;
+    const int strips = static_cast<int>(n_pad / kStripChannels);
+    // same slab rule as the context path, additionally bounded by the fixed partial-sum area
+    int64_t slabs = static_cast<int64_t>(st->sm_count) * st->blocks_per_sm / strips;
+    if (slabs < 1) slabs = 1;
+    if (slabs > kMaxSlabs) slabs = kMaxSlabs;
+    if (slabs > kStaticPartialDoubles / n_pad) slabs = kStaticPartialDoubles / n_pad;
+    const int64_t min_rows = kCalibWarps * kRowsInFlight;
+    const int64_t max_slabs_by_rows = (n_tokens + min_rows - 1) / min_rows;
+    if (slabs > max_slabs_by_rows) slabs = max_slabs_by_rows;
+    int64_t rows_per_slab = (n_tokens + slabs - 1) / slabs;
+    rows_per_slab = (rows_per_slab + kCalibWarps - 1) / kCalibWarps * kCalibWarps;
+    slabs = (n_tokens + rows_per_slab - 1) / rows_per_slab;
+
+    // The arrival counter of the finalisation kernel must start at zero whatever an earlier
+    // call left behind; every other field is written before it is read.
+    cudaError_t e = cudaMemsetAsync(&sc->scalars, 0, sizeof(DeviceScalars), stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+
+    const bool vec = aligned16(X) && (ldx % 8 == 0) && (n % 8 == 0);
+    const bool bf16 = dtype == SP_BF16;
+    dim3 grid(static_cast<unsigned>(strips), static_cast<unsigned>(slabs));
+    const uint16_t *Xp = static_cast<const uint16_t *>(X);
+#define SP_LAUNCH(B, V)                                                                       \
+    calib_accumulate_kernel<B, V><<<grid, kCalibThreads, 0, stream>>>(                        \
+        Xp, ldx, n_tokens, n, rows_per_slab, sc->partial, n_pad, /*first_fresh_slab=*/0)
+    if (bf16) {
+        if (vec) SP_LAUNCH(true, true); else SP_LAUNCH(true, false);
+    } else {
+        if (vec) SP_LAUNCH(false, true); else SP_LAUNCH(false, false);
+    }
+#undef SP_LAUNCH
+    status = check_launch();
+    if (status != SP_OK) return status;
+    finalize_kernel<<<strips, kStripChannels, 0, stream>>>(
+        sc->partial, static_cast<int>(slabs), n, n_pad, strips, sc->colsq, sc->strip_sum,
+        sc->factor, &sc->scalars);
+    status = check_launch();
+    if (status != SP_OK) return status;
+
+    if (colsq_out != nullptr) {
+        e = cudaMemcpyAsync(colsq_out, sc->colsq, sizeof(double) * n, cudaMemcpyDeviceToDevice, stream);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    if (factor_out != nullptr) {
+        e = cudaMemcpyAsync(factor_out, sc->factor, sizeof(float) * n, cudaMemcpyDeviceToDevice, stream);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    if (S_out != nullptr) {
+        e = cudaMemcpyAsync(S_out, &sc->scalars.S, sizeof(double), cudaMemcpyDeviceToDevice, stream);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    return SP_OK;
 }
 
 }  // namespace sp

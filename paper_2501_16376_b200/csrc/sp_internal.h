@@ -74,6 +74,10 @@ int calib_query_blocks_per_sm();
 sp_status launch_calib_accumulate(sp_ctx *ctx, const void *X, sp_dtype dtype, int64_t n_tokens,
                                   int64_t ldx, cudaStream_t stream);
 sp_status launch_finalize(sp_ctx *ctx, cudaStream_t stream);
+int64_t calib_static_max_d_in();
+sp_status launch_calib_stats_static(int device, const void *X, sp_dtype dtype, int64_t n_tokens,
+                                    int64_t d_in, int64_t ldx, double *colsq_out,
+                                    float *factor_out, double *S_out, cudaStream_t stream);
 
 // elementwise.cu
 sp_status launch_score(const sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,

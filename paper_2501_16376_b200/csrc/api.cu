@@ -98,7 +98,8 @@ sp_status sp_create(sp_ctx **out, int64_t d_in, int device) {
     const size_t np = static_cast<size_t>(ctx->n_pad);
     void *ptrs[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
     const size_t sizes[5] = {sizeof(double) * np * kMaxSlabs, sizeof(double) * np,
-                             sizeof(double) * static_cast<size_t>(ctx->strips), sizeof(float) * np,
+                             sizeof(double) * static_cast<size_t>(ctx->strips),
+                             sizeof(float) * (np + kStripChannels),
                              sizeof(DeviceScalars)};
     for (int i = 0; i < 5; ++i) {
         e = cudaMalloc(&ptrs[i], sizes[i]);

@@ -4,14 +4,17 @@
 // Frozen-S path (scan kernel).  With S fixed, est and dev do not depend on the prune
 // decisions: est_i = a est_{i-1} + alpha L_i and dev_i = b dev_{i-1} + beta |est_i - L_i|
 // (a = 1-alpha, b = 1-beta) are first-order linear recurrences, evaluated as affine scans.
-// One warp owns one row and walks it in tiles of 256 weights; a lane owns 8 consecutive
-// weights.  Per tile: the lane runs both recurrences over its 8 elements from a zero state,
-// a 5-step shuffle scan with the constant multipliers a^(8*2^k) combines the lane totals, and
-// the state entering the lane (the scan's exclusive prefix plus a^(8*lane) times the state
-// carried in from the previous tile) is folded back into the 8 local values.  Element i is
+// One warp owns one row and walks it in tiles of 32*P weights; a lane owns P consecutive
+// weights (P = 8 by default, 16 as a build option).  Per tile and recurrence: the lane runs the
+// recurrence over its P elements from a zero state to get its total, a 5-step shuffle scan with
+// the constant multipliers a^(P*2^k) combines the lane totals, and the lane runs the recurrence
+// again from the state entering it (the scan's exclusive prefix plus a^(P*lane) times the state
+// carried in from the previous tile), which needs no per-element constants and keeps few values
+// live.  Element i is
 // tested against the state before its own update, est_{i-1} - la*dev_{i-1}; est_{-1} = L_0 and
-// dev_{-1} = 0 (Table 2), so column 0 is never pruned.  The next tile's weights are loaded
-// before the current tile is processed; only the two carried scalars serialise the tiles.
+// dev_{-1} = 0 (Table 2), so column 0 is never pruned.  The weights of the next few tiles are
+// already on their way into shared memory (asynchronous copies) while a tile is processed; only
+// the two carried scalars serialise the tiles.
 //
 // Literal-S path (sequential kernel).  Algorithm 1's "S = S - w_i^2" makes L_i depend on
 // earlier decisions, so the row is evaluated in order by one thread, every operation in
@@ -23,9 +26,27 @@
 
 namespace sp {
 
+#ifndef SP_EWMA_MIN_BLOCKS
+#define SP_EWMA_MIN_BLOCKS 4
+#endif
 constexpr int kEwmaThreads = 256;
 constexpr int kEwmaWarps = kEwmaThreads / 32;
+#ifndef SP_EWMA_PER_LANE
+#define SP_EWMA_PER_LANE 8
+#endif
+#ifndef SP_EWMA_RING
+#define SP_EWMA_RING 1
+#endif
+constexpr int kEwmaPerLane = SP_EWMA_PER_LANE;    // consecutive weights per lane (8 or 16)
+constexpr int kEwmaHalves = kEwmaPerLane / 8;     // 16-byte pieces per lane and tile
+constexpr bool kEwmaRing = SP_EWMA_RING != 0;     // stage tiles through shared memory
+constexpr int kEwmaTile = 32 * kEwmaPerLane;      // weights per warp tile
+#ifndef SP_EWMA_STAGES
+#define SP_EWMA_STAGES 6
+#endif
+constexpr int kEwmaStages = SP_EWMA_STAGES;       // tiles of a row in flight per warp (ring in smem)
 
+// Running packed maximum of |w| (two 16-bit floats per word).
 template <bool BF16>
 __device__ __forceinline__ uint32_t packed_abs_max(uint32_t acc, uint32_t v) {
     if constexpr (BF16) {
@@ -41,7 +62,7 @@ __device__ __forceinline__ uint32_t packed_abs_max(uint32_t acc, uint32_t v) {
     }
 }
 
-// Inclusive scan over lanes of x with the recurrence multiplier step[k] = m^(8*2^k).
+// Inclusive scan over lanes of x with the recurrence multiplier step[k] = m^(P*2^k).
 __device__ __forceinline__ float lane_affine_scan(float x, const float (&step)[5], int lane) {
 #pragma unroll
     for (int k = 0; k < 5; ++k) {
@@ -51,116 +72,201 @@ __device__ __forceinline__ float lane_affine_scan(float x, const float (&step)[5
     return x;
 }
 
-template <bool BF16, bool VEC>
-__global__ void __launch_bounds__(kEwmaThreads)
-ewma_scan_kernel(const uint16_t *__restrict__ W, int64_t ldw, int64_t n_rows, int64_t n,
+// The kernel carries the two states in scaled form, E = est/alpha and D = dev/beta:
+//     E_i = a E_{i-1} + L_i ,   D_i = b D_{i-1} + |alpha E_i - L_i| ,
+// and element i is pruned iff  L_i - alpha E_{i-1} + (la beta) D_{i-1} < 0.
+// Keeps a kernel parameter in a register for the whole kernel (the compiler would otherwise be
+// free to re-read it from the constant bank at every use).
+__device__ __forceinline__ float pinned(float v) {
+    float r;
+    asm volatile("mov.f32 %0, %1;" : "=f"(r) : "f"(v));
+    return r;
+}
+
+// COUNT: also produce the kept-weight count and the S-hazard flag of the row.
+template <bool BF16, bool VEC, bool COUNT>
+__global__ void __launch_bounds__(kEwmaThreads, SP_EWMA_MIN_BLOCKS)
+ewma_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
                  const float *__restrict__ factor, const DeviceScalars *__restrict__ scalars,
                  const __grid_constant__ ScanConstants sc, uint32_t *__restrict__ mask,
-                 int64_t mask_words, uint16_t *__restrict__ W_out, int64_t ldo,
+                 int mask_words, uint16_t *__restrict__ W_out, int ldo,
                  unsigned long long *__restrict__ counters) {
     const int lane = threadIdx.x & 31;
-    const int64_t row = static_cast<int64_t>(blockIdx.x) * kEwmaWarps + (threadIdx.x >> 5);
+    const int row = blockIdx.x * kEwmaWarps + (threadIdx.x >> 5);
     if (row >= n_rows) return;  // warp-uniform
-    const uint16_t *wrow = W + row * ldw;
-    uint16_t *orow = W_out != nullptr ? W_out + row * ldo : nullptr;
-    uint32_t *mrow = mask != nullptr ? mask + row * mask_words : nullptr;
+    const uint16_t *wrow = W + static_cast<int64_t>(row) * ldw;
+    uint16_t *orow = W_out != nullptr ? W_out + static_cast<int64_t>(row) * ldo : nullptr;
+    uint32_t *mrow = mask != nullptr ? mask + static_cast<int64_t>(row) * mask_words : nullptr;
 
-    const float alpha = sc.alpha, beta = sc.beta, neg_la = -sc.la, a = sc.a, b = sc.b;
-    const float a_lane = sc.a_lane[lane], b_lane = sc.b_lane[lane];
+    const float alpha = pinned(sc.alpha), neg_alpha = pinned(-sc.alpha);
+    const float la_beta = pinned(sc.la * sc.beta);
+    const float a = pinned(sc.a), b = pinned(sc.b);
+    const float a_lane = pinned(sc.a_lane[lane]), b_lane = pinned(sc.b_lane[lane]);
     float a_step[5], b_step[5];
 #pragma unroll
-    for (int k = 0; k < 5; ++k) { a_step[k] = sc.a_step[k]; b_step[k] = sc.b_step[k]; }
+    for (int k = 0; k < 5; ++k) { a_step[k] = pinned(sc.a_step[k]); b_step[k] = pinned(sc.b_step[k]); }
 
-    const int tiles = static_cast<int>((n + kTile - 1) / kTile);
-    float carry_e = 0.0f, carry_d = 0.0f;
+    const int tiles = (n + kEwmaTile - 1) / kEwmaTile;
+    float carry_E = 0.0f, carry_D = 0.0f;
     uint32_t kept = 0;
     uint32_t wmax = 0;  // packed running max of |w| over this lane's elements
 
-    uint32_t p_next[4];
-    load8<VEC, true>(wrow, lane * 8, n, p_next);
+    // Aligned path: every lane streams its own 16*kEwmaHalves bytes of each tile through a private
+    // slot of a shared-memory ring with asynchronous copies, kEwmaStages-1 tiles ahead of the tile
+    // being processed; a lane only ever reads what it copied itself, so waiting on its own copy
+    // groups is the only synchronisation.  (Layout: the 16-byte pieces of the 32 lanes are stored
+    // as contiguous 512-byte rows, which keeps the 16-byte shared loads conflict-free.)
+    constexpr bool RING = VEC && kEwmaRing;
+    constexpr int kSlot = 32 * kEwmaHalves;  // uint4 per warp and stage
+    __shared__ __align__(16) uint4 ring[RING ? kEwmaWarps * kEwmaStages * kSlot : 1];
+    uint4 *my_ring = ring + (RING ? (threadIdx.x >> 5) * kEwmaStages * kSlot + lane : 0);
+    auto issue_tile = [&](int t) {
+        if constexpr (RING) {
+            if (t < tiles) {
+                const int c0 = t * kEwmaTile + lane * kEwmaPerLane;
+                uint4 *slot = my_ring + (t % kEwmaStages) * kSlot;
+#pragma unroll
+                for (int h = 0; h < kEwmaHalves; ++h)
+                    cp_async16(slot + 32 * h, wrow + min(c0 + 8 * h, n - 8),
+                               c0 + 8 * h < n ? 16 : 0);
+            }
+            cp_async_commit();
+        }
+    };
+#pragma unroll
+    for (int t = 0; t < kEwmaStages - 1; ++t) issue_tile(t);
+    uint32_t p_next[kEwmaHalves][4];
+    if constexpr (!RING) {
+#pragma unroll
+        for (int h = 0; h < kEwmaHalves; ++h)
+            load8<VEC, true>(wrow, lane * kEwmaPerLane + 8 * h, n, p_next[h]);
+    }
 
     for (int tile = 0; tile < tiles; ++tile) {
-        const int64_t col = static_cast<int64_t>(tile) * kTile + lane * 8;
-        uint32_t p[4];
+        const int col = tile * kEwmaTile + lane * kEwmaPerLane;
+        uint32_t p[kEwmaHalves][4];
+        if constexpr (RING) {
+            issue_tile(tile + kEwmaStages - 1);
+            cp_async_wait<kEwmaStages - 1>();
+            const uint4 *slot = my_ring + (tile % kEwmaStages) * kSlot;
 #pragma unroll
-        for (int k = 0; k < 4; ++k) p[k] = p_next[k];
-        if (tile + 1 < tiles) load8<VEC, true>(wrow, col + kTile, n, p_next);
+            for (int h = 0; h < kEwmaHalves; ++h) {
+                const uint4 v = slot[32 * h];
+                p[h][0] = v.x; p[h][1] = v.y; p[h][2] = v.z; p[h][3] = v.w;
+            }
+        } else {
+#pragma unroll
+            for (int h = 0; h < kEwmaHalves; ++h) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k) p[h][k] = p_next[h][k];
+                if (tile + 1 < tiles) load8<VEC, true>(wrow, col + kEwmaTile + 8 * h, n, p_next[h]);
+            }
+        }
 
-        float w[8], c[8], L[8];
-        unpack8<BF16>(p, w);
-        load_factor8(factor, col, c);  // zero past d_in: scores of padding are 0
+        float L[kEwmaPerLane];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) wmax = packed_abs_max<BF16>(wmax, p[k]);
+        for (int h = 0; h < kEwmaHalves; ++h) {
+            float w[8], c[8];
+            unpack8<BF16>(p[h], w);
+            load_factor8(factor, col + 8 * h, c);  // zero past d_in: scores of padding are 0
 #pragma unroll
-        for (int j = 0; j < 8; ++j) L[j] = __fmul_rn(__fmul_rn(w[j], w[j]), c[j]);
+            for (int j = 0; j < 8; ++j) L[8 * h + j] = __fmul_rn(__fmul_rn(w[j], w[j]), c[j]);
+            if constexpr (COUNT) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k) wmax = packed_abs_max<BF16>(wmax, p[h][k]);
+            }
+        }
 
-        if (tile == 0) carry_e = __shfl_sync(kFullWarp, L[0], 0);  // est starts at L_0
+        if (tile == 0) carry_E = __shfl_sync(kFullWarp, L[0], 0) / alpha;  // est starts at L_0
 
-        // est: local recurrence from zero, lane scan, fold the incoming state back in
-        float e[8];
-        e[0] = alpha * L[0];
+        // Pass A: E over the lane's elements from a zero state -> lane total -> scan.
+        float acc = L[0];
 #pragma unroll
-        for (int j = 1; j < 8; ++j) e[j] = fmaf(a, e[j - 1], alpha * L[j]);
-        float incl = lane_affine_scan(e[7], a_step, lane);
+        for (int j = 1; j < kEwmaPerLane; ++j) acc = fmaf(a, acc, L[j]);
+        float incl = lane_affine_scan(acc, a_step, lane);
         float excl = __shfl_up_sync(kFullWarp, incl, 1);
         if (lane == 0) excl = 0.0f;
-        const float est_in = fmaf(a_lane, carry_e, excl);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) e[j] = fmaf(sc.a_pow[j], est_in, e[j]);
+        const float E_in = fmaf(a_lane, carry_E, excl);  // E before this lane's first element
 
-        // dev: same with the inputs beta * |est_i - L_i|
-        float d[8];
-        d[0] = beta * fabsf(e[0] - L[0]);
+        // Pass B: the true E from E_in; per element q_j = L_j - alpha E_{j-1} (the part of the
+        // decision that does not need D) and |alpha E_j - L_j| (the input of D); D from a zero
+        // state -> lane total -> scan.
+        float q[kEwmaPerLane], dabs[kEwmaPerLane];
+        float E_run = E_in, D_loc = 0.0f;
 #pragma unroll
-        for (int j = 1; j < 8; ++j) d[j] = fmaf(b, d[j - 1], beta * fabsf(e[j] - L[j]));
-        incl = lane_affine_scan(d[7], b_step, lane);
+        for (int j = 0; j < kEwmaPerLane; ++j) {
+            q[j] = fmaf(neg_alpha, E_run, L[j]);
+            E_run = fmaf(a, E_run, L[j]);
+            dabs[j] = fabsf(fmaf(alpha, E_run, -L[j]));
+            D_loc = __fadd_rn(__fmul_rn(b, D_loc), dabs[j]);
+        }
+        incl = lane_affine_scan(D_loc, b_step, lane);
         excl = __shfl_up_sync(kFullWarp, incl, 1);
         if (lane == 0) excl = 0.0f;
-        const float dev_in = fmaf(b_lane, carry_d, excl);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) d[j] = fmaf(sc.b_pow[j], dev_in, d[j]);
+        const float D_in = fmaf(b_lane, carry_D, excl);
 
-        // decisions against the state before each element's update: element j is pruned iff
-        // L_j - (est_{j-1} - la*dev_{j-1}) is negative.  The difference of two floats has the
-        // exact sign (it is never rounded to zero, equal operands give +0, a NaN result is the
-        // positive canonical NaN), so the prune flag is its sign bit; a byte permute with sign
-        // replication turns two of them into the half-word mask of a packed pair.
-        float diff[8];
-        diff[0] = L[0] - fmaf(neg_la, dev_in, est_in);
+        // Pass C: the true D from D_in and the decisions against the state before each element's
+        // update.  The sign bit of  L_i - est_{i-1} + la dev_{i-1}  is the prune flag (a NaN is
+        // the positive canonical NaN: kept, as "L < threshold" is false); a byte permute with
+        // sign replication turns two flags into the half-word mask of a packed pair of weights.
+        float diff[kEwmaPerLane];
+        float D_run = D_in;
 #pragma unroll
-        for (int j = 1; j < 8; ++j) diff[j] = L[j] - fmaf(neg_la, d[j - 1], e[j - 1]);
-        uint32_t pm[4];
+        for (int j = 0; j < kEwmaPerLane; ++j) {
+            diff[j] = fmaf(la_beta, D_run, q[j]);
+            D_run = __fadd_rn(__fmul_rn(b, D_run), dabs[j]);
+        }
+        uint32_t pm[kEwmaHalves][4];
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
-            pm[k] = prmt(__float_as_uint(diff[2 * k]), __float_as_uint(diff[2 * k + 1]), 0xffbbu);
-        uint32_t keep8 = ~halfmasks_to_bits(pm) & 0xffu;
-        const int64_t left = n - col;
-        if (left < 8) keep8 &= left > 0 ? ((1u << left) - 1u) : 0u;
-        kept += __popc(keep8);
+        for (int h = 0; h < kEwmaHalves; ++h)
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                pm[h][k] = prmt(__float_as_uint(diff[8 * h + 2 * k]),
+                                __float_as_uint(diff[8 * h + 2 * k + 1]), 0xffbbu);
+        uint32_t pruned = halfmasks_to_bits(pm[0]);
+        if constexpr (kEwmaHalves == 2) pruned |= halfmasks_to_bits(pm[kEwmaHalves - 1]) << 8;
+        uint32_t keep16 = ~pruned & ((1u << kEwmaPerLane) - 1u);
+        if (tile == 0 && lane == 0 && (keep16 & 1u) == 0u) {
+            // column 0 is kept by definition (est starts at L_0); alpha*(L_0/alpha) may round up
+            keep16 |= 1u;
+            pm[0][0] &= 0xffff0000u;
+        }
+        const int left = n - col;
+        if (left < kEwmaPerLane) keep16 &= left > 0 ? ((1u << left) - 1u) : 0u;
+        if constexpr (COUNT) kept += __popc(keep16);
 
-        carry_e = __shfl_sync(kFullWarp, e[7], 31);
-        carry_d = __shfl_sync(kFullWarp, d[7], 31);
+        carry_E = __shfl_sync(kFullWarp, E_run, 31);
+        carry_D = __shfl_sync(kFullWarp, D_run, 31);
 
         if (orow != nullptr) {
 #pragma unroll
-            for (int k = 0; k < 4; ++k) p[k] &= ~pm[k];
-            store8<VEC>(orow, col, n, p);
+            for (int h = 0; h < kEwmaHalves; ++h) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k) p[h][k] &= ~pm[h][k];
+                store8<VEC>(orow, col + 8 * h, n, p[h]);
+            }
         }
-        const uint32_t word = gather_mask_word(keep8, lane);
-        if (mrow != nullptr && (lane & 3) == 0 && col < n) mrow[col >> 5] = word;
+        if constexpr (kEwmaPerLane == 16) {  // two lanes share a 32-bit mask word
+            uint32_t word = keep16 << (16 * (lane & 1));
+            word |= __shfl_xor_sync(kFullWarp, word, 1);
+            if (mrow != nullptr && (lane & 1) == 0 && col < n) mrow[col >> 5] = word;
+        } else {                             // four lanes share one
+            const uint32_t word = gather_mask_word(keep16, lane);
+            if (mrow != nullptr && (lane & 3) == 0 && col < n) mrow[col >> 5] = word;
+        }
     }
 
-    if (counters != nullptr) {
+    if constexpr (COUNT) {
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) kept += __shfl_xor_sync(kFullWarp, kept, off);
-        float2 m = unpack2<BF16>(wmax);
-        float mx = fmaxf(m.x, m.y);
+        float2 m2 = unpack2<BF16>(wmax);
+        float bound = fmaxf(m2.x, m2.y);
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1)
-            mx = fmaxf(mx, __shfl_xor_sync(kFullWarp, mx, off));
+            bound = fmaxf(bound, __shfl_xor_sync(kFullWarp, bound, off));
         if (lane == 0) {
             atomicAdd(counters + SP_COUNTER_KEPT, static_cast<unsigned long long>(kept));
-            if (!(mx * mx < scalars->hazard_w2)) atomicAdd(counters + SP_COUNTER_S_HAZARD, 1ULL);
+            if (!(bound * bound < scalars->hazard_w2)) atomicAdd(counters + SP_COUNTER_S_HAZARD, 1ULL);
         }
     }
 }
@@ -219,17 +325,13 @@ static void fill_scan_constants(const sp_ewma_params &p, ScanConstants &sc) {
     sc.a = 1.0f - p.alpha;
     sc.b = 1.0f - p.beta;
     const double a = static_cast<double>(sc.a), b = static_cast<double>(sc.b);
-    for (int j = 0; j < 8; ++j) {
-        sc.a_pow[j] = static_cast<float>(pow(a, j + 1));
-        sc.b_pow[j] = static_cast<float>(pow(b, j + 1));
-    }
     for (int l = 0; l < 32; ++l) {
-        sc.a_lane[l] = static_cast<float>(pow(a, 8.0 * l));
-        sc.b_lane[l] = static_cast<float>(pow(b, 8.0 * l));
+        sc.a_lane[l] = static_cast<float>(pow(a, static_cast<double>(kEwmaPerLane) * l));
+        sc.b_lane[l] = static_cast<float>(pow(b, static_cast<double>(kEwmaPerLane) * l));
     }
     for (int k = 0; k < 5; ++k) {
-        sc.a_step[k] = static_cast<float>(pow(a, 8.0 * (1 << k)));
-        sc.b_step[k] = static_cast<float>(pow(b, 8.0 * (1 << k)));
+        sc.a_step[k] = static_cast<float>(pow(a, static_cast<double>(kEwmaPerLane) * (1 << k)));
+        sc.b_step[k] = static_cast<float>(pow(b, static_cast<double>(kEwmaPerLane) * (1 << k)));
     }
 }
 
@@ -238,6 +340,7 @@ sp_status launch_select_ewma(const sp_ctx *ctx, const void *W, sp_dtype dtype, i
                              int64_t ldo, unsigned long long *counters, cudaStream_t stream) {
     const int64_t n = ctx->d_in;
     if (n_rows == 0) return SP_OK;
+    if (n_rows > 0x7fffffffLL || ldw > 0x7fffffffLL || ldo > 0x7fffffffLL) return SP_ERR_SHAPE;
     const uint16_t *Wp = static_cast<const uint16_t *>(W);
     uint16_t *Op = static_cast<uint16_t *>(W_out);
     const int64_t words = (n + 31) / 32;
@@ -264,15 +367,21 @@ sp_status launch_select_ewma(const sp_ctx *ctx, const void *W, sp_dtype dtype, i
     const bool vec = aligned16(W) && ldw % 8 == 0 && n % 8 == 0 &&
                      (W_out == nullptr || (aligned16(W_out) && ldo % 8 == 0));
     const unsigned grid = static_cast<unsigned>(blocks);
+#define SP_LAUNCH_C(B, V, C)                                                                 \
+    ewma_scan_kernel<B, V, C><<<grid, kEwmaThreads, 0, stream>>>(                            \
+        Wp, static_cast<int>(ldw), static_cast<int>(n_rows), static_cast<int>(n), ctx->factor,   \
+        ctx->scalars, sc, mask, static_cast<int>(words), Op, static_cast<int>(ldo), counters)
 #define SP_LAUNCH(B, V)                                                                      \
-    ewma_scan_kernel<B, V><<<grid, kEwmaThreads, 0, stream>>>(                               \
-        Wp, ldw, n_rows, n, ctx->factor, ctx->scalars, sc, mask, words, Op, ldo, counters)
+    do {                                                                                     \
+        if (counters != nullptr) SP_LAUNCH_C(B, V, true); else SP_LAUNCH_C(B, V, false);     \
+    } while (0)
     if (bf16) {
         if (vec) SP_LAUNCH(true, true); else SP_LAUNCH(true, false);
     } else {
         if (vec) SP_LAUNCH(false, true); else SP_LAUNCH(false, false);
     }
 #undef SP_LAUNCH
+#undef SP_LAUNCH_C
     return check_launch();
 }
 

@@ -24,11 +24,36 @@ namespace sp {
 #define SP_NM_ROWS_IN_FLIGHT 4
 #endif
 #ifndef SP_NM_MIN_BLOCKS
-#define SP_NM_MIN_BLOCKS 4
+#define SP_NM_MIN_BLOCKS 8
 #endif
-constexpr int kNmThreads = 256;
+#ifndef SP_NM_THREADS
+#define SP_NM_THREADS 128
+#endif
+constexpr int kNmThreads = SP_NM_THREADS;
 constexpr int kNmWarps = kNmThreads / 32;
 constexpr int kNmRowsInFlight = SP_NM_ROWS_IN_FLIGHT;
+
+// if (a > b) r += MOVE, as a compare and one predicated add.
+template <uint32_t MOVE>
+__device__ __forceinline__ void add_if_greater(uint32_t &r, uint32_t a, uint32_t b) {
+    asm("{\n\t.reg .pred p;\n\tsetp.gt.u32 p, %1, %2;\n\t@p add.u32 %0, %0, %3;\n\t}"
+        : "+r"(r)
+        : "r"(a), "r"(b), "n"(MOVE));
+}
+
+// if (a > b) { ra += 1 << (8*I); rb -= 1 << (8*J); }
+template <int I, int J>
+__device__ __forceinline__ void move_across(uint32_t &ra, uint32_t &rb, uint32_t a, uint32_t b) {
+    asm("{\n\t.reg .pred p;\n\tsetp.gt.u32 p, %2, %3;\n\t@p add.u32 %0, %0, %4;\n\t"
+        "@p sub.u32 %1, %1, %5;\n\t}"
+        : "+r"(ra), "+r"(rb)
+        : "r"(a), "r"(b), "n"(1u << (8 * I)), "n"(1u << (8 * J)));
+}
+
+template <int I, int J>
+__device__ __forceinline__ void rank_pair(uint32_t &r, const uint32_t *key) {
+    add_if_greater<(1u << (8 * I)) - (1u << (8 * J))>(r, key[I], key[J]);
+}
 
 // Ranks of one lane's 8 scores, one byte per element (elements 0..3 in ra, 4..7 in rb).
 // A byte holds  bias + (number of elements of the group that order before this element)  with
@@ -36,91 +61,108 @@ constexpr int kNmRowsInFlight = SP_NM_ROWS_IN_FLIGHT;
 // i < j the constant part counts "i orders before j"; when key_i > key_j the count moves from
 // j's byte to i's byte.  No byte can overflow or borrow: the counts stay within 0..M-1.
 template <int M>
-__device__ __forceinline__ void nm_rank_bytes(const uint32_t (&key)[8], uint32_t bias_bytes,
-                                              uint32_t &ra, uint32_t &rb) {
-    // constant part: byte j receives one count per i < j inside its group
-    ra = bias_bytes + 0x03020100u;
-    rb = bias_bytes + (M == 4 ? 0x03020100u : 0x07060504u);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-#pragma unroll
-        for (int j = i + 1; j < 4; ++j) {
-            const uint32_t move = (1u << (8 * i)) - (1u << (8 * j));
-            if (key[i] > key[j]) ra += move;
-            if (key[4 + i] > key[4 + j]) rb += move;
-        }
-    }
+__device__ __forceinline__ void nm_rank_bytes(const uint32_t (&key)[8], uint32_t bias_lo,
+                                              uint32_t bias_hi, uint32_t &ra, uint32_t &rb) {
+    ra = bias_lo;  // bias + 0x03020100: byte j receives one count per i < j of its group
+    rb = bias_hi;  // same for M == 4; bias + 0x07060504 for M == 8
+    rank_pair<0, 1>(ra, key); rank_pair<0, 2>(ra, key); rank_pair<0, 3>(ra, key);
+    rank_pair<1, 2>(ra, key); rank_pair<1, 3>(ra, key); rank_pair<2, 3>(ra, key);
+    rank_pair<0, 1>(rb, key + 4); rank_pair<0, 2>(rb, key + 4); rank_pair<0, 3>(rb, key + 4);
+    rank_pair<1, 2>(rb, key + 4); rank_pair<1, 3>(rb, key + 4); rank_pair<2, 3>(rb, key + 4);
     if constexpr (M == 8) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                if (key[i] > key[4 + j]) {
-                    ra += 1u << (8 * i);
-                    rb -= 1u << (8 * j);
-                }
-            }
-        }
+#define SP_ROW(I)                                                                             \
+    move_across<I, 0>(ra, rb, key[I], key[4]); move_across<I, 1>(ra, rb, key[I], key[5]);      \
+    move_across<I, 2>(ra, rb, key[I], key[6]); move_across<I, 3>(ra, rb, key[I], key[7]);
+        SP_ROW(0) SP_ROW(1) SP_ROW(2) SP_ROW(3)
+#undef SP_ROW
     }
+}
+
+// One row of one lane: score, rank, masks, write-back.  Returns the 8 keep bits.
+template <bool BF16, bool VEC, int M>
+__device__ __forceinline__ uint32_t nm_process_row(uint32_t (&p)[4], const float (&c)[8],
+                                                   uint32_t bias_lo, uint32_t bias_hi,
+                                                   uint32_t valid, uint16_t *out_row, int64_t col,
+                                                   int64_t n) {
+    float w[8];
+    unpack8<BF16>(p, w);
+    uint32_t key[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) key[j] = __float_as_uint(__fmul_rn(__fmul_rn(w[j], w[j]), c[j]));
+    uint32_t ra, rb;
+    nm_rank_bytes<M>(key, bias_lo, bias_hi, ra, rb);
+    // half-word masks from the top bit of each rank byte (sign replication)
+    uint32_t m[4];
+    m[0] = prmt(ra, 0u, 0x9988u);
+    m[1] = prmt(ra, 0u, 0xbbaau);
+    m[2] = prmt(rb, 0u, 0x9988u);
+    m[3] = prmt(rb, 0u, 0xbbaau);
+    if (out_row != nullptr) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) p[k] &= m[k];
+        store8<VEC>(out_row, col, n, p);
+    }
+    return halfmasks_to_bits(m) & valid;
 }
 
 template <bool BF16, bool VEC, int M>
 __global__ void __launch_bounds__(kNmThreads, SP_NM_MIN_BLOCKS)
-select_nm_kernel(const uint16_t *__restrict__ W, int64_t ldw, int64_t n_rows, int64_t n,
+select_nm_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int64_t n,
                  int rows_per_warp, const float *__restrict__ factor, int prune_count,
-                 uint32_t *__restrict__ mask, int64_t mask_words, uint16_t *__restrict__ W_out,
-                 int64_t ldo) {
+                 uint32_t *__restrict__ mask, int mask_words, uint16_t *__restrict__ W_out,
+                 int ldo) {
     const int lane = threadIdx.x & 31;
     const int64_t col = static_cast<int64_t>(blockIdx.x) * kStripChannels + lane * 8;
-    const int64_t slab = static_cast<int64_t>(blockIdx.y) * kNmWarps + (threadIdx.x >> 5);
-    const int64_t row_begin = slab * rows_per_warp;
-    const int64_t row_end = min(n_rows, row_begin + rows_per_warp);
-    if (row_begin >= row_end) return;  // warp-uniform
+    const int slab = blockIdx.y * kNmWarps + (threadIdx.x >> 5);
+    const int64_t row_begin64 = static_cast<int64_t>(slab) * rows_per_warp;
+    if (row_begin64 >= n_rows) return;  // warp-uniform
+    const int row_begin = static_cast<int>(row_begin64);
+    const int rows = min(n_rows - row_begin, rows_per_warp);
 
     float c[8];
     load_factor8(factor, col, c);  // zero past d_in
     const int64_t left = n - col;
     const uint32_t valid = left >= 8 ? 0xffu : (left > 0 ? (1u << left) - 1u : 0u);
-    uint32_t *mdst = mask != nullptr ? mask + (col >> 5) : nullptr;
-    const uint32_t bias_bytes = static_cast<uint32_t>(0x80 - prune_count) * 0x01010101u;
+    const uint32_t bias = static_cast<uint32_t>(0x80 - prune_count) * 0x01010101u;
+    const uint32_t bias_lo = bias + 0x03020100u;
+    const uint32_t bias_hi = bias + (M == 4 ? 0x03020100u : 0x07060504u);
+    const bool store_word = mask != nullptr && (lane & 3) == 0 && left > 0;
 
-    for (int64_t r0 = row_begin; r0 < row_end; r0 += kNmRowsInFlight) {
+    // Row pointers advance by whole rows; row index times leading dimension is a 32x32->64
+    // multiply-add on the current pointer.
+    const uint16_t *wp = W + static_cast<int64_t>(row_begin) * ldw;
+    uint16_t *op = W_out != nullptr ? W_out + static_cast<int64_t>(row_begin) * ldo : nullptr;
+    uint32_t *mp = mask != nullptr ? mask + static_cast<int64_t>(row_begin) * mask_words + (col >> 5)
+                                   : nullptr;
+
+    int r = 0;
+    for (; r + kNmRowsInFlight <= rows; r += kNmRowsInFlight) {
         uint32_t p[kNmRowsInFlight][4];
 #pragma unroll
-        for (int u = 0; u < kNmRowsInFlight; ++u) {
-            if (r0 + u < row_end) {
-                load8<VEC, true>(W + (r0 + u) * ldw, col, n, p[u]);
-            } else {
-                p[u][0] = p[u][1] = p[u][2] = p[u][3] = 0u;
-            }
-        }
+        for (int u = 0; u < kNmRowsInFlight; ++u)
+            load8<VEC, true>(wp + static_cast<int64_t>(u) * ldw, col, n, p[u]);
 #pragma unroll
         for (int u = 0; u < kNmRowsInFlight; ++u) {
-            const int64_t r = r0 + u;
-            if (r >= row_end) break;  // warp-uniform
-            float w[8];
-            unpack8<BF16>(p[u], w);
-            uint32_t key[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-                key[j] = __float_as_uint(__fmul_rn(__fmul_rn(w[j], w[j]), c[j]));
-            uint32_t ra, rb;
-            nm_rank_bytes<M>(key, bias_bytes, ra, rb);
-            // half-word masks from the top bit of each rank byte (sign replication)
-            uint32_t m[4];
-            m[0] = prmt(ra, 0u, 0x9988u);
-            m[1] = prmt(ra, 0u, 0xbbaau);
-            m[2] = prmt(rb, 0u, 0x9988u);
-            m[3] = prmt(rb, 0u, 0xbbaau);
-            const uint32_t keep8 = halfmasks_to_bits(m) & valid;
-            if (W_out != nullptr) {
-#pragma unroll
-                for (int k = 0; k < 4; ++k) p[u][k] &= m[k];
-                store8<VEC>(W_out + r * ldo, col, n, p[u]);
-            }
+            uint16_t *orow = op != nullptr ? op + static_cast<int64_t>(u) * ldo : nullptr;
+            const uint32_t keep8 =
+                nm_process_row<BF16, VEC, M>(p[u], c, bias_lo, bias_hi, valid, orow, col, n);
             const uint32_t word = gather_mask_word(keep8, lane);
-            if (mdst != nullptr && (lane & 3) == 0 && left > 0) mdst[r * mask_words] = word;
+            if (store_word) mp[static_cast<int64_t>(u) * mask_words] = word;
         }
+        wp += static_cast<int64_t>(kNmRowsInFlight) * ldw;
+        if (op != nullptr) op += static_cast<int64_t>(kNmRowsInFlight) * ldo;
+        if (mp != nullptr) mp += static_cast<int64_t>(kNmRowsInFlight) * mask_words;
+    }
+    for (; r < rows; ++r) {  // fewer than kNmRowsInFlight rows left in the slab
+        uint32_t p[4];
+        load8<VEC, true>(wp, col, n, p);
+        const uint32_t keep8 =
+            nm_process_row<BF16, VEC, M>(p, c, bias_lo, bias_hi, valid, op, col, n);
+        const uint32_t word = gather_mask_word(keep8, lane);
+        if (store_word) *mp = word;
+        wp += ldw;
+        if (op != nullptr) op += ldo;
+        if (mp != nullptr) mp += mask_words;
     }
 }
 
@@ -141,7 +183,9 @@ sp_status launch_select_nm(const sp_ctx *ctx, const void *W, sp_dtype dtype, int
         rows_per_warp = (n_rows + max_grid_y * kNmWarps - 1) / (max_grid_y * kNmWarps);
         rows_per_warp = (rows_per_warp + kNmRowsInFlight - 1) / kNmRowsInFlight * kNmRowsInFlight;
     }
-    if (rows_per_warp > 0x7fffffffLL) return SP_ERR_SHAPE;
+    if (rows_per_warp > 0x7fffffffLL || n_rows > 0x7fffffffLL || ldw > 0x7fffffffLL ||
+        ldo > 0x7fffffffLL)
+        return SP_ERR_SHAPE;
     const int64_t slabs = (n_rows + rows_per_warp - 1) / rows_per_warp;
     const dim3 grid(static_cast<unsigned>(strips),
                     static_cast<unsigned>((slabs + kNmWarps - 1) / kNmWarps));
@@ -154,7 +198,8 @@ sp_status launch_select_nm(const sp_ctx *ctx, const void *W, sp_dtype dtype, int
     const int rpw = static_cast<int>(rows_per_warp);
 #define SP_LAUNCH(B, V, MM)                                                                  \
     select_nm_kernel<B, V, MM><<<grid, kNmThreads, 0, stream>>>(                              \
-        Wp, ldw, n_rows, n, rpw, ctx->factor, prune_count, mask, words, Op, ldo)
+        Wp, static_cast<int>(ldw), static_cast<int>(n_rows), n, rpw, ctx->factor, prune_count,   \
+        mask, static_cast<int>(words), Op, static_cast<int>(ldo))
 #define SP_LAUNCH_M(B, V)                                                                     \
     do {                                                                                      \
         if (M == 8) SP_LAUNCH(B, V, 8); else SP_LAUNCH(B, V, 4);                              \

@@ -97,6 +97,20 @@ __device__ __forceinline__ void zero_pruned(uint32_t (&p)[4], uint32_t keep) {
     }
 }
 
+// Asynchronous 16-byte copy global -> shared (bypassing L1).  src_bytes < 16 zero-fills the
+// rest; src_bytes == 0 reads nothing.
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src, int src_bytes) {
+    const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(gmem_src),
+                 "r"(src_bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
 // prmt.b32 in its generic mode: result byte k is byte (sel nibble k & 7) of the pair {a, b};
 // when bit 3 of the nibble is set the byte's sign bit is replicated over the whole byte.
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {

@@ -25,16 +25,14 @@ struct DeviceScalars {
     unsigned int ticket;  // arrival counter of the finalisation kernel (returns to 0)
 };
 
-// Powers of (1-alpha) and (1-beta) that the scan kernel needs, computed on the host in
-// fp64 and rounded once.
+// Powers of a = 1-alpha and b = 1-beta that the scan kernel needs (a lane owns P consecutive
+// weights), computed on the host in fp64 and rounded once.
 struct ScanConstants {
     float alpha, beta, la;
     float a, b;            // 1-alpha, 1-beta (rounded in fp32 like the definition)
-    float a_pow[8];        // a^(j+1)
-    float b_pow[8];
-    float a_lane[32];      // a^(8*lane)
+    float a_lane[32];      // a^(P*lane)
     float b_lane[32];
-    float a_step[5];       // a^(8*2^k)
+    float a_step[5];       // a^(P*2^k)
     float b_step[5];
 };
 
@@ -53,7 +51,7 @@ struct sp_ctx {
     double *partial;           // [kMaxSlabs][n_pad] fp64 partial column sums
     double *colsq;             // [n_pad]
     double *strip_sum;         // [strips]
-    float *factor;             // [n_pad] c_q, zero in the padding
+    float *factor;             // [n_pad + 256] c_q, zero in the padding
     sp::DeviceScalars *scalars;
 };
 

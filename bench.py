@@ -321,6 +321,30 @@ def gpu_arm(args):
         "clocks": clocks, "gpu_launches": int(launches),
     }
 
+    # End to end: the same pass with every input and output in pinned HOST memory, through the
+    # library's host-buffer entry points (copies inside the timed region).
+    if args.e2e_steps > 0:
+        hb = pipeline.allocate_host(mb, batch_tokens)
+        pipeline.prune_model_host(
+            pipeline.ModelBuffers(synth.Workload(**{**w.__dict__, "blocks": 1}), device,
+                                  mb.weights, mb.outputs, mb.masks, mb.acts, mb.ctxs),
+            hb, arg)                                           # warm-up: one block
+        barrier()
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.e2e_steps):
+            h2d, d2h = pipeline.prune_model_host(mb, hb, arg)
+        e1.record()
+        barrier()
+        e2e_ms = sharding.max_over_ranks(e0.elapsed_time(e1), world, device)
+        line["e2e"] = {"value": total_weights * args.e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
+                       "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                       "ms_per_step": e2e_ms / args.e2e_steps, "steps": args.e2e_steps,
+                       "note": "host buffers are pinned; one calibration batch and one block's "
+                               "weights are the host-side source for every batch / block"}
+        del hb
+
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import swiftprune_oracle as so
         cb = oracle_sample(w, so.max_threads())

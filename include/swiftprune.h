@@ -15,8 +15,7 @@
  *     The library owns only the context (O(d_in) device memory).
  *   - Calls enqueue work on the caller's stream (sp_stream = cudaStream_t passed
  *     as void*; NULL = the default stream) and return without synchronising,
- *     except sp_create, sp_destroy, sp_get_stats, sp_set_stats and
- *     the *_host entry point, which say so.
+ *     except sp_create, sp_destroy, sp_get_stats and sp_set_stats, which say so.
  *   - Arguments are validated on the host before anything is launched; a
  *     non-SP_OK status means nothing was enqueued by that call.  No call
  *     throws, traps or aborts.
@@ -220,6 +219,30 @@ sp_status sp_select_nm(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_row
  */
 sp_status sp_apply_mask(const void *W, sp_dtype dtype, int64_t n_rows, int64_t n_cols, int64_t ldw,
                         const uint32_t *mask, void *W_out, int64_t ldo, sp_stream stream);
+
+/* ------------------------------------------------------------------ host-buffer variants */
+
+/*
+ * The same operations (Algorithm 1 step 1; Section 3.3; Algorithm 1) for data that lives in
+ * HOST memory: X_host, W_host, mask_host and W_out_host are host pointers (pinned memory lets
+ * the transfers overlap the kernels; pageable memory works but copies synchronously).  The
+ * matrix is streamed through two device staging slots of 64 MiB owned by the context (created,
+ * together with two internal streams, by the first such call on a context - that call
+ * allocates): host->device copy, kernel and device->host copy of successive row chunks overlap.
+ * Work is ordered after everything already queued on `stream`, and `stream` completes only
+ * after the last result has reached the host; the calls themselves do not wait.  mask_host and
+ * W_out_host may each be NULL; W_out_host may equal W_host (same ld) for in-place pruning.
+ * Results are identical to the device-pointer calls.
+ */
+sp_status sp_calib_accumulate_host(sp_ctx *ctx, const void *X_host, sp_dtype dtype,
+                                   int64_t n_tokens, int64_t ldx, sp_stream stream);
+sp_status sp_select_nm_host(sp_ctx *ctx, const void *W_host, sp_dtype dtype, int64_t n_rows,
+                            int64_t ldw, int N, int M, uint32_t *mask_host, void *W_out_host,
+                            int64_t ldo, sp_stream stream);
+sp_status sp_select_unstructured_host(sp_ctx *ctx, const void *W_host, sp_dtype dtype,
+                                      int64_t n_rows, int64_t ldw, float sparsity,
+                                      uint32_t *mask_host, void *W_out_host, int64_t ldo,
+                                      sp_stream stream);
 
 /* ------------------------------------------------------------------ diagnostics */
 

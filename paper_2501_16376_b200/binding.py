@@ -27,7 +27,8 @@ SP_COUNTER_KEPT, SP_COUNTER_S_HAZARD, SP_NUM_COUNTERS = 0, 1, 2
 EXPORTS = (
     "sp_create", "sp_destroy", "sp_calib_reset", "sp_calib_accumulate", "sp_get_stats",
     "sp_set_stats", "sp_calib_stats_noalloc", "sp_score", "sp_la_for_sparsity", "sp_select_unstructured",
-    "sp_select_unstructured_ex", "sp_select_nm", "sp_apply_mask", "sp_status_string",
+    "sp_select_unstructured_ex", "sp_select_nm", "sp_apply_mask", "sp_calib_accumulate_host",
+    "sp_select_nm_host", "sp_select_unstructured_host", "sp_status_string",
     "sp_last_cuda_error", "sp_launch_count",
 )
 
@@ -64,6 +65,9 @@ def _load() -> ctypes.CDLL:
                                               vp, vp, i64, vp, vp]
     lib.sp_select_nm.argtypes = [vp, vp, ci, i64, i64, ci, ci, vp, vp, i64, vp]
     lib.sp_apply_mask.argtypes = [vp, ci, i64, i64, i64, vp, vp, i64, vp]
+    lib.sp_calib_accumulate_host.argtypes = [vp, vp, ci, i64, i64, vp]
+    lib.sp_select_nm_host.argtypes = [vp, vp, ci, i64, i64, ci, ci, vp, vp, i64, vp]
+    lib.sp_select_unstructured_host.argtypes = [vp, vp, ci, i64, i64, f32, vp, vp, i64, vp]
     lib.sp_status_string.argtypes = [ci]
     lib.sp_status_string.restype = ctypes.c_char_p
     lib.sp_last_cuda_error.restype = ctypes.c_char_p
@@ -94,11 +98,12 @@ def _dtype_of(t: torch.Tensor) -> int:
     raise SpError(SP_ERR_DTYPE, "expected a float16 or bfloat16 tensor, got %s" % t.dtype)
 
 
-def _matrix(t: torch.Tensor, what: str):
+def _matrix(t: torch.Tensor, what: str, host: bool = False):
     if t.dim() != 2 or (t.shape[1] > 1 and t.stride(1) != 1):
         raise SpError(SP_ERR_SHAPE, "%s must be 2-D with unit stride along its rows" % what)
-    if not t.is_cuda:
-        raise SpError(SP_ERR_INVALID_ARG, "%s must be a CUDA tensor" % what)
+    if t.is_cuda == host:
+        raise SpError(SP_ERR_INVALID_ARG,
+                      "%s must be a %s tensor" % (what, "CPU" if host else "CUDA"))
     ld = t.stride(0) if t.shape[0] > 1 else max(t.stride(0), t.shape[1])
     return t.data_ptr(), t.shape[0], t.shape[1], ld
 
@@ -233,6 +238,36 @@ class Context:
         _check(lib.sp_select_nm(self._h, ptr, _dtype_of(W), R, ld, int(N), int(M), _ptr(mask),
                                 optr, ldo, _stream(stream)))
         return mask, W_out
+
+
+class HostMixin:
+    """Host-buffer variants: tensors are CPU tensors (pinned for overlap); see the C header."""
+
+    def sp_calib_accumulate_host(self, X: torch.Tensor, stream=None):
+        ptr, T, n, ld = _matrix(X, "X", host=True)
+        if n != self.d_in:
+            raise SpError(SP_ERR_SHAPE, "X has %d channels, context has %d" % (n, self.d_in))
+        _check(lib.sp_calib_accumulate_host(self._h, ptr, _dtype_of(X), T, ld, _stream(stream)))
+
+    def sp_select_nm_host(self, W, N, M, mask, W_out, stream=None):
+        ptr, R, n, ld = _matrix(W, "W", host=True)
+        self._check_width(n)
+        optr, ldo = (None, ld) if W_out is None else (_matrix(W_out, "W_out", host=True)[0],
+                                                      _matrix(W_out, "W_out", host=True)[3])
+        _check(lib.sp_select_nm_host(self._h, ptr, _dtype_of(W), R, ld, int(N), int(M),
+                                     _ptr(mask), optr, ldo, _stream(stream)))
+
+    def sp_select_unstructured_host(self, W, sparsity, mask, W_out, stream=None):
+        ptr, R, n, ld = _matrix(W, "W", host=True)
+        self._check_width(n)
+        optr, ldo = (None, ld) if W_out is None else (_matrix(W_out, "W_out", host=True)[0],
+                                                      _matrix(W_out, "W_out", host=True)[3])
+        _check(lib.sp_select_unstructured_host(self._h, ptr, _dtype_of(W), R, ld, float(sparsity),
+                                               _ptr(mask), optr, ldo, _stream(stream)))
+
+
+for _name in ("sp_calib_accumulate_host", "sp_select_nm_host", "sp_select_unstructured_host"):
+    setattr(Context, _name, getattr(HostMixin, _name))
 
 
 def sp_apply_mask(W: torch.Tensor, mask: torch.Tensor, W_out: torch.Tensor | None = None,

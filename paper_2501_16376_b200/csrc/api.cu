@@ -91,6 +91,7 @@ sp_status sp_create(sp_ctx **out, int64_t d_in, int device) {
     ctx->n_tokens = 0;
     ctx->slabs_valid = 0;
     ctx->dirty = false;
+    ctx->host_pipe = nullptr;
     e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
     if (e != cudaSuccess) { delete ctx; return cuda_fail(e); }
     ctx->calib_blocks_per_sm = calib_query_blocks_per_sm();
@@ -125,6 +126,7 @@ sp_status sp_destroy(sp_ctx *ctx) {
     if (ctx == nullptr) return SP_OK;
     DeviceGuard guard(ctx->device);
     cudaDeviceSynchronize();
+    host_pipe_destroy(ctx->host_pipe);
     cudaFree(ctx->partial);
     cudaFree(ctx->colsq);
     cudaFree(ctx->strip_sum);
@@ -312,6 +314,57 @@ sp_status sp_apply_mask(const void *W, sp_dtype dtype, int64_t n_rows, int64_t n
     if (W_out == W && ldo != ldw) return SP_ERR_SHAPE;
     return launch_apply_mask(W, dtype, n_rows, n_cols, ldw, mask, W_out, ldo,
                              static_cast<cudaStream_t>(stream));
+}
+
+sp_status sp_calib_accumulate_host(sp_ctx *ctx, const void *X_host, sp_dtype dtype,
+                                   int64_t n_tokens, int64_t ldx, sp_stream stream) {
+    if (ctx == nullptr) return SP_ERR_INVALID_ARG;
+    if (!valid_dtype(dtype)) return SP_ERR_DTYPE;
+    if (n_tokens < 0) return SP_ERR_INVALID_ARG;
+    if (n_tokens == 0) return SP_OK;
+    if (X_host == nullptr) return SP_ERR_INVALID_ARG;
+    if (ldx < ctx->d_in) return SP_ERR_SHAPE;
+    DeviceGuard guard(ctx->device);
+    if (guard.error() != cudaSuccess) return cuda_fail(guard.error());
+    return host_calib_accumulate(ctx, X_host, dtype, n_tokens, ldx, static_cast<cudaStream_t>(stream));
+}
+
+sp_status sp_select_nm_host(sp_ctx *ctx, const void *W_host, sp_dtype dtype, int64_t n_rows,
+                            int64_t ldw, int N, int M, uint32_t *mask_host, void *W_out_host,
+                            int64_t ldo, sp_stream stream) {
+    sp_status st = check_matrix_args(ctx, W_host, dtype, n_rows, ldw, W_out_host, ldo);
+    if (st != SP_OK) return st;
+    if (M != 4 && M != 8) return SP_ERR_INVALID_ARG;
+    if (N <= 0 || N >= M) return SP_ERR_INVALID_ARG;
+    if (ctx->d_in % M != 0) return SP_ERR_SHAPE;
+    if (ctx->n_tokens <= 0) return SP_ERR_STATE;
+    DeviceGuard guard(ctx->device);
+    if (guard.error() != cudaSuccess) return cuda_fail(guard.error());
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    st = ensure_finalized(ctx, s);
+    if (st != SP_OK) return st;
+    return host_select(ctx, 0, W_host, dtype, n_rows, ldw, N, M, nullptr, mask_host, W_out_host, ldo, s);
+}
+
+sp_status sp_select_unstructured_host(sp_ctx *ctx, const void *W_host, sp_dtype dtype,
+                                      int64_t n_rows, int64_t ldw, float sparsity,
+                                      uint32_t *mask_host, void *W_out_host, int64_t ldo,
+                                      sp_stream stream) {
+    sp_status st = check_matrix_args(ctx, W_host, dtype, n_rows, ldw, W_out_host, ldo);
+    if (st != SP_OK) return st;
+    sp_ewma_params p;
+    p.alpha = 0.125f;
+    p.beta = 0.125f;
+    p.s_update = SP_S_FROZEN;
+    st = sp_la_for_sparsity(sparsity, &p.la);
+    if (st != SP_OK) return st;
+    if (ctx->n_tokens <= 0) return SP_ERR_STATE;
+    DeviceGuard guard(ctx->device);
+    if (guard.error() != cudaSuccess) return cuda_fail(guard.error());
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    st = ensure_finalized(ctx, s);
+    if (st != SP_OK) return st;
+    return host_select(ctx, 1, W_host, dtype, n_rows, ldw, 0, 0, &p, mask_host, W_out_host, ldo, s);
 }
 
 const char *sp_status_string(sp_status status) {

@@ -36,6 +36,8 @@ struct ScanConstants {
     float b_step[5];
 };
 
+struct HostPipe;  // staging slots and streams of the host-buffer entry points (host_pipe.cu)
+
 }  // namespace sp
 
 struct sp_ctx {
@@ -53,6 +55,7 @@ struct sp_ctx {
     double *strip_sum;         // [strips]
     float *factor;             // [n_pad + 256] c_q, zero in the padding
     sp::DeviceScalars *scalars;
+    sp::HostPipe *host_pipe;   // created by the first host-buffer call
 };
 
 namespace sp {
@@ -93,6 +96,14 @@ sp_status launch_select_nm(const sp_ctx *ctx, const void *W, sp_dtype dtype, int
 sp_status launch_select_ewma(const sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
                              int64_t ldw, const sp_ewma_params &p, uint32_t *mask, void *W_out,
                              int64_t ldo, unsigned long long *counters, cudaStream_t stream);
+
+// host_pipe.cu
+void host_pipe_destroy(HostPipe *hp);
+sp_status host_calib_accumulate(sp_ctx *ctx, const void *X_host, sp_dtype dtype, int64_t n_tokens,
+                                int64_t ldx, cudaStream_t stream);
+sp_status host_select(sp_ctx *ctx, int kind, const void *W_host, sp_dtype dtype, int64_t n_rows,
+                      int64_t ldw, int N, int M, const sp_ewma_params *params,
+                      uint32_t *mask_host, void *W_out_host, int64_t ldo, cudaStream_t stream);
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 

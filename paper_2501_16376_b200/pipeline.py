@@ -117,3 +117,55 @@ def prune_model(mb: ModelBuffers, mode_arg, batch_tokens: int, phase_events=None
                 phase_events.append(("calib", e0, e1, d_in))
                 phase_events.append(("select", e1, e2, d_in))
     return {"calib": n_calib, "finalize": n_final, "select": n_select}
+
+
+@dataclass
+class HostBuffers:
+    """Pinned host copies for the end-to-end path: one calibration batch per layer input and the
+    weights / outputs / masks of one block (reused for every block: the bytes that cross the
+    bus per step are those of the whole model)."""
+    x_batch: dict = field(default_factory=dict)    # input name -> [batch_tokens, d_in]
+    weights: list = field(default_factory=list)    # per layer of a block
+    outputs: list = field(default_factory=list)
+    masks: list = field(default_factory=list)
+
+
+def allocate_host(mb: ModelBuffers, batch_tokens: int) -> HostBuffers:
+    hb = HostBuffers()
+    w = mb.workload
+    for name, d_in in w.input_widths().items():
+        hb.x_batch[name] = mb.acts[name][:batch_tokens].cpu().pin_memory()
+    for li, layer in enumerate(w.layers):
+        hb.weights.append(mb.weights[0][li].cpu().pin_memory())
+        hb.outputs.append(torch.empty(layer.d_out, layer.d_in, dtype=w.torch_dtype).pin_memory())
+        hb.masks.append(torch.empty(layer.d_out, (layer.d_in + 31) // 32,
+                                    dtype=torch.int32).pin_memory())
+    return hb
+
+
+def prune_model_host(mb: ModelBuffers, hb: HostBuffers, mode_arg, stream=None):
+    """One pass of the whole hot path with every input and output in host memory, through the
+    host-buffer entry points.  Returns (h2d_bytes, d2h_bytes) that crossed the bus."""
+    w = mb.workload
+    h2d = d2h = 0
+    for b in range(w.blocks):
+        for name, d_in in w.input_widths().items():
+            ctx = mb.ctxs[name]
+            ctx.sp_calib_reset(stream)
+            xb = hb.x_batch[name]
+            for t0 in range(0, w.tokens, xb.shape[0]):
+                rows = min(xb.shape[0], w.tokens - t0)
+                ctx.sp_calib_accumulate_host(xb[:rows], stream)
+                h2d += rows * d_in * 2
+            for li, layer in enumerate(w.layers):
+                if layer.input != name:
+                    continue
+                if w.mode == "nm":
+                    ctx.sp_select_nm_host(hb.weights[li], mode_arg[0], mode_arg[1], hb.masks[li],
+                                          hb.outputs[li], stream)
+                else:
+                    ctx.sp_select_unstructured_host(hb.weights[li], mode_arg, hb.masks[li],
+                                                    hb.outputs[li], stream)
+                h2d += layer.d_out * layer.d_in * 2
+                d2h += layer.d_out * layer.d_in * 2 + hb.masks[li].numel() * 4
+    return h2d, d2h

@@ -400,3 +400,46 @@ def test_launch_counter_counts_kernels(sp):
         ctx.sp_calib_accumulate(_activations(1, 64, n, torch.float16))   # 1
         ctx.sp_select_nm(_gen(1, (8, n), torch.float16, 0.02), 2, 4)      # finalise + select
     assert sp.sp_launch_count() - before == 3
+
+
+# ------------------------------------------------------------------ host-buffer entry points
+
+@pytest.mark.parametrize("pinned", [True, False])
+def test_host_buffer_calls_match_device_calls(sp, pinned):
+    # wide enough that the 64 MiB staging slots are cycled several times
+    R, n, T = 20000, 4096, 40000
+    W = _gen(61, (R, n), torch.float16, 0.02)
+    X = _activations(62, T, n, torch.float16)
+
+    def host(t):
+        h = t.cpu()
+        return h.pin_memory() if pinned else h
+
+    Wh, Xh = host(W), host(X)
+    words = (n + 31) // 32
+    with sp.Context(n) as dev_ctx, sp.Context(n) as host_ctx:
+        dev_ctx.sp_calib_accumulate(X)
+        host_ctx.sp_calib_accumulate_host(Xh[:15000])
+        host_ctx.sp_calib_accumulate_host(Xh[15000:])
+        c_dev, S_dev, f_dev, _ = dev_ctx.sp_get_stats()
+        c_host, S_host, f_host, ntok = host_ctx.sp_get_stats()
+        assert ntok == T
+        assert P.rel_err(c_host.numpy(), c_dev.numpy()) <= 1e-6   # chunking changes slab cuts only
+        host_ctx.sp_set_stats(c_dev, T)                            # identical statistics from here on
+        m_dev, o_dev = dev_ctx.sp_select_nm(W, 2, 4)
+        m_host = host(torch.zeros(R, words, dtype=torch.int32))
+        o_host = host(torch.zeros(R, n, dtype=torch.float16))
+        host_ctx.sp_select_nm_host(Wh, 2, 4, m_host, o_host)
+        torch.cuda.synchronize()
+        assert torch.equal(m_host, m_dev.cpu())
+        assert torch.equal(o_host.view(torch.int16), o_dev.cpu().view(torch.int16))
+        m_dev, o_dev = dev_ctx.sp_select_unstructured(W, 0.5)
+        host_ctx.sp_select_unstructured_host(Wh, 0.5, m_host, o_host)
+        torch.cuda.synchronize()
+        assert torch.equal(m_host, m_dev.cpu())
+        assert torch.equal(o_host.view(torch.int16), o_dev.cpu().view(torch.int16))
+        # in place on the host, mask not wanted
+        Wh2 = host(W)
+        host_ctx.sp_select_nm_host(Wh2, 2, 4, None, Wh2)
+        torch.cuda.synchronize()
+        assert torch.equal(Wh2.view(torch.int16), dev_ctx.sp_select_nm(W, 2, 4)[1].cpu().view(torch.int16))

@@ -279,26 +279,29 @@ def gpu_arm(args):
 
     calib_ms = sum(a.elapsed_time(b) for k, a, b, _ in phase_events if k == "calib")
     select_ms = sum(a.elapsed_time(b) for k, a, b, _ in phase_events if k == "select")
-    x_elements = sum(w.tokens * d for d in w.input_widths().values()) * w.blocks * args.steps
+    final_ms = sum(a.elapsed_time(b) for k, a, b, _ in phase_events if k == "finalize")
+    x_elements = sum(u for k, _, _, u in phase_events if k == "calib")
+    sel_weights = sum(u for k, _, _, u in phase_events if k == "select")
     calib_launches = counts["calib"] * args.steps
     select_launches = counts["select"] * args.steps
     peak, peak_kind = measured_peaks()
     calib_gbs = CALIB_BYTES_PER_ELEMENT * x_elements / (calib_ms * 1e-3) / 1e9
-    select_gbs = SELECT_BYTES_PER_WEIGHT * w.total_weights() * args.steps / (select_ms * 1e-3) / 1e9
+    select_gbs = SELECT_BYTES_PER_WEIGHT * sel_weights / (select_ms * 1e-3) / 1e9
     roofline = {
         "kernel": "calib_accumulate_kernel", "bound": "hbm", "achieved": calib_gbs, "peak": peak,
         "peak_kind": peak_kind, "unit": "GB/s", "frac": calib_gbs / peak, "traffic": None,
         "avg_launch_ms": calib_ms / calib_launches,
         "bytes_per_launch": CALIB_BYTES_PER_ELEMENT * x_elements / calib_launches,
+        "note": "events bracket the back-to-back accumulate launches of one layer input",
     }
     roofline_select = {
         "kernel": "select_nm_kernel" if w.mode == "nm" else "ewma_scan_kernel",
         "bound": "hbm", "achieved": select_gbs, "peak": peak, "peak_kind": peak_kind,
         "unit": "GB/s", "frac": select_gbs / peak, "frac_of_8TBs": select_gbs / 8000.0,
         "traffic": None, "avg_launch_ms": select_ms / select_launches,
-        "bytes_per_launch": SELECT_BYTES_PER_WEIGHT * w.total_weights() * args.steps / select_launches,
-        "weights_per_sec": w.total_weights() * args.steps / (select_ms * 1e-3),
-        "note": "phase time includes one finalisation launch per layer input",
+        "bytes_per_launch": SELECT_BYTES_PER_WEIGHT * sel_weights / select_launches,
+        "weights_per_sec": sel_weights / (select_ms * 1e-3),
+        "note": "events bracket every selection launch on its own",
     }
 
     line = {
@@ -315,6 +318,7 @@ def gpu_arm(args):
                               + 4 * w.total_weights()) / 1e9),
                    "parallelism": "independent models per rank" if world > 1 else "single GPU"},
         "whole_model_prune_s": {"calib": calib_ms / args.steps * 1e-3,
+                                "finalize": final_ms / args.steps * 1e-3,
                                 "select_apply": select_ms / args.steps * 1e-3,
                                 "total": elapsed_ms / args.steps * 1e-3},
         "roofline": roofline, "roofline_select": roofline_select,

@@ -25,6 +25,10 @@ __global__ void __launch_bounds__(kCalibThreads)
 calib_accumulate_kernel(const uint16_t *__restrict__ X, int64_t ldx, int64_t n_tokens, int64_t n,
                         int64_t rows_per_slab, double *__restrict__ partial, int64_t n_pad,
                         int first_fresh_slab) {
+    // Programmatic dependent launch: the next kernel in the stream may start as soon as this
+    // grid's CTAs are all resident, and this kernel's own streaming phase may overlap the tail of
+    // the previous one; only the read-modify-write of the partial sums below waits for it.
+    pdl_launch_dependents();
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const int strip = blockIdx.x;
@@ -67,6 +71,7 @@ calib_accumulate_kernel(const uint16_t *__restrict__ X, int64_t ldx, int64_t n_t
 #pragma unroll
     for (int j = 0; j < 8; ++j) sm[warp][lane * 8 + j] = acc[j];
     __syncthreads();
+    pdl_wait();  // earlier kernels' partial sums are final
     const int t = threadIdx.x;
     const int64_t ch = static_cast<int64_t>(strip) * kStripChannels + t;
     if (ch < n) {
@@ -92,11 +97,23 @@ finalize_kernel(const double *__restrict__ partial, int slabs_valid, int64_t n, 
                 float *__restrict__ factor, DeviceScalars *__restrict__ scalars) {
     __shared__ double red[kStripChannels];
     __shared__ bool is_last;
+    pdl_launch_dependents();
+    pdl_wait();  // all partial sums are in place
     const int t = threadIdx.x;
     const int64_t ch = static_cast<int64_t>(blockIdx.x) * kStripChannels + t;
     double v = 0.0;
     if (ch < n) {
-        for (int s = 0; s < slabs_valid; ++s) v += partial[static_cast<int64_t>(s) * n_pad + ch];
+        // ascending slab order; eight loads in flight at a time
+        const double *src = partial + ch;
+        int s = 0;
+        for (; s + 8 <= slabs_valid; s += 8) {
+            double x[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) x[k] = __ldcg(src + static_cast<int64_t>(s + k) * n_pad);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) v += x[k];
+        }
+        for (; s < slabs_valid; ++s) v += __ldcg(src + static_cast<int64_t>(s) * n_pad);
     }
     colsq[ch] = v;  // ch < n_pad always; padding gets 0
     red[t] = v;
@@ -115,11 +132,21 @@ finalize_kernel(const double *__restrict__ partial, int slabs_valid, int64_t n, 
     if (!is_last) return;
     __threadfence();
 
-    __shared__ double S_sh;
+    // S: every thread adds the strip totals t, t+256, ... in ascending order, then the same
+    // fixed tree as above combines the 256 partial sums (deterministic, loads in parallel).
+    {
+        double part = 0.0;
+        for (int s = t; s < strips; s += kStripChannels) part += __ldcg(strip_sum + s);
+        red[t] = part;
+    }
+    __syncthreads();
+    for (int half = kStripChannels / 2; half > 0; half >>= 1) {
+        if (t < half) red[t] += red[t + half];
+        __syncthreads();
+    }
+    const double S = red[0];
+    const float S32 = static_cast<float>(S);
     if (t == 0) {
-        double S = 0.0;
-        for (int s = 0; s < strips; ++s) S += __ldcg(strip_sum + s);
-        const float S32 = static_cast<float>(S);
         int flags = 0;
         if (!(S > 0.0) || isinf(S) || isnan(S) || isinf(S32)) flags |= kFlagDegenerate;
         // "S - w^2" leaves S unchanged in binary32 whenever w^2 is below a quarter of the
@@ -134,19 +161,28 @@ finalize_kernel(const double *__restrict__ partial, int slabs_valid, int64_t n, 
         scalars->hazard_w2 = hazard;
         scalars->flags = flags;
         scalars->ticket = 0u;
-        S_sh = S;
     }
-    __syncthreads();
-    const float S32 = static_cast<float>(S_sh);
-    for (int64_t q = t; q < n_pad; q += kStripChannels) {
-        float c = 0.0f;
-        if (q < n) {
-            const float x2 = static_cast<float>(__ldcg(colsq + q));
-            const float u = __fdiv_rn(x2, S32);
-            const float den = __fsub_rn(1.0f, u);
-            c = __fdiv_rn(0.5f, den);
+    // per-channel factors, eight channels per thread in flight
+    for (int64_t q0 = t; q0 < n_pad; q0 += 8 * kStripChannels) {
+        double x[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int64_t q = q0 + static_cast<int64_t>(k) * kStripChannels;
+            x[k] = q < n ? __ldcg(colsq + q) : 0.0;
         }
-        factor[q] = c;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int64_t q = q0 + static_cast<int64_t>(k) * kStripChannels;
+            if (q < n_pad) {
+                float c = 0.0f;
+                if (q < n) {
+                    const float u = __fdiv_rn(static_cast<float>(x[k]), S32);
+                    const float den = __fsub_rn(1.0f, u);
+                    c = __fdiv_rn(0.5f, den);
+                }
+                factor[q] = c;
+            }
+        }
     }
 }
 
@@ -180,15 +216,21 @@ sp_status launch_calib_accumulate(sp_ctx *ctx, const void *X, sp_dtype dtype, in
     const bool bf16 = dtype == SP_BF16;
     dim3 grid(static_cast<unsigned>(ctx->strips), static_cast<unsigned>(slabs));
     const uint16_t *Xp = static_cast<const uint16_t *>(X);
+    PdlConfig pdl(grid, dim3(kCalibThreads), stream);
+    double *partial = ctx->partial;
+    int64_t n_pad = ctx->n_pad;
+    int first_fresh = ctx->slabs_valid;
+    cudaError_t launch_err = cudaSuccess;
 #define SP_LAUNCH(B, V)                                                                       \
-    calib_accumulate_kernel<B, V><<<grid, kCalibThreads, 0, stream>>>(                        \
-        Xp, ldx, n_tokens, n, rows_per_slab, ctx->partial, ctx->n_pad, ctx->slabs_valid)
+    launch_err = cudaLaunchKernelEx(&pdl.cfg, calib_accumulate_kernel<B, V>, Xp, ldx, n_tokens, n, \
+                                    rows_per_slab, partial, n_pad, first_fresh)
     if (bf16) {
         if (vec) SP_LAUNCH(true, true); else SP_LAUNCH(true, false);
     } else {
         if (vec) SP_LAUNCH(false, true); else SP_LAUNCH(false, false);
     }
 #undef SP_LAUNCH
+    if (launch_err != cudaSuccess) return cuda_fail(launch_err);
     sp_status st = check_launch();
     if (st != SP_OK) return st;
     if (slabs > ctx->slabs_valid) ctx->slabs_valid = static_cast<int>(slabs);
@@ -198,9 +240,12 @@ sp_status launch_calib_accumulate(sp_ctx *ctx, const void *X, sp_dtype dtype, in
 }
 
 sp_status launch_finalize(sp_ctx *ctx, cudaStream_t stream) {
-    finalize_kernel<<<ctx->strips, kStripChannels, 0, stream>>>(
-        ctx->partial, ctx->slabs_valid, ctx->d_in, ctx->n_pad, ctx->strips, ctx->colsq,
-        ctx->strip_sum, ctx->factor, ctx->scalars);
+    PdlConfig pdl(dim3(ctx->strips), dim3(kStripChannels), stream);
+    const double *partial = ctx->partial;
+    cudaError_t e = cudaLaunchKernelEx(&pdl.cfg, finalize_kernel, partial, ctx->slabs_valid,
+                                       ctx->d_in, ctx->n_pad, ctx->strips, ctx->colsq,
+                                       ctx->strip_sum, ctx->factor, ctx->scalars);
+    if (e != cudaSuccess) return cuda_fail(e);
     sp_status st = check_launch();
     if (st == SP_OK) ctx->dirty = false;
     return st;

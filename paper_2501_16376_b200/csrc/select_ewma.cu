@@ -91,6 +91,8 @@ ewma_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
                  const __grid_constant__ ScanConstants sc, uint32_t *__restrict__ mask,
                  int mask_words, uint16_t *__restrict__ W_out, int ldo,
                  unsigned long long *__restrict__ counters) {
+    pdl_launch_dependents();
+    pdl_wait();  // the per-channel factors come from an earlier kernel of the stream
     const int lane = threadIdx.x & 31;
     const int row = blockIdx.x * kEwmaWarps + (threadIdx.x >> 5);
     if (row >= n_rows) return;  // warp-uniform
@@ -367,10 +369,15 @@ sp_status launch_select_ewma(const sp_ctx *ctx, const void *W, sp_dtype dtype, i
     const bool vec = aligned16(W) && ldw % 8 == 0 && n % 8 == 0 &&
                      (W_out == nullptr || (aligned16(W_out) && ldo % 8 == 0));
     const unsigned grid = static_cast<unsigned>(blocks);
+    PdlConfig pdl(dim3(grid), dim3(kEwmaThreads), stream);
+    const float *factor = ctx->factor;
+    const DeviceScalars *scalars = ctx->scalars;
+    cudaError_t launch_err = cudaSuccess;
 #define SP_LAUNCH_C(B, V, C)                                                                 \
-    ewma_scan_kernel<B, V, C><<<grid, kEwmaThreads, 0, stream>>>(                            \
-        Wp, static_cast<int>(ldw), static_cast<int>(n_rows), static_cast<int>(n), ctx->factor,   \
-        ctx->scalars, sc, mask, static_cast<int>(words), Op, static_cast<int>(ldo), counters)
+    launch_err = cudaLaunchKernelEx(&pdl.cfg, ewma_scan_kernel<B, V, C>, Wp,                  \
+                                    static_cast<int>(ldw), static_cast<int>(n_rows),          \
+                                    static_cast<int>(n), factor, scalars, sc, mask,           \
+                                    static_cast<int>(words), Op, static_cast<int>(ldo), counters)
 #define SP_LAUNCH(B, V)                                                                      \
     do {                                                                                     \
         if (counters != nullptr) SP_LAUNCH_C(B, V, true); else SP_LAUNCH_C(B, V, false);     \
@@ -382,6 +389,7 @@ sp_status launch_select_ewma(const sp_ctx *ctx, const void *W, sp_dtype dtype, i
     }
 #undef SP_LAUNCH
 #undef SP_LAUNCH_C
+    if (launch_err != cudaSuccess) return cuda_fail(launch_err);
     return check_launch();
 }
 

@@ -111,6 +111,8 @@ select_nm_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int64_t n,
                  int rows_per_warp, const float *__restrict__ factor, int prune_count,
                  uint32_t *__restrict__ mask, int mask_words, uint16_t *__restrict__ W_out,
                  int ldo) {
+    pdl_launch_dependents();
+    pdl_wait();  // the per-channel factors come from an earlier kernel of the stream
     const int lane = threadIdx.x & 31;
     const int64_t col = static_cast<int64_t>(blockIdx.x) * kStripChannels + lane * 8;
     const int slab = blockIdx.y * kNmWarps + (threadIdx.x >> 5);
@@ -196,10 +198,14 @@ sp_status launch_select_nm(const sp_ctx *ctx, const void *W, sp_dtype dtype, int
     const int64_t words = (n + 31) / 32;
     const int prune_count = M - N;
     const int rpw = static_cast<int>(rows_per_warp);
+    PdlConfig pdl(grid, dim3(kNmThreads), stream);
+    const float *factor = ctx->factor;
+    cudaError_t launch_err = cudaSuccess;
 #define SP_LAUNCH(B, V, MM)                                                                  \
-    select_nm_kernel<B, V, MM><<<grid, kNmThreads, 0, stream>>>(                              \
-        Wp, static_cast<int>(ldw), static_cast<int>(n_rows), n, rpw, ctx->factor, prune_count,   \
-        mask, static_cast<int>(words), Op, static_cast<int>(ldo))
+    launch_err = cudaLaunchKernelEx(&pdl.cfg, select_nm_kernel<B, V, MM>, Wp,                 \
+                                    static_cast<int>(ldw), static_cast<int>(n_rows), n, rpw,  \
+                                    factor, prune_count, mask, static_cast<int>(words), Op,   \
+                                    static_cast<int>(ldo))
 #define SP_LAUNCH_M(B, V)                                                                     \
     do {                                                                                      \
         if (M == 8) SP_LAUNCH(B, V, 8); else SP_LAUNCH(B, V, 4);                              \
@@ -211,6 +217,7 @@ sp_status launch_select_nm(const sp_ctx *ctx, const void *W, sp_dtype dtype, int
     }
 #undef SP_LAUNCH_M
 #undef SP_LAUNCH
+    if (launch_err != cudaSuccess) return cuda_fail(launch_err);
     return check_launch();
 }
 

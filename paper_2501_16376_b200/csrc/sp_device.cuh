@@ -97,6 +97,14 @@ __device__ __forceinline__ void zero_pruned(uint32_t (&p)[4], uint32_t keep) {
     }
 }
 
+// Programmatic dependent launch: let the next kernel of the stream be scheduled early / wait
+// until every earlier kernel of the stream has completed and its writes are visible.  Both are
+// no-ops for kernels launched without the attribute.
+__device__ __forceinline__ void pdl_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;");
+}
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // Asynchronous 16-byte copy global -> shared (bypassing L1).  src_bytes < 16 zero-fills the
 // rest; src_bytes == 0 reads nothing.
 __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src, int src_bytes) {

@@ -105,6 +105,24 @@ sp_status host_select(sp_ctx *ctx, int kind, const void *W_host, sp_dtype dtype,
                       int64_t ldw, int N, int M, const sp_ewma_params *params,
                       uint32_t *mask_host, void *W_out_host, int64_t ldo, cudaStream_t stream);
 
+// Launch configuration with programmatic dependent launch allowed: the kernel may be scheduled
+// while the previous kernel of the stream drains; every kernel launched this way executes
+// griddepcontrol.wait before it touches memory an earlier kernel may still be writing.
+struct PdlConfig {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    PdlConfig(dim3 grid, dim3 block, cudaStream_t stream) : cfg{}, attr{} {
+        cfg.gridDim = grid;
+        cfg.blockDim = block;
+        cfg.dynamicSmemBytes = 0;
+        cfg.stream = stream;
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    }
+};
+
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace sp

@@ -89,33 +89,44 @@ def select_layer(ctx: sp.Context, w: synth.Workload, W, mask, W_out, mode_arg, s
 
 def prune_model(mb: ModelBuffers, mode_arg, batch_tokens: int, phase_events=None, stream=None):
     """One pass of the whole hot path over the model: for every block and every distinct layer
-    input, accumulate the calibration statistics, then select + write back every layer that
-    reads this input.  phase_events, if given, is a list that receives (kind, start, end)
-    CUDA-event triples for the calibration and selection phases.  Returns launch counts."""
+    input, accumulate the calibration statistics, finalise them, then select + write back every
+    layer that reads this input.  phase_events, if given, is a list that receives
+    (kind, start_event, end_event, units) tuples: one "calib" entry per layer input (units =
+    activation elements), one "select" entry per selection launch (units = weights) and one
+    "finalize" entry per layer input.  Returns launch counts."""
     w = mb.workload
     n_calib = n_select = n_final = 0
+
+    def mark():
+        e = torch.cuda.Event(enable_timing=True)
+        e.record(stream)
+        return e
+
     for b in range(w.blocks):
         for name, d_in in w.input_widths().items():
             ctx = mb.ctxs[name]
+            X = mb.acts[name]
             if phase_events is not None:
-                e0 = torch.cuda.Event(enable_timing=True)
-                e1 = torch.cuda.Event(enable_timing=True)
-                e2 = torch.cuda.Event(enable_timing=True)
-                e0.record(stream)
-            n_calib += calibrate_input(ctx, mb.acts[name], batch_tokens, stream)
+                e0 = mark()
+            n_calib += calibrate_input(ctx, X, batch_tokens, stream)
             if phase_events is not None:
-                e1.record(stream)
+                e1 = mark()
+            ctx.sp_score(None, stream=stream)          # finalisation only
             n_final += 1
+            if phase_events is not None:
+                e2 = mark()
+                phase_events.append(("calib", e0, e1, X.shape[0] * d_in))
+                phase_events.append(("finalize", e1, e2, d_in))
             for li, layer in enumerate(w.layers):
                 if layer.input != name:
                     continue
+                if phase_events is not None:
+                    s0 = mark()
                 select_layer(ctx, w, mb.weights[b][li], mb.masks[b][li], mb.outputs[b][li],
                              mode_arg, stream)
                 n_select += 1
-            if phase_events is not None:
-                e2.record(stream)
-                phase_events.append(("calib", e0, e1, d_in))
-                phase_events.append(("select", e1, e2, d_in))
+                if phase_events is not None:
+                    phase_events.append(("select", s0, mark(), layer.d_out * layer.d_in))
     return {"calib": n_calib, "finalize": n_final, "select": n_select}
 
 

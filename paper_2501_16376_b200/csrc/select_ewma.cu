@@ -42,9 +42,10 @@ constexpr int kEwmaHalves = kEwmaPerLane / 8;     // 16-byte pieces per lane and
 constexpr bool kEwmaRing = SP_EWMA_RING != 0;     // stage tiles through shared memory
 constexpr int kEwmaTile = 32 * kEwmaPerLane;      // weights per warp tile
 #ifndef SP_EWMA_STAGES
-#define SP_EWMA_STAGES 6
+#define SP_EWMA_STAGES 4
 #endif
-constexpr int kEwmaStages = SP_EWMA_STAGES;       // tiles of a row in flight per warp (ring in smem)
+constexpr int kEwmaStages = SP_EWMA_STAGES;       // ring slots per warp (a power of two)
+static_assert((kEwmaStages & (kEwmaStages - 1)) == 0, "ring size must be a power of two");
 
 // Running packed maximum of |w| (two 16-bit floats per word).
 template <bool BF16>
@@ -126,7 +127,7 @@ ewma_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
         if constexpr (RING) {
             if (t < tiles) {
                 const int c0 = t * kEwmaTile + lane * kEwmaPerLane;
-                uint4 *slot = my_ring + (t % kEwmaStages) * kSlot;
+                uint4 *slot = my_ring + (t & (kEwmaStages - 1)) * kSlot;
 #pragma unroll
                 for (int h = 0; h < kEwmaHalves; ++h)
                     cp_async16(slot + 32 * h, wrow + min(c0 + 8 * h, n - 8),
@@ -150,7 +151,7 @@ ewma_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
         if constexpr (RING) {
             issue_tile(tile + kEwmaStages - 1);
             cp_async_wait<kEwmaStages - 1>();
-            const uint4 *slot = my_ring + (tile % kEwmaStages) * kSlot;
+            const uint4 *slot = my_ring + (tile & (kEwmaStages - 1)) * kSlot;
 #pragma unroll
             for (int h = 0; h < kEwmaHalves; ++h) {
                 const uint4 v = slot[32 * h];
@@ -200,7 +201,7 @@ ewma_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
             q[j] = fmaf(neg_alpha, E_run, L[j]);
             E_run = fmaf(a, E_run, L[j]);
             dabs[j] = fabsf(fmaf(alpha, E_run, -L[j]));
-            D_loc = __fadd_rn(__fmul_rn(b, D_loc), dabs[j]);
+            D_loc = fmaf(b, D_loc, dabs[j]);
         }
         incl = lane_affine_scan(D_loc, b_step, lane);
         excl = __shfl_up_sync(kFullWarp, incl, 1);
@@ -216,7 +217,7 @@ ewma_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
 #pragma unroll
         for (int j = 0; j < kEwmaPerLane; ++j) {
             diff[j] = fmaf(la_beta, D_run, q[j]);
-            D_run = __fadd_rn(__fmul_rn(b, D_run), dabs[j]);
+            D_run = fmaf(b, D_run, dabs[j]);
         }
         uint32_t pm[kEwmaHalves][4];
 #pragma unroll

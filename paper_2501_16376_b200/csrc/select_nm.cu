@@ -172,7 +172,7 @@ sp_status launch_select_nm(const sp_ctx *ctx, const void *W, sp_dtype dtype, int
                            int64_t ldw, int N, int M, uint32_t *mask, void *W_out, int64_t ldo,
                            cudaStream_t stream) {
     const int64_t n = ctx->d_in;
-    if (n_rows == 0) return SP_OK;
+    if (n_rows == 0 || (mask == nullptr && W_out == nullptr)) return SP_OK;  // nothing to produce
     const int strips = ctx->strips;
     // Enough warps to fill the GPU a few times over, at least two steps of rows per warp.
     const int64_t target_warps = static_cast<int64_t>(ctx->sm_count) * 64;

@@ -15,7 +15,7 @@
  *     The library owns only the context (O(d_in) device memory).
  *   - Calls enqueue work on the caller's stream (sp_stream = cudaStream_t passed
  *     as void*; NULL = the default stream) and return without synchronising,
- *     except sp_create, sp_destroy, sp_get_stats and sp_set_stats, which say so.
+ *     except sp_create, sp_destroy, sp_get_stats, sp_set_stats and sp_search_la, which say so.
  *   - Arguments are validated on the host before anything is launched; a
  *     non-SP_OK status means nothing was enqueued by that call.  No call
  *     throws, traps or aborts.
@@ -200,6 +200,21 @@ sp_status sp_select_unstructured_ex(sp_ctx *ctx, const void *W, sp_dtype dtype, 
                                     int64_t ldw, const sp_ewma_params *params /* host */,
                                     uint32_t *mask_out, void *W_out, int64_t ldo,
                                     unsigned long long *counters, sp_stream stream);
+
+/*
+ * Searches la for a requested pruning ratio (the paper tunes la per ratio by hand, Table 3, and
+ * names "finding the optimal sparsity" and frequent re-pruning as the use, Sections 1 and 4.2).
+ * With S frozen the pruned fraction is a non-increasing function of la, so the call bisects
+ * la on [-8, 8]: each of the `iterations` (1..64) steps runs Algorithm 1 over W at the midpoint
+ * in count-only mode (W is read, nothing is written) and reads the kept count back, i.e. the
+ * call SYNCHRONISES the stream once per step.  *la_out (host) receives the visited la whose
+ * pruned fraction is closest to target_sparsity, *achieved_out (host, nullable) that fraction.
+ * Follow with sp_select_unstructured_ex(la) to prune.
+ */
+sp_status sp_search_la(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows, int64_t ldw,
+                       float target_sparsity, float alpha, float beta, int iterations,
+                       float *la_out /* host */, double *achieved_out /* host */,
+                       sp_stream stream);
 
 /*
  * Section 3.3: N:M selection fused with the write-back.  Every row is cut into

@@ -248,6 +248,31 @@ def select_unstructured(W_bits, dtype, stats: Stats, sparsity: float, **kw) -> S
     return select_ewma(W_bits, dtype, stats, la_for_sparsity(sparsity), **kw)
 
 
+def search_la(W_bits, dtype, stats: Stats, target_sparsity: float, alpha: float = ALPHA,
+              beta: float = BETA, iterations: int = 24, threads: int = 1):
+    """Bisection of la on [-8, 8] for a requested pruning ratio (the paper sets la per ratio by
+    hand, Table 3): the pruned fraction of Algorithm 1 with S fixed never increases with la.
+    Every step evaluates Algorithm 1 at the midpoint (float32 arithmetic for the midpoint);
+    returns the visited la whose pruned fraction is closest to the target, and that fraction."""
+    lo, hi = np.float32(-8.0), np.float32(8.0)
+    best = (2.0, np.float32(0.0), 0.0)
+    W = _bits2d(W_bits)
+    n = W.shape[1]
+    for _ in range(iterations):
+        la = np.float32(0.5) * (lo + hi)
+        sel = select_ewma(W, dtype, stats, float(la), alpha, beta, s_update=S_FROZEN,
+                          threads=threads)
+        pruned = 1.0 - float(sel.keep_bool(n).mean(dtype=np.float64))
+        gap = abs(pruned - float(np.float32(target_sparsity)))
+        if gap < best[0]:
+            best = (gap, la, pruned)
+        if pruned > float(np.float32(target_sparsity)):
+            lo = la
+        else:
+            hi = la
+    return float(best[1]), best[2]
+
+
 def select_nm(W_bits, dtype, stats: Stats, N: int, M: int, want_trace: bool = False,
               threads: int = 1) -> Selection:
     """Section 3.3: keep N of every M contiguous weights (largest L kept)."""

@@ -27,7 +27,7 @@ SP_COUNTER_KEPT, SP_COUNTER_S_HAZARD, SP_NUM_COUNTERS = 0, 1, 2
 EXPORTS = (
     "sp_create", "sp_destroy", "sp_calib_reset", "sp_calib_accumulate", "sp_get_stats",
     "sp_set_stats", "sp_calib_stats_noalloc", "sp_score", "sp_la_for_sparsity", "sp_select_unstructured",
-    "sp_select_unstructured_ex", "sp_select_nm", "sp_apply_mask", "sp_calib_accumulate_host",
+    "sp_select_unstructured_ex", "sp_search_la", "sp_select_nm", "sp_apply_mask", "sp_calib_accumulate_host",
     "sp_select_nm_host", "sp_select_unstructured_host", "sp_status_string",
     "sp_last_cuda_error", "sp_launch_count",
 )
@@ -64,6 +64,8 @@ def _load() -> ctypes.CDLL:
     lib.sp_select_unstructured_ex.argtypes = [vp, vp, ci, i64, i64, ctypes.POINTER(EwmaParams),
                                               vp, vp, i64, vp, vp]
     lib.sp_select_nm.argtypes = [vp, vp, ci, i64, i64, ci, ci, vp, vp, i64, vp]
+    lib.sp_search_la.argtypes = [vp, vp, ci, i64, i64, f32, f32, f32, ci, ctypes.POINTER(f32),
+                                 ctypes.POINTER(ctypes.c_double), vp]
     lib.sp_apply_mask.argtypes = [vp, ci, i64, i64, i64, vp, vp, i64, vp]
     lib.sp_calib_accumulate_host.argtypes = [vp, vp, ci, i64, i64, vp]
     lib.sp_select_nm_host.argtypes = [vp, vp, ci, i64, i64, ci, ci, vp, vp, i64, vp]
@@ -227,6 +229,18 @@ class Context:
                                               _ptr(mask), optr, ldo, _ptr(counters),
                                               _stream(stream)))
         return mask, W_out
+
+    def sp_search_la(self, W, target_sparsity: float, alpha: float = 0.125, beta: float = 0.125,
+                     iterations: int = 24, stream=None):
+        """Bisects la so that Algorithm 1 prunes target_sparsity of W.  Returns (la, achieved)."""
+        ptr, R, n, ld = _matrix(W, "W")
+        self._check_width(n)
+        la = ctypes.c_float()
+        got = ctypes.c_double()
+        _check(lib.sp_search_la(self._h, ptr, _dtype_of(W), R, ld, float(target_sparsity),
+                                float(alpha), float(beta), int(iterations), ctypes.byref(la),
+                                ctypes.byref(got), _stream(stream)))
+        return la.value, got.value
 
     def sp_select_nm(self, W, N: int, M: int, *, mask=None, W_out=None, inplace=False,
                      want_mask=True, stream=None):

@@ -287,6 +287,58 @@ sp_status sp_select_unstructured(sp_ctx *ctx, const void *W, sp_dtype dtype, int
                                      stream);
 }
 
+sp_status sp_search_la(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows, int64_t ldw,
+                       float target_sparsity, float alpha, float beta, int iterations,
+                       float *la_out, double *achieved_out, sp_stream stream) {
+    sp_status st = check_matrix_args(ctx, W, dtype, n_rows, ldw, nullptr, 0);
+    if (st != SP_OK) return st;
+    if (la_out == nullptr || !(target_sparsity > 0.0f) || !(target_sparsity < 1.0f) ||
+        !(alpha > 0.0f) || !(alpha <= 1.0f) || !(beta > 0.0f) || !(beta <= 1.0f) ||
+        iterations < 1 || iterations > 64 || n_rows < 1)
+        return SP_ERR_INVALID_ARG;
+    if (ctx->n_tokens <= 0) return SP_ERR_STATE;
+    DeviceGuard guard(ctx->device);
+    if (guard.error() != cudaSuccess) return cuda_fail(guard.error());
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    st = ensure_finalized(ctx, s);
+    if (st != SP_OK) return st;
+    // The pruned fraction never increases with la (the threshold est - la*dev only moves down
+    // and, with S frozen, est and dev do not depend on the decisions): bisection on [-8, 8].
+    const double total = static_cast<double>(n_rows) * static_cast<double>(ctx->d_in);
+    float lo = -8.0f, hi = 8.0f, best_la = 0.0f;
+    double best_gap = 2.0, best_frac = 0.0;
+    unsigned long long *counters = ctx->scalars->search_counters;
+    for (int it = 0; it < iterations; ++it) {
+        sp_ewma_params p;
+        p.alpha = alpha;
+        p.beta = beta;
+        p.la = 0.5f * (lo + hi);
+        p.s_update = SP_S_FROZEN;
+        cudaError_t e = cudaMemsetAsync(counters, 0, sizeof(unsigned long long) * SP_NUM_COUNTERS, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+        st = launch_select_ewma(ctx, W, dtype, n_rows, ldw, p, nullptr, nullptr, ldw, counters, s);
+        if (st != SP_OK) return st;
+        unsigned long long host[SP_NUM_COUNTERS];
+        e = cudaMemcpyAsync(host, counters, sizeof host, cudaMemcpyDeviceToHost, s);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+        if (e != cudaSuccess) return cuda_fail(e);
+        const double pruned = 1.0 - static_cast<double>(host[SP_COUNTER_KEPT]) / total;
+        const double gap = std::fabs(pruned - static_cast<double>(target_sparsity));
+        if (gap < best_gap) {
+            best_gap = gap;
+            best_la = p.la;
+            best_frac = pruned;
+        }
+        if (pruned > static_cast<double>(target_sparsity))
+            lo = p.la;  // too much pruned: raise la
+        else
+            hi = p.la;
+    }
+    *la_out = best_la;
+    if (achieved_out != nullptr) *achieved_out = best_frac;
+    return SP_OK;
+}
+
 sp_status sp_select_nm(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows, int64_t ldw,
                        int N, int M, uint32_t *mask_out, void *W_out, int64_t ldo,
                        sp_stream stream) {

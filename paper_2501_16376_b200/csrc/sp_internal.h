@@ -23,6 +23,7 @@ struct DeviceScalars {
     float hazard_w2;      // a weight with w^2 >= this could change S in "S - w^2" (binary32)
     int flags;            // kFlag*
     unsigned int ticket;  // arrival counter of the finalisation kernel (returns to 0)
+    unsigned long long search_counters[SP_NUM_COUNTERS];  // scratch of sp_search_la
 };
 
 // Powers of a = 1-alpha and b = 1-beta that the scan kernel needs (a lane owns P consecutive

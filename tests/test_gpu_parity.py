@@ -443,3 +443,25 @@ def test_host_buffer_calls_match_device_calls(sp, pinned):
         host_ctx.sp_select_nm_host(Wh2, 2, 4, None, Wh2)
         torch.cuda.synchronize()
         assert torch.equal(Wh2.view(torch.int16), dev_ctx.sp_select_nm(W, 2, 4)[1].cpu().view(torch.int16))
+
+
+# ------------------------------------------------------------------ la search
+
+@pytest.mark.parametrize("target", [0.5, 0.35, 0.75])
+def test_la_search_matches_oracle_bisection(sp, target):
+    R, n = 256, 4096
+    W = _gen(91, (R, n), torch.bfloat16, 0.02)
+    X = _activations(92, 2048, n, torch.bfloat16)
+    with _ctx_with_stats(sp, [X], n) as ctx:
+        la, achieved = ctx.sp_search_la(W, target)
+        colsq = ctx.sp_get_stats()[0]
+        st = so.Stats(colsq.numpy().copy(), 1)
+        la_o, achieved_o = so.search_la(P.bits(W), so.BF16, st, target, threads=so.max_threads())
+        # counts may differ by entries inside the threshold band, which can move the bisection
+        # by at most its final resolution
+        assert abs(achieved - achieved_o) <= 2e-6 + 1.0 / (R * n)
+        assert abs(la - la_o) <= 16.0 / 2 ** 20
+        assert abs(achieved - target) < 1e-4
+        mask, _ = ctx.sp_select_unstructured(W, params=sp.EwmaParams(0.125, 0.125, la, 0))
+        keep = so.unpack_mask(P.mask_np(mask), n)
+        assert abs((1.0 - keep.mean()) - achieved) < 1e-12

@@ -468,3 +468,26 @@ def test_apply_mask_bits_and_layout():
     out = so.apply_mask(W, mask)
     assert np.array_equal(out, np.where(keep, W, 0))
     assert np.array_equal(so.unpack_mask(mask, n), keep)
+
+
+# ---------------------------------------------------------------- la search
+
+def test_pruned_fraction_is_monotone_in_la_and_search_hits_the_target():
+    rng = np.random.default_rng(20)
+    n = 2048
+    W = _f16_bits(rng.standard_normal((16, n)) * 0.02)
+    st = _stats_from(rng.uniform(0.9, 1.1, n) * 1e5)
+    fracs = []
+    for la in (-2.0, -1.0, 0.0, 0.5, 1.0, 2.0):
+        sel = so.select_ewma(W, so.F16, st, la, s_update=so.S_FROZEN)
+        fracs.append(1.0 - sel.keep_bool(n).mean())
+    assert fracs == sorted(fracs, reverse=True)
+    # a pruned weight stays pruned when la decreases (thresholds only move up)
+    hi = so.select_ewma(W, so.F16, st, 0.5, s_update=so.S_FROZEN).keep_bool(n)
+    lo = so.select_ewma(W, so.F16, st, -0.5, s_update=so.S_FROZEN).keep_bool(n)
+    assert not (hi < lo).any()
+    for target in (0.3, 0.5, 0.65):
+        la, got = so.search_la(W, so.F16, st, target)
+        assert abs(got - target) < 2e-4          # 32768 weights: resolution 3e-5
+        again = so.select_ewma(W, so.F16, st, la, s_update=so.S_FROZEN)
+        assert 1.0 - again.keep_bool(n).mean() == pytest.approx(got, abs=1e-12)

@@ -37,6 +37,17 @@ SELECT_BYTES_PER_WEIGHT = 4.125
 CALIB_BYTES_PER_ELEMENT = 2.0
 
 
+# DRAM bytes (read + write) per launch from one ncu capture of the timed pass
+# (profiles/dram_traffic_per_launch.md), for the launch shapes of the default configuration
+# (32768-token calibration batches).  Keys: calibration -> d_in; selection -> (rows, d_in).
+# Valid for the kernels as committed with that capture; other shapes report null.
+NCU_CALIB_TRAFFIC = {4096: 269.85e6, 11008: 722.67e6, 14336: 941.03e6}
+NCU_SELECT_TRAFFIC = {
+    "select_nm_kernel": {(4096, 4096): 33.68e6, (11008, 4096): 131.77e6, (4096, 11008): 131.10e6},
+    "ewma_scan_kernel": {(4096, 4096): 84.94e6, (1024, 4096): 8.41e6, (14336, 4096): 185.78e6},
+}
+
+
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -287,21 +298,33 @@ def gpu_arm(args):
     peak, peak_kind = measured_peaks()
     calib_gbs = CALIB_BYTES_PER_ELEMENT * x_elements / (calib_ms * 1e-3) / 1e9
     select_gbs = SELECT_BYTES_PER_WEIGHT * sel_weights / (select_ms * 1e-3) / 1e9
+    calib_traffic = None
+    widths = list(w.input_widths().values())
+    if batch_tokens == 32768 and w.tokens % batch_tokens == 0 and \
+            all(d in NCU_CALIB_TRAFFIC for d in widths):
+        calib_traffic = sum(NCU_CALIB_TRAFFIC[d] for d in widths) / len(widths)
+    sel_kernel = "select_nm_kernel" if w.mode == "nm" else "ewma_scan_kernel"
+    sel_traffic = None
+    shapes = [(l.d_out, l.d_in) for l in w.layers]
+    table = NCU_SELECT_TRAFFIC[sel_kernel]
+    if all(sh in table for sh in shapes) and (w.mode != "nm" or arg == (2, 4)):
+        sel_traffic = sum(table[sh] for sh in shapes) / len(shapes)
     roofline = {
         "kernel": "calib_accumulate_kernel", "bound": "hbm", "achieved": calib_gbs, "peak": peak,
-        "peak_kind": peak_kind, "unit": "GB/s", "frac": calib_gbs / peak, "traffic": None,
+        "peak_kind": peak_kind, "unit": "GB/s", "frac": calib_gbs / peak, "traffic": calib_traffic,
         "avg_launch_ms": calib_ms / calib_launches,
         "bytes_per_launch": CALIB_BYTES_PER_ELEMENT * x_elements / calib_launches,
         "note": "events bracket the back-to-back accumulate launches of one layer input",
     }
     roofline_select = {
-        "kernel": "select_nm_kernel" if w.mode == "nm" else "ewma_scan_kernel",
+        "kernel": sel_kernel,
         "bound": "hbm", "achieved": select_gbs, "peak": peak, "peak_kind": peak_kind,
         "unit": "GB/s", "frac": select_gbs / peak, "frac_of_8TBs": select_gbs / 8000.0,
-        "traffic": None, "avg_launch_ms": select_ms / select_launches,
+        "traffic": sel_traffic, "avg_launch_ms": select_ms / select_launches,
         "bytes_per_launch": SELECT_BYTES_PER_WEIGHT * sel_weights / select_launches,
         "weights_per_sec": sel_weights / (select_ms * 1e-3),
-        "note": "events bracket every selection launch on its own",
+        "note": "events bracket every selection launch on its own; ncu traffic counts DRAM bytes "
+                "while the kernel runs (part of the output is still in L2 when it ends)",
     }
 
     line = {

@@ -44,7 +44,8 @@ CALIB_BYTES_PER_ELEMENT = 2.0
 NCU_CALIB_TRAFFIC = {4096: 269.85e6, 11008: 722.67e6, 14336: 941.03e6}
 NCU_SELECT_TRAFFIC = {
     "select_nm_kernel": {(4096, 4096): 33.68e6, (11008, 4096): 131.77e6, (4096, 11008): 131.10e6},
-    "ewma_scan_kernel": {(4096, 4096): 84.94e6, (1024, 4096): 8.41e6, (14336, 4096): 185.78e6},
+    "ewma_scan_kernel": {(4096, 4096): 34.3e6, (1024, 4096): 8.41e6, (14336, 4096): 185.78e6,
+                         (4096, 14336): 189.5e6},
 }
 
 

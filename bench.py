@@ -63,6 +63,10 @@ def parse_args():
                     help="profiling aid: prune only the first BLOCKS blocks (0 = the whole model)")
     ap.add_argument("--mode-index", type=int, default=0,
                     help="which of the workload's sparsities / N:M patterns to run")
+    ap.add_argument("--graph", action="store_true",
+                    help="replay the whole-model pass as one CUDA graph in the timed region "
+                         "(for launch-bound small models); the per-kernel breakdown then comes "
+                         "from one instrumented pass after it")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
 
@@ -271,18 +275,33 @@ def gpu_arm(args):
     sampler.start()
 
     phase_events = []
+    graph = None
+    if args.graph:
+        graph, counts = pipeline.capture_model_graph(mb, arg, batch_tokens)
+        for _ in range(3):
+            graph.replay()
     launches_before = sp.sp_launch_count()
     start = torch.cuda.Event(enable_timing=True)
     stop = torch.cuda.Event(enable_timing=True)
     barrier()
     start.record()
-    counts = None
-    for _ in range(args.steps):
-        counts = pipeline.prune_model(mb, arg, batch_tokens, phase_events)
+    if graph is not None:
+        for _ in range(args.steps):
+            graph.replay()
+    else:
+        counts = None
+        for _ in range(args.steps):
+            counts = pipeline.prune_model(mb, arg, batch_tokens, phase_events)
     stop.record()
     barrier()
     elapsed_ms = start.elapsed_time(stop)
-    launches = sp.sp_launch_count() - launches_before
+    if graph is not None:
+        launches = sum(counts.values()) * args.steps
+        for _ in range(args.steps):        # instrumented passes, outside the timed region
+            pipeline.prune_model(mb, arg, batch_tokens, phase_events)
+        torch.cuda.synchronize()
+    else:
+        launches = sp.sp_launch_count() - launches_before
     clocks = sampler.stop()
 
     elapsed_ms = sharding.max_over_ranks(elapsed_ms, world, device)
@@ -324,7 +343,7 @@ def gpu_arm(args):
         "traffic": sel_traffic, "avg_launch_ms": select_ms / select_launches,
         "bytes_per_launch": SELECT_BYTES_PER_WEIGHT * sel_weights / select_launches,
         "weights_per_sec": sel_weights / (select_ms * 1e-3),
-        "note": "events bracket every selection launch on its own; ncu traffic counts DRAM bytes "
+        "note": "events bracket the back-to-back selection launches of one layer input; ncu traffic counts DRAM bytes "
                 "while the kernel runs (part of the output is still in L2 when it ends)",
     }
 
@@ -340,6 +359,7 @@ def gpu_arm(args):
                          "%.1f GB stream between reuses)" % (
                              (CALIB_BYTES_PER_ELEMENT * x_elements / args.steps
                               + 4 * w.total_weights()) / 1e9),
+                   "launch": "cuda graph replay" if graph is not None else "stream launches",
                    "parallelism": "independent models per rank" if world > 1 else "single GPU"},
         "whole_model_prune_s": {"calib": calib_ms / args.steps * 1e-3,
                                 "finalize": final_ms / args.steps * 1e-3,

@@ -19,6 +19,8 @@ namespace sp {
 constexpr int kCalibThreads = 256;
 constexpr int kCalibWarps = kCalibThreads / 32;
 constexpr int kRowsInFlight = 8;
+constexpr int kFinalGroups = 4;  // slab groups summed in parallel by the finalisation kernel
+constexpr int kFinalThreads = kFinalGroups * kStripChannels;
 
 template <bool BF16, bool VEC>
 __global__ void __launch_bounds__(kCalibThreads)
@@ -86,43 +88,57 @@ calib_accumulate_kernel(const uint16_t *__restrict__ X, int64_t ldx, int64_t n_t
     }
 }
 
-// Finalisation.  CTA `strip` sums its 256 channels over the valid slab rows (ascending slab
-// order), writes colsq and its strip total; the last CTA to arrive adds the strip totals in
+// Finalisation.  CTA `strip` sums its 256 channels over the valid slab rows (four slab groups
+// in parallel, each in ascending order, then the groups in order), writes colsq and its strip
+// total; the last CTA to arrive adds the strip totals in
 // ascending order to S and writes the per-channel factor for every channel:
 //     u = colsq32 / S32 ;  den = 1 - u ;  c = 0.5 / den          (binary32, round to nearest)
 // No CTA waits for another one (the last arrival does the tail), so the kernel cannot hang.
-__global__ void __launch_bounds__(kStripChannels)
+__global__ void __launch_bounds__(kFinalThreads)
 finalize_kernel(const double *__restrict__ partial, int slabs_valid, int64_t n, int64_t n_pad,
                 int strips, double *__restrict__ colsq, double *__restrict__ strip_sum,
                 float *__restrict__ factor, DeviceScalars *__restrict__ scalars) {
+    __shared__ double part[kFinalGroups][kStripChannels];
     __shared__ double red[kStripChannels];
     __shared__ bool is_last;
     pdl_launch_dependents();
     pdl_wait();  // all partial sums are in place
-    const int t = threadIdx.x;
+    const int t = threadIdx.x & (kStripChannels - 1);  // channel within the strip
+    const int g = threadIdx.x / kStripChannels;        // slab group
     const int64_t ch = static_cast<int64_t>(blockIdx.x) * kStripChannels + t;
+    // Group g adds a contiguous range of slabs in ascending order (eight loads in flight);
+    // the groups are then added in ascending order: a fixed summation order.
+    const int per_group = (slabs_valid + kFinalGroups - 1) / kFinalGroups;
+    const int s_begin = g * per_group;
+    const int s_end = min(slabs_valid, s_begin + per_group);
     double v = 0.0;
     if (ch < n) {
-        // ascending slab order; eight loads in flight at a time
         const double *src = partial + ch;
-        int s = 0;
-        for (; s + 8 <= slabs_valid; s += 8) {
+        int s = s_begin;
+        for (; s + 8 <= s_end; s += 8) {
             double x[8];
 #pragma unroll
             for (int k = 0; k < 8; ++k) x[k] = __ldcg(src + static_cast<int64_t>(s + k) * n_pad);
 #pragma unroll
             for (int k = 0; k < 8; ++k) v += x[k];
         }
-        for (; s < slabs_valid; ++s) v += __ldcg(src + static_cast<int64_t>(s) * n_pad);
+        for (; s < s_end; ++s) v += __ldcg(src + static_cast<int64_t>(s) * n_pad);
     }
-    colsq[ch] = v;  // ch < n_pad always; padding gets 0
-    red[t] = v;
+    part[g][t] = v;
+    __syncthreads();
+    if (g == 0) {
+        v = part[0][t];
+#pragma unroll
+        for (int k = 1; k < kFinalGroups; ++k) v += part[k][t];
+        colsq[ch] = v;  // ch < n_pad always; padding gets 0
+        red[t] = v;
+    }
     __syncthreads();
     for (int half = kStripChannels / 2; half > 0; half >>= 1) {
-        if (t < half) red[t] += red[t + half];
+        if (threadIdx.x < half) red[threadIdx.x] += red[threadIdx.x + half];
         __syncthreads();
     }
-    if (t == 0) {
+    if (threadIdx.x == 0) {
         strip_sum[blockIdx.x] = red[0];
         __threadfence();
         unsigned int ticket = atomicAdd(&scalars->ticket, 1u);
@@ -132,21 +148,21 @@ finalize_kernel(const double *__restrict__ partial, int slabs_valid, int64_t n, 
     if (!is_last) return;
     __threadfence();
 
-    // S: every thread adds the strip totals t, t+256, ... in ascending order, then the same
+    // S: thread i < 256 adds the strip totals i, i+256, ... in ascending order, then the same
     // fixed tree as above combines the 256 partial sums (deterministic, loads in parallel).
-    {
-        double part = 0.0;
-        for (int s = t; s < strips; s += kStripChannels) part += __ldcg(strip_sum + s);
-        red[t] = part;
+    if (threadIdx.x < kStripChannels) {
+        double acc = 0.0;
+        for (int s = threadIdx.x; s < strips; s += kStripChannels) acc += __ldcg(strip_sum + s);
+        red[threadIdx.x] = acc;
     }
     __syncthreads();
     for (int half = kStripChannels / 2; half > 0; half >>= 1) {
-        if (t < half) red[t] += red[t + half];
+        if (threadIdx.x < half) red[threadIdx.x] += red[threadIdx.x + half];
         __syncthreads();
     }
     const double S = red[0];
     const float S32 = static_cast<float>(S);
-    if (t == 0) {
+    if (threadIdx.x == 0) {
         int flags = 0;
         if (!(S > 0.0) || isinf(S) || isnan(S) || isinf(S32)) flags |= kFlagDegenerate;
         // "S - w^2" leaves S unchanged in binary32 whenever w^2 is below a quarter of the
@@ -162,17 +178,17 @@ finalize_kernel(const double *__restrict__ partial, int slabs_valid, int64_t n, 
         scalars->flags = flags;
         scalars->ticket = 0u;
     }
-    // per-channel factors, eight channels per thread in flight
-    for (int64_t q0 = t; q0 < n_pad; q0 += 8 * kStripChannels) {
-        double x[8];
+    // per-channel factors, four channels per thread in flight
+    for (int64_t q0 = threadIdx.x; q0 < n_pad; q0 += 4 * kFinalThreads) {
+        double x[4];
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const int64_t q = q0 + static_cast<int64_t>(k) * kStripChannels;
+        for (int k = 0; k < 4; ++k) {
+            const int64_t q = q0 + static_cast<int64_t>(k) * kFinalThreads;
             x[k] = q < n ? __ldcg(colsq + q) : 0.0;
         }
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const int64_t q = q0 + static_cast<int64_t>(k) * kStripChannels;
+        for (int k = 0; k < 4; ++k) {
+            const int64_t q = q0 + static_cast<int64_t>(k) * kFinalThreads;
             if (q < n_pad) {
                 float c = 0.0f;
                 if (q < n) {
@@ -240,7 +256,7 @@ sp_status launch_calib_accumulate(sp_ctx *ctx, const void *X, sp_dtype dtype, in
 }
 
 sp_status launch_finalize(sp_ctx *ctx, cudaStream_t stream) {
-    PdlConfig pdl(dim3(ctx->strips), dim3(kStripChannels), stream);
+    PdlConfig pdl(dim3(ctx->strips), dim3(kFinalThreads), stream);
     const double *partial = ctx->partial;
     cudaError_t e = cudaLaunchKernelEx(&pdl.cfg, finalize_kernel, partial, ctx->slabs_valid,
                                        ctx->d_in, ctx->n_pad, ctx->strips, ctx->colsq,
@@ -347,7 +363,7 @@ sp_status launch_calib_stats_static(int device, const void *X, sp_dtype dtype, i
 #undef SP_LAUNCH
     status = check_launch();
     if (status != SP_OK) return status;
-    finalize_kernel<<<strips, kStripChannels, 0, stream>>>(
+    finalize_kernel<<<strips, kFinalThreads, 0, stream>>>(
         sc->partial, static_cast<int>(slabs), n, n_pad, strips, sc->colsq, sc->strip_sum,
         sc->factor, &sc->scalars);
     status = check_launch();

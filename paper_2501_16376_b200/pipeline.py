@@ -91,9 +91,10 @@ def prune_model(mb: ModelBuffers, mode_arg, batch_tokens: int, phase_events=None
     """One pass of the whole hot path over the model: for every block and every distinct layer
     input, accumulate the calibration statistics, finalise them, then select + write back every
     layer that reads this input.  phase_events, if given, is a list that receives
-    (kind, start_event, end_event, units) tuples: one "calib" entry per layer input (units =
-    activation elements), one "select" entry per selection launch (units = weights) and one
-    "finalize" entry per layer input.  Returns launch counts."""
+    (kind, start_event, end_event, units) tuples per layer input: "calib" (units = activation
+    elements, brackets its back-to-back accumulate launches), "finalize", and "select" (units =
+    weights, brackets the back-to-back selection launches of the layers reading this input).
+    Returns launch counts."""
     w = mb.workload
     n_calib = n_select = n_final = 0
 
@@ -102,12 +103,12 @@ def prune_model(mb: ModelBuffers, mode_arg, batch_tokens: int, phase_events=None
         e.record(stream)
         return e
 
+    last = mark() if phase_events is not None else None
     for b in range(w.blocks):
         for name, d_in in w.input_widths().items():
             ctx = mb.ctxs[name]
             X = mb.acts[name]
-            if phase_events is not None:
-                e0 = mark()
+            e0 = last
             n_calib += calibrate_input(ctx, X, batch_tokens, stream)
             if phase_events is not None:
                 e1 = mark()
@@ -117,17 +118,30 @@ def prune_model(mb: ModelBuffers, mode_arg, batch_tokens: int, phase_events=None
                 e2 = mark()
                 phase_events.append(("calib", e0, e1, X.shape[0] * d_in))
                 phase_events.append(("finalize", e1, e2, d_in))
+            sel_weights = 0
             for li, layer in enumerate(w.layers):
                 if layer.input != name:
                     continue
-                if phase_events is not None:
-                    s0 = mark()
                 select_layer(ctx, w, mb.weights[b][li], mb.masks[b][li], mb.outputs[b][li],
                              mode_arg, stream)
                 n_select += 1
-                if phase_events is not None:
-                    phase_events.append(("select", s0, mark(), layer.d_out * layer.d_in))
+                sel_weights += layer.d_out * layer.d_in
+            if phase_events is not None:
+                last = mark()
+                phase_events.append(("select", e2, last, sel_weights))
     return {"calib": n_calib, "finalize": n_final, "select": n_select}
+
+
+def capture_model_graph(mb: ModelBuffers, mode_arg, batch_tokens: int):
+    """Captures one whole-model pass into a CUDA graph (for models whose layers are so small
+    that the pass is bound by launch overhead).  The library's calls only enqueue kernels on the
+    current stream, so they can be captured as they are.  Returns (graph, launch counts)."""
+    prune_model(mb, mode_arg, batch_tokens)       # everything allocated and finalised once
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        counts = prune_model(mb, mode_arg, batch_tokens)
+    return graph, counts
 
 
 @dataclass

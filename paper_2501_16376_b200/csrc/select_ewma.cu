@@ -44,6 +44,10 @@ constexpr int kEwmaTile = 32 * kEwmaPerLane;      // weights per warp tile
 #ifndef SP_EWMA_STAGES
 #define SP_EWMA_STAGES 4
 #endif
+#ifndef SP_EWMA_UNROLL
+#define SP_EWMA_UNROLL 1
+#endif
+constexpr int kEwmaUnroll = SP_EWMA_UNROLL;       // tiles per iteration of the tile loop
 constexpr int kEwmaStages = SP_EWMA_STAGES;       // ring slots per warp (a power of two)
 static_assert((kEwmaStages & (kEwmaStages - 1)) == 0, "ring size must be a power of two");
 
@@ -145,6 +149,7 @@ ewma_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
             load8<VEC, true>(wrow, lane * kEwmaPerLane + 8 * h, n, p_next[h]);
     }
 
+#pragma unroll kEwmaUnroll
     for (int tile = 0; tile < tiles; ++tile) {
         const int col = tile * kEwmaTile + lane * kEwmaPerLane;
         uint32_t p[kEwmaHalves][4];

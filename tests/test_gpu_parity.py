@@ -465,3 +465,36 @@ def test_la_search_matches_oracle_bisection(sp, target):
         mask, _ = ctx.sp_select_unstructured(W, params=sp.EwmaParams(0.125, 0.125, la, 0))
         keep = so.unpack_mask(P.mask_np(mask), n)
         assert abs((1.0 - keep.mean()) - achieved) < 1e-12
+
+
+# ------------------------------------------------------------------ CUDA graph capture
+
+def test_whole_pass_can_be_captured_and_replayed_as_a_cuda_graph(sp):
+    from paper_2501_16376_b200 import pipeline, synth
+    w = synth.scaled(synth.WORKLOADS["llama2-7b"], blocks=2, n_seqs=4, seq_len=128, shrink=16)
+    mb = pipeline.allocate_model(w, "cuda")
+    try:
+        batch_tokens = 2 * w.seq_len
+        pipeline.prune_model(mb, (2, 4), batch_tokens)
+        torch.cuda.synchronize()
+        want_masks = [[m.clone() for m in ms] for ms in mb.masks]
+        want_out = [[o.clone() for o in os_] for os_ in mb.outputs]
+        for ms, os_ in zip(mb.masks, mb.outputs):
+            for m, o in zip(ms, os_):
+                m.zero_()
+                o.zero_()
+        graph, counts = pipeline.capture_model_graph(mb, (2, 4), batch_tokens)
+        for ms, os_ in zip(mb.masks, mb.outputs):
+            for m, o in zip(ms, os_):
+                m.zero_()
+                o.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert counts["select"] == 2 * len(w.layers)
+        for b in range(w.blocks):
+            for li in range(len(w.layers)):
+                assert torch.equal(mb.masks[b][li], want_masks[b][li])
+                assert torch.equal(mb.outputs[b][li].view(torch.int16),
+                                   want_out[b][li].view(torch.int16))
+    finally:
+        mb.close()

@@ -229,6 +229,25 @@ sp_status sp_select_nm(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_row
                        sp_stream stream);
 
 /*
+ * Section 3.3, compressed output: 2:4 selection (exactly as sp_select_nm with N = 2, M = 4)
+ * written as the kept values plus per-group indices in the same pass, so that a consumer of
+ * 2:4 sparsity needs no dense pruned matrix and no separate conversion (the paper's remark that
+ * the pattern "eliminates format conversion overhead").  The layout is this library's own:
+ *   values_out  [n_rows, d_in/2] of `dtype`, leading dimension ldv (elements, >= d_in/2): the
+ *               two kept weights of group g of a row at columns 2g, 2g+1, in column order,
+ *               copied bit for bit;
+ *   meta_out    [n_rows, ceil(d_in/32)] uint32, no padding between rows: bits 4g..4g+3 of
+ *               word k describe group 8k+g as  idx0 | idx1 << 2,  idx0 < idx1 being the
+ *               positions (0..3) of the kept weights inside the group; bits past d_in/4 groups
+ *               are 0.
+ * d_in % 4 == 0 (else SP_ERR_SHAPE).  The fast path needs values_out 8-byte aligned and
+ * ldv % 4 == 0 in addition to the usual conditions on W.
+ */
+sp_status sp_select_24_compressed(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
+                                  int64_t ldw, void *values_out, int64_t ldv, uint32_t *meta_out,
+                                  sp_stream stream);
+
+/*
  * Algorithm 1's write-back on its own: W_out = W where the mask bit is 1, +0
  * elsewhere.  W_out may alias W exactly.  Needs no context.
  */

@@ -291,6 +291,39 @@ def select_nm(W_bits, dtype, stats: Stats, N: int, M: int, want_trace: bool = Fa
     return Selection(mask, W_out, L, None)
 
 
+def compress_24(W_bits, keep: np.ndarray):
+    """Compressed form of a 2:4 selection (Section 3.3): for every group of four columns the two
+    kept weights in column order, and a 4-bit record idx0 | idx1 << 2 of their positions in the
+    group; eight records per uint32 word, group 8k+g at bits 4g..4g+3 of word k.
+    Returns (values uint16 [R, n/2], meta uint32 [R, ceil(n/32)])."""
+    W = _bits2d(W_bits)
+    R, n = W.shape
+    keep = np.asarray(keep, dtype=bool)
+    if n % 4 or keep.shape != (R, n) or not (keep.reshape(R, n // 4, 4).sum(-1) == 2).all():
+        raise ValueError("needs exactly two kept weights in every group of four")
+    values = np.zeros((R, n // 2), dtype=np.uint16)
+    meta = np.zeros((R, (n + 31) // 32), dtype=np.uint32)
+    for r in range(R):
+        for g in range(n // 4):
+            idx = [j for j in range(4) if keep[r, 4 * g + j]]
+            values[r, 2 * g] = W[r, 4 * g + idx[0]]
+            values[r, 2 * g + 1] = W[r, 4 * g + idx[1]]
+            meta[r, g // 8] |= np.uint32((idx[0] | (idx[1] << 2)) << (4 * (g % 8)))
+    return values, meta
+
+
+def expand_24(values: np.ndarray, meta: np.ndarray, n: int) -> np.ndarray:
+    """Inverse of compress_24: the dense pruned matrix (uint16 [R, n])."""
+    R = values.shape[0]
+    out = np.zeros((R, n), dtype=np.uint16)
+    for r in range(R):
+        for g in range(n // 4):
+            rec = (int(meta[r, g // 8]) >> (4 * (g % 8))) & 0xF
+            out[r, 4 * g + (rec & 3)] = values[r, 2 * g]
+            out[r, 4 * g + (rec >> 2)] = values[r, 2 * g + 1]
+    return out
+
+
 def apply_mask(W_bits, mask) -> np.ndarray:
     W = _bits2d(W_bits)
     R, n = W.shape

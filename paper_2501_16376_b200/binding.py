@@ -27,7 +27,7 @@ SP_COUNTER_KEPT, SP_COUNTER_S_HAZARD, SP_NUM_COUNTERS = 0, 1, 2
 EXPORTS = (
     "sp_create", "sp_destroy", "sp_calib_reset", "sp_calib_accumulate", "sp_get_stats",
     "sp_set_stats", "sp_calib_stats_noalloc", "sp_score", "sp_la_for_sparsity", "sp_select_unstructured",
-    "sp_select_unstructured_ex", "sp_search_la", "sp_select_nm", "sp_apply_mask", "sp_calib_accumulate_host",
+    "sp_select_unstructured_ex", "sp_search_la", "sp_select_nm", "sp_select_24_compressed", "sp_apply_mask", "sp_calib_accumulate_host",
     "sp_select_nm_host", "sp_select_unstructured_host", "sp_status_string",
     "sp_last_cuda_error", "sp_launch_count",
 )
@@ -64,6 +64,7 @@ def _load() -> ctypes.CDLL:
     lib.sp_select_unstructured_ex.argtypes = [vp, vp, ci, i64, i64, ctypes.POINTER(EwmaParams),
                                               vp, vp, i64, vp, vp]
     lib.sp_select_nm.argtypes = [vp, vp, ci, i64, i64, ci, ci, vp, vp, i64, vp]
+    lib.sp_select_24_compressed.argtypes = [vp, vp, ci, i64, i64, vp, i64, vp, vp]
     lib.sp_search_la.argtypes = [vp, vp, ci, i64, i64, f32, f32, f32, ci, ctypes.POINTER(f32),
                                  ctypes.POINTER(ctypes.c_double), vp]
     lib.sp_apply_mask.argtypes = [vp, ci, i64, i64, i64, vp, vp, i64, vp]
@@ -196,6 +197,20 @@ class Context:
         scores = torch.empty(R, n, dtype=torch.float32, device=W.device)
         _check(lib.sp_score(self._h, ptr, _dtype_of(W), R, ld, scores.data_ptr(), _stream(stream)))
         return scores
+
+    def sp_select_24_compressed(self, W, values=None, meta=None, stream=None):
+        """2:4 selection emitted as kept values [R, d_in/2] + 4-bit-per-group indices
+        [R, ceil(d_in/32)] int32 (layout in the C header).  Returns (values, meta)."""
+        ptr, R, n, ld = _matrix(W, "W")
+        self._check_width(n)
+        if values is None:
+            values = torch.empty(R, n // 2, dtype=W.dtype, device=W.device)
+        if meta is None:
+            meta = torch.zeros(R, (n + 31) // 32, dtype=torch.int32, device=W.device)
+        vptr, _, _, ldv = _matrix(values, "values")
+        _check(lib.sp_select_24_compressed(self._h, ptr, _dtype_of(W), R, ld, vptr, ldv,
+                                           meta.data_ptr(), _stream(stream)))
+        return values, meta
 
     def _check_width(self, n):
         if n != self.d_in:

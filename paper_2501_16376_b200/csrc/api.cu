@@ -356,6 +356,22 @@ sp_status sp_select_nm(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_row
     return launch_select_nm(ctx, W, dtype, n_rows, ldw, N, M, mask_out, W_out, ldo, s);
 }
 
+sp_status sp_select_24_compressed(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
+                                  int64_t ldw, void *values_out, int64_t ldv, uint32_t *meta_out,
+                                  sp_stream stream) {
+    sp_status st = check_matrix_args(ctx, W, dtype, n_rows, ldw, nullptr, 0);
+    if (st != SP_OK) return st;
+    if (n_rows > 0 && (values_out == nullptr || meta_out == nullptr)) return SP_ERR_INVALID_ARG;
+    if (ctx->d_in % 4 != 0 || ldv < ctx->d_in / 2) return SP_ERR_SHAPE;
+    if (ctx->n_tokens <= 0) return SP_ERR_STATE;
+    DeviceGuard guard(ctx->device);
+    if (guard.error() != cudaSuccess) return cuda_fail(guard.error());
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    st = ensure_finalized(ctx, s);
+    if (st != SP_OK) return st;
+    return launch_select_24_compressed(ctx, W, dtype, n_rows, ldw, values_out, ldv, meta_out, s);
+}
+
 sp_status sp_apply_mask(const void *W, sp_dtype dtype, int64_t n_rows, int64_t n_cols, int64_t ldw,
                         const uint32_t *mask, void *W_out, int64_t ldo, sp_stream stream) {
     if (!valid_dtype(dtype)) return SP_ERR_DTYPE;

@@ -93,6 +93,11 @@ sp_status launch_select_nm(const sp_ctx *ctx, const void *W, sp_dtype dtype, int
                            int64_t ldw, int N, int M, uint32_t *mask, void *W_out, int64_t ldo,
                            cudaStream_t stream);
 
+// select_nm_compressed.cu
+sp_status launch_select_24_compressed(const sp_ctx *ctx, const void *W, sp_dtype dtype,
+                                      int64_t n_rows, int64_t ldw, void *values, int64_t ldv,
+                                      uint32_t *meta, cudaStream_t stream);
+
 // select_ewma.cu
 sp_status launch_select_ewma(const sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
                              int64_t ldw, const sp_ewma_params &p, uint32_t *mask, void *W_out,

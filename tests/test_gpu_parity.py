@@ -498,3 +498,22 @@ def test_whole_pass_can_be_captured_and_replayed_as_a_cuda_graph(sp):
                                    want_out[b][li].view(torch.int16))
     finally:
         mb.close()
+
+
+# ------------------------------------------------------------------ compressed 2:4 emission
+
+@pytest.mark.parametrize("R,n,dtype", [(130, 2048, torch.float16), (65, 520, torch.bfloat16),
+                                       (33, 1028, torch.float16), (3, 4, torch.float16)])
+def test_compressed_24_matches_oracle_and_dense_path(sp, R, n, dtype):
+    W = _gen(R * 5 + n, (R, n), dtype, 0.02)
+    X = _activations(n + 7, 512, n, dtype)
+    with _ctx_with_stats(sp, [X], n) as ctx:
+        values, meta = ctx.sp_select_24_compressed(W)
+        mask, dense = ctx.sp_select_nm(W, 2, 4)
+        colsq = ctx.sp_get_stats()[0]
+    sel = so.select_nm(P.bits(W), P.odtype(W), so.Stats(colsq.numpy().copy(), 1), 2, 4)
+    v_want, m_want = so.compress_24(P.bits(W), sel.keep_bool(n))
+    assert np.array_equal(P.bits(values), v_want)
+    assert np.array_equal(P.mask_np(meta), m_want)
+    # and it expands to exactly what the dense call wrote
+    assert np.array_equal(so.expand_24(P.bits(values), P.mask_np(meta), n), P.bits(dense))

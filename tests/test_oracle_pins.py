@@ -491,3 +491,25 @@ def test_pruned_fraction_is_monotone_in_la_and_search_hits_the_target():
         assert abs(got - target) < 2e-4          # 32768 weights: resolution 3e-5
         again = so.select_ewma(W, so.F16, st, la, s_update=so.S_FROZEN)
         assert 1.0 - again.keep_bool(n).mean() == pytest.approx(got, abs=1e-12)
+
+
+# ---------------------------------------------------------------- compressed 2:4 form
+
+def test_compressed_24_hand_example_and_round_trip():
+    # one row, two groups: keep columns (1, 3) of the first and (0, 2) of the second group
+    W = np.array([[10, 11, 12, 13, 20, 21, 22, 23]], dtype=np.uint16)
+    keep = np.array([[0, 1, 0, 1, 1, 0, 1, 0]], dtype=bool)
+    values, meta = so.compress_24(W, keep)
+    assert values.tolist() == [[11, 13, 20, 22]]
+    # records: (1 | 3 << 2) = 0xd for group 0, (0 | 2 << 2) = 0x8 for group 1 -> 0x8d
+    assert meta.tolist() == [[0x8D]]
+    assert np.array_equal(so.expand_24(values, meta, 8), np.where(keep, W, 0))
+    rng = np.random.default_rng(30)
+    n = 72
+    Wr = _f16_bits(rng.standard_normal((5, n)) * 0.02)
+    sel = so.select_nm(Wr, so.F16, _stats_from(rng.uniform(1, 2, n)), 2, 4)
+    v, m = so.compress_24(Wr, sel.keep_bool(n))
+    assert v.shape == (5, 36) and m.shape == (5, 3)
+    assert np.array_equal(so.expand_24(v, m, n), sel.W_out)
+    with pytest.raises(ValueError):
+        so.compress_24(W, np.ones((1, 8), dtype=bool))

@@ -202,6 +202,19 @@ sp_status sp_select_unstructured_ex(sp_ctx *ctx, const void *W, sp_dtype dtype, 
                                     unsigned long long *counters, sp_stream stream);
 
 /*
+ * Diagnostic behind the paper's Fig. 2 (est and dev tracking the mean and the L1 deviation of L
+ * along a row): writes, for every weight of every row, the state Algorithm 1 tests it against -
+ * est_out[r, i] and dev_out[r, i] are est and dev BEFORE the update of element i (so
+ * est_out[r, 0] = L_0, dev_out[r, 0] = 0) - and scores_out[r, i] = L_i; each fp32
+ * [n_rows, d_in], dense, nullable.  Evaluated sequentially along each row in binary32 with one
+ * rounding per operation (one thread per row: meant for a handful of rows, not for speed);
+ * params->s_update selects whether "S = S - w_i^2" is applied to pruned weights.
+ */
+sp_status sp_ewma_trace(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows, int64_t ldw,
+                        const sp_ewma_params *params /* host */, float *est_out, float *dev_out,
+                        float *scores_out, sp_stream stream);
+
+/*
  * Searches la for a requested pruning ratio (the paper tunes la per ratio by hand, Table 3, and
  * names "finding the optimal sparsity" and frequent re-pruning as the use, Sections 1 and 4.2).
  * With S frozen the pruned fraction is a non-increasing function of la, so the call bisects

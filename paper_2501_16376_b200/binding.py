@@ -27,7 +27,7 @@ SP_COUNTER_KEPT, SP_COUNTER_S_HAZARD, SP_NUM_COUNTERS = 0, 1, 2
 EXPORTS = (
     "sp_create", "sp_destroy", "sp_calib_reset", "sp_calib_accumulate", "sp_get_stats",
     "sp_set_stats", "sp_calib_stats_noalloc", "sp_score", "sp_la_for_sparsity", "sp_select_unstructured",
-    "sp_select_unstructured_ex", "sp_search_la", "sp_select_nm", "sp_select_24_compressed", "sp_apply_mask", "sp_calib_accumulate_host",
+    "sp_select_unstructured_ex", "sp_search_la", "sp_ewma_trace", "sp_select_nm", "sp_select_24_compressed", "sp_apply_mask", "sp_calib_accumulate_host",
     "sp_select_nm_host", "sp_select_unstructured_host", "sp_status_string",
     "sp_last_cuda_error", "sp_launch_count",
 )
@@ -65,6 +65,7 @@ def _load() -> ctypes.CDLL:
                                               vp, vp, i64, vp, vp]
     lib.sp_select_nm.argtypes = [vp, vp, ci, i64, i64, ci, ci, vp, vp, i64, vp]
     lib.sp_select_24_compressed.argtypes = [vp, vp, ci, i64, i64, vp, i64, vp, vp]
+    lib.sp_ewma_trace.argtypes = [vp, vp, ci, i64, i64, ctypes.POINTER(EwmaParams), vp, vp, vp, vp]
     lib.sp_search_la.argtypes = [vp, vp, ci, i64, i64, f32, f32, f32, ci, ctypes.POINTER(f32),
                                  ctypes.POINTER(ctypes.c_double), vp]
     lib.sp_apply_mask.argtypes = [vp, ci, i64, i64, i64, vp, vp, i64, vp]
@@ -244,6 +245,16 @@ class Context:
                                               _ptr(mask), optr, ldo, _ptr(counters),
                                               _stream(stream)))
         return mask, W_out
+
+    def sp_ewma_trace(self, W, params: EwmaParams, stream=None):
+        """est, dev (state before each element's update) and L along every row: three fp32
+        tensors [R, d_in].  Sequential diagnostic, meant for a few rows."""
+        ptr, R, n, ld = _matrix(W, "W")
+        self._check_width(n)
+        est, dev, L = (torch.empty(R, n, dtype=torch.float32, device=W.device) for _ in range(3))
+        _check(lib.sp_ewma_trace(self._h, ptr, _dtype_of(W), R, ld, ctypes.byref(params),
+                                 est.data_ptr(), dev.data_ptr(), L.data_ptr(), _stream(stream)))
+        return est, dev, L
 
     def sp_search_la(self, W, target_sparsity: float, alpha: float = 0.125, beta: float = 0.125,
                      iterations: int = 24, stream=None):

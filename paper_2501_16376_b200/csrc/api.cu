@@ -287,6 +287,25 @@ sp_status sp_select_unstructured(sp_ctx *ctx, const void *W, sp_dtype dtype, int
                                      stream);
 }
 
+sp_status sp_ewma_trace(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows, int64_t ldw,
+                        const sp_ewma_params *params, float *est_out, float *dev_out,
+                        float *scores_out, sp_stream stream) {
+    sp_status st = check_matrix_args(ctx, W, dtype, n_rows, ldw, nullptr, 0);
+    if (st != SP_OK) return st;
+    if (params == nullptr || !(params->alpha > 0.0f) || !(params->alpha <= 1.0f) ||
+        !(params->beta > 0.0f) || !(params->beta <= 1.0f) || !std::isfinite(params->la))
+        return SP_ERR_INVALID_ARG;
+    if (params->s_update != SP_S_FROZEN && params->s_update != SP_S_LITERAL_W2)
+        return SP_ERR_INVALID_ARG;
+    if (ctx->n_tokens <= 0) return SP_ERR_STATE;
+    DeviceGuard guard(ctx->device);
+    if (guard.error() != cudaSuccess) return cuda_fail(guard.error());
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    st = ensure_finalized(ctx, s);
+    if (st != SP_OK) return st;
+    return launch_ewma_trace(ctx, W, dtype, n_rows, ldw, *params, est_out, dev_out, scores_out, s);
+}
+
 sp_status sp_search_la(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows, int64_t ldw,
                        float target_sparsity, float alpha, float beta, int iterations,
                        float *la_out, double *achieved_out, sp_stream stream) {

@@ -326,6 +326,62 @@ ewma_literal_kernel(const uint16_t *__restrict__ W, int64_t ldw, int64_t n_rows,
     if (counters != nullptr) atomicAdd(counters + SP_COUNTER_KEPT, kept);
 }
 
+// Diagnostic: the state Algorithm 1 tests every weight against (est and dev before the update
+// of element i) and the score L_i, written out along each row; one thread per row, sequential,
+// binary32 with one rounding per operation like the literal kernel (S updated when s_update
+// says so).  This is the data behind the paper's Fig. 2 (est / dev tracking the mean and the
+// L1 deviation of L along a row).
+template <bool BF16>
+__global__ void __launch_bounds__(128)
+ewma_trace_kernel(const uint16_t *__restrict__ W, int64_t ldw, int64_t n_rows, int64_t n,
+                  const double *__restrict__ colsq, const DeviceScalars *__restrict__ scalars,
+                  float alpha, float beta, float la, int literal_s, float *__restrict__ est_out,
+                  float *__restrict__ dev_out, float *__restrict__ score_out) {
+    const int64_t row = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (row >= n_rows) return;
+    const uint16_t *wrow = W + row * ldw;
+    const float one_minus_alpha = __fsub_rn(1.0f, alpha);
+    const float one_minus_beta = __fsub_rn(1.0f, beta);
+    float S = scalars->S32;
+    float est = 0.0f, dev = 0.0f;
+    for (int64_t i = 0; i < n; ++i) {
+        const uint16_t bits = wrow[i];
+        const float w = BF16 ? __uint_as_float(static_cast<uint32_t>(bits) << 16)
+                             : __half2float(__ushort_as_half(bits));
+        const float u = __fdiv_rn(static_cast<float>(colsq[i]), S);
+        const float c = __fdiv_rn(0.5f, __fsub_rn(1.0f, u));
+        const float w2 = __fmul_rn(w, w);
+        const float L = __fmul_rn(w2, c);
+        if (i == 0) est = L;
+        if (est_out != nullptr) est_out[row * n + i] = est;
+        if (dev_out != nullptr) dev_out[row * n + i] = dev;
+        if (score_out != nullptr) score_out[row * n + i] = L;
+        const float thr = __fsub_rn(est, __fmul_rn(la, dev));
+        if (L < thr && literal_s) S = __fsub_rn(S, w2);
+        est = __fadd_rn(__fmul_rn(one_minus_alpha, est), __fmul_rn(alpha, L));
+        dev = __fadd_rn(__fmul_rn(one_minus_beta, dev), __fmul_rn(beta, fabsf(__fsub_rn(est, L))));
+    }
+}
+
+sp_status launch_ewma_trace(const sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
+                            int64_t ldw, const sp_ewma_params &p, float *est_out, float *dev_out,
+                            float *score_out, cudaStream_t stream) {
+    if (n_rows == 0) return SP_OK;
+    const int64_t blocks = (n_rows + 127) / 128;
+    if (blocks > 0x7fffffffLL) return SP_ERR_SHAPE;
+    const uint16_t *Wp = static_cast<const uint16_t *>(W);
+    const int literal = p.s_update == SP_S_LITERAL_W2 ? 1 : 0;
+    if (dtype == SP_BF16)
+        ewma_trace_kernel<true><<<static_cast<unsigned>(blocks), 128, 0, stream>>>(
+            Wp, ldw, n_rows, ctx->d_in, ctx->colsq, ctx->scalars, p.alpha, p.beta, p.la, literal,
+            est_out, dev_out, score_out);
+    else
+        ewma_trace_kernel<false><<<static_cast<unsigned>(blocks), 128, 0, stream>>>(
+            Wp, ldw, n_rows, ctx->d_in, ctx->colsq, ctx->scalars, p.alpha, p.beta, p.la, literal,
+            est_out, dev_out, score_out);
+    return check_launch();
+}
+
 static void fill_scan_constants(const sp_ewma_params &p, ScanConstants &sc) {
     sc.alpha = p.alpha;
     sc.beta = p.beta;

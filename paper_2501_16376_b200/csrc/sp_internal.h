@@ -129,6 +129,10 @@ struct PdlConfig {
     }
 };
 
+sp_status launch_ewma_trace(const sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
+                            int64_t ldw, const sp_ewma_params &p, float *est_out, float *dev_out,
+                            float *score_out, cudaStream_t stream);
+
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace sp

@@ -517,3 +517,28 @@ def test_compressed_24_matches_oracle_and_dense_path(sp, R, n, dtype):
     assert np.array_equal(P.mask_np(meta), m_want)
     # and it expands to exactly what the dense call wrote
     assert np.array_equal(so.expand_24(P.bits(values), P.mask_np(meta), n), P.bits(dense))
+
+
+# ------------------------------------------------------------------ EWMA trace diagnostic
+
+@pytest.mark.parametrize("s_update", [0, 1])
+def test_ewma_trace_matches_oracle_state(sp, s_update):
+    R, n = 6, 1500
+    W = _gen(71, (R, n), torch.float16, 0.02)
+    colsq = np.random.default_rng(5).uniform(1.0, 2.0, n) * (1e-4 if s_update else 1e4)
+    with sp.Context(n) as ctx:
+        ctx.sp_set_stats(torch.from_numpy(colsq), 10)
+        est, dev, L = ctx.sp_ewma_trace(W, sp.EwmaParams(0.125, 0.125, 0.5, s_update))
+    st = so.Stats(colsq.copy(), 10)
+    # the oracle's recorded threshold est - la*dev gives est (la = 0) and est - dev (la = 1);
+    # with the S update on, decisions (hence S) depend on la, so compare at the la used
+    ref = so.select_ewma(P.bits(W), so.F16, st, 0.5, s_update=s_update, want_trace=True)
+    thr = est.cpu().numpy() - np.float32(0.5) * dev.cpu().numpy()
+    assert np.array_equal(L.cpu().numpy(), ref.L)
+    assert np.array_equal(thr.astype(np.float32), ref.thr)
+    if not s_update:
+        e0 = so.select_ewma(P.bits(W), so.F16, st, 0.0, s_update=0, want_trace=True).thr
+        e1 = so.select_ewma(P.bits(W), so.F16, st, 1.0, s_update=0, want_trace=True).thr
+        assert np.array_equal(est.cpu().numpy(), e0)
+        assert np.array_equal((est.cpu().numpy() - dev.cpu().numpy()).astype(np.float32), e1)
+    assert (dev[:, 0] == 0).all() and torch.equal(est[:, 0], L[:, 0])

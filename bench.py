@@ -38,7 +38,7 @@ CALIB_BYTES_PER_ELEMENT = 2.0
 
 
 # DRAM bytes (read + write) per launch from one ncu capture of the timed pass
-# (profiles/dram_traffic_per_launch.md), for the launch shapes of the default configuration
+# (summarised under profiles/), for the launch shapes of the default configuration
 # (32768-token calibration batches).  Keys: calibration -> d_in; selection -> (rows, d_in).
 # Valid for the kernels as committed with that capture; other shapes report null.
 NCU_CALIB_TRAFFIC = {4096: 269.85e6, 11008: 722.67e6, 14336: 941.03e6}

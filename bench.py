@@ -398,6 +398,9 @@ def gpu_arm(args):
         cb = oracle_sample(w, so.max_threads())
         line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
         line["cpu_baseline"]["whole_model_seconds"] = cb["whole_model_seconds"]
+        one = oracle_sample(w, 1)                  # the same sample on a single thread
+        line["cpu_baseline"]["single_thread_value"] = one["value"]
+        line["cpu_baseline"]["single_thread_whole_model_seconds"] = one["whole_model_seconds"]
 
     mb.close()
     if world > 1:

@@ -280,46 +280,78 @@ ewma_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
 }
 
 // Algorithm 1 exactly as printed, one thread per row, binary32 with one rounding per operation.
-template <bool BF16>
+// The row is read and written in chunks of 8 weights (16 bytes when aligned).  While S still
+// has its initial value the per-channel factor computed at finalisation is used: it was formed
+// by the same three operations from the same S, so the result is bit-identical to recomputing
+// it; once a pruned weight has changed S the factor is recomputed for every element.
+template <bool BF16, bool VEC>
 __global__ void __launch_bounds__(128)
 ewma_literal_kernel(const uint16_t *__restrict__ W, int64_t ldw, int64_t n_rows, int64_t n,
-                    const double *__restrict__ colsq, const DeviceScalars *__restrict__ scalars,
-                    float alpha, float beta, float la, uint32_t *__restrict__ mask,
-                    int64_t mask_words, uint16_t *__restrict__ W_out, int64_t ldo,
+                    const double *__restrict__ colsq, const float *__restrict__ factor,
+                    const DeviceScalars *__restrict__ scalars, float alpha, float beta, float la,
+                    uint32_t *__restrict__ mask, int64_t mask_words,
+                    uint16_t *__restrict__ W_out, int64_t ldo,
                     unsigned long long *__restrict__ counters) {
     const int64_t row = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (row >= n_rows) return;
     const uint16_t *wrow = W + row * ldw;
+    uint16_t *orow = W_out != nullptr ? W_out + row * ldo : nullptr;
+    uint32_t *mrow = mask != nullptr ? mask + row * mask_words : nullptr;
     const float one_minus_alpha = __fsub_rn(1.0f, alpha);
     const float one_minus_beta = __fsub_rn(1.0f, beta);
-    float S = scalars->S32;
+    const float S0 = scalars->S32;
+    float S = S0;
     float est = 0.0f, dev = 0.0f;
     uint32_t word = 0;
     unsigned long long kept = 0;
-    for (int64_t i = 0; i < n; ++i) {
-        uint16_t bits = wrow[i];
-        const float w = BF16 ? __uint_as_float(static_cast<uint32_t>(bits) << 16)
-                             : __half2float(__ushort_as_half(bits));
-        const float x2 = static_cast<float>(colsq[i]);
-        const float u = __fdiv_rn(x2, S);
-        const float den = __fsub_rn(1.0f, u);
-        const float c = __fdiv_rn(0.5f, den);
-        const float w2 = __fmul_rn(w, w);
-        const float L = __fmul_rn(w2, c);
-        if (i == 0) est = L;
-        const float thr = __fsub_rn(est, __fmul_rn(la, dev));
-        if (L < thr) {
-            S = __fsub_rn(S, w2);
-            bits = 0;
-        } else {
-            word |= 1u << (i & 31);
-            ++kept;
+    // two chunks are kept in flight ahead of the one being evaluated
+    uint32_t ahead[2][4];
+    load8<VEC, true>(wrow, 0, n, ahead[0]);
+    load8<VEC, true>(wrow, 8, n, ahead[1]);
+    for (int64_t i0 = 0; i0 < n; i0 += 8) {
+        uint32_t p[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            p[k] = ahead[0][k];
+            ahead[0][k] = ahead[1][k];
         }
-        est = __fadd_rn(__fmul_rn(one_minus_alpha, est), __fmul_rn(alpha, L));
-        dev = __fadd_rn(__fmul_rn(one_minus_beta, dev), __fmul_rn(beta, fabsf(__fsub_rn(est, L))));
-        if (W_out != nullptr) W_out[row * ldo + i] = bits;
-        if ((i & 31) == 31 || i == n - 1) {
-            if (mask != nullptr) mask[row * mask_words + (i >> 5)] = word;
+        load8<VEC, true>(wrow, i0 + 16, n, ahead[1]);
+        float w[8];
+        unpack8<BF16>(p, w);
+        uint32_t keep8 = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int64_t i = i0 + j;
+            if (i < n) {
+                float c;
+                if (S == S0) {
+                    c = __ldg(factor + i);
+                } else {
+                    const float u = __fdiv_rn(static_cast<float>(colsq[i]), S);
+                    c = __fdiv_rn(0.5f, __fsub_rn(1.0f, u));
+                }
+                const float w2 = __fmul_rn(w[j], w[j]);
+                const float L = __fmul_rn(w2, c);
+                if (i == 0) est = L;
+                const float thr = __fsub_rn(est, __fmul_rn(la, dev));
+                if (L < thr) {
+                    S = __fsub_rn(S, w2);
+                } else {
+                    keep8 |= 1u << j;
+                }
+                est = __fadd_rn(__fmul_rn(one_minus_alpha, est), __fmul_rn(alpha, L));
+                dev = __fadd_rn(__fmul_rn(one_minus_beta, dev),
+                                __fmul_rn(beta, fabsf(__fsub_rn(est, L))));
+            }
+        }
+        kept += __popc(keep8);
+        if (orow != nullptr) {
+            zero_pruned(p, keep8);
+            store8<VEC>(orow, i0, n, p);
+        }
+        word |= keep8 << (i0 & 31);
+        if ((i0 & 31) == 24 || i0 + 8 >= n) {
+            if (mrow != nullptr) mrow[i0 >> 5] = word;
             word = 0;
         }
     }
@@ -413,14 +445,19 @@ sp_status launch_select_ewma(const sp_ctx *ctx, const void *W, sp_dtype dtype, i
     if (p.s_update == SP_S_LITERAL_W2) {
         const int64_t blocks = (n_rows + 127) / 128;
         if (blocks > 0x7fffffffLL) return SP_ERR_SHAPE;
-        if (bf16)
-            ewma_literal_kernel<true><<<static_cast<unsigned>(blocks), 128, 0, stream>>>(
-                Wp, ldw, n_rows, n, ctx->colsq, ctx->scalars, p.alpha, p.beta, p.la, mask, words,
-                Op, ldo, counters);
-        else
-            ewma_literal_kernel<false><<<static_cast<unsigned>(blocks), 128, 0, stream>>>(
-                Wp, ldw, n_rows, n, ctx->colsq, ctx->scalars, p.alpha, p.beta, p.la, mask, words,
-                Op, ldo, counters);
+        const bool lvec = aligned16(W) && ldw % 8 == 0 && n % 8 == 0 &&
+                          (W_out == nullptr || (aligned16(W_out) && ldo % 8 == 0));
+        const unsigned lgrid = static_cast<unsigned>(blocks);
+#define SP_LAUNCH_L(B, V)                                                                    \
+    ewma_literal_kernel<B, V><<<lgrid, 128, 0, stream>>>(                                    \
+        Wp, ldw, n_rows, n, ctx->colsq, ctx->factor, ctx->scalars, p.alpha, p.beta, p.la, mask, \
+        words, Op, ldo, counters)
+        if (bf16) {
+            if (lvec) SP_LAUNCH_L(true, true); else SP_LAUNCH_L(true, false);
+        } else {
+            if (lvec) SP_LAUNCH_L(false, true); else SP_LAUNCH_L(false, false);
+        }
+#undef SP_LAUNCH_L
         return check_launch();
     }
 

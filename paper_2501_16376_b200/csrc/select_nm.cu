@@ -45,14 +45,18 @@ __device__ __forceinline__ uint32_t nm_process_row(uint32_t (&p)[4], const float
     uint32_t key[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) key[j] = __float_as_uint(__fmul_rn(__fmul_rn(w[j], w[j]), c[j]));
-    uint32_t ra, rb;
-    nm_rank_bytes<M>(key, bias_lo, bias_hi, ra, rb);
-    // half-word masks from the top bit of each rank byte (sign replication)
+    // half-word masks from the top bit of each rank field (sign replication)
     uint32_t m[4];
-    m[0] = prmt(ra, 0u, 0x9988u);
-    m[1] = prmt(ra, 0u, 0xbbaau);
-    m[2] = prmt(rb, 0u, 0x9988u);
-    m[3] = prmt(rb, 0u, 0xbbaau);
+    if constexpr (M == 4) {
+        uint32_t ra, rb;
+        nm_rank_bytes<4>(key, bias_lo, bias_hi, ra, rb);
+        m[0] = prmt(ra, 0u, 0x9988u);
+        m[1] = prmt(ra, 0u, 0xbbaau);
+        m[2] = prmt(rb, 0u, 0x9988u);
+        m[3] = prmt(rb, 0u, 0xbbaau);
+    } else {
+        masks_from_nibbles(nm_rank_nibbles8(key, bias_lo), m);  // bias_lo holds the nibble bias
+    }
     if (out_row != nullptr) {
 #pragma unroll
         for (int k = 0; k < 4; ++k) p[k] &= m[k];
@@ -81,9 +85,11 @@ select_nm_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int64_t n,
     load_factor8(factor, col, c);  // zero past d_in
     const int64_t left = n - col;
     const uint32_t valid = left >= 8 ? 0xffu : (left > 0 ? (1u << left) - 1u : 0u);
-    const uint32_t bias = static_cast<uint32_t>(0x80 - prune_count) * 0x01010101u;
-    const uint32_t bias_lo = bias + 0x03020100u;
-    const uint32_t bias_hi = bias + (M == 4 ? 0x03020100u : 0x07060504u);
+    // M == 4: rank bytes in two registers; M == 8: rank nibbles in one (see nm_rank.cuh)
+    const uint32_t bias_lo =
+        M == 4 ? static_cast<uint32_t>(0x80 - prune_count) * 0x01010101u + 0x03020100u
+               : static_cast<uint32_t>(8 - prune_count) * 0x11111111u + 0x76543210u;
+    const uint32_t bias_hi = bias_lo;
     const bool store_word = mask != nullptr && (lane & 3) == 0 && left > 0;
 
     // Row pointers advance by whole rows; row index times leading dimension is a 32x32->64

@@ -5,7 +5,8 @@
 // per row), i.e. two groups of four or one group of eight: a group never straddles lanes, so
 // the selection needs no cross-lane traffic.  The 8 per-channel factors c_q of the lane's
 // columns are loaded once and stay in registers for the whole slab, and several rows are kept
-// in flight per lane.
+// in flight per lane: on the aligned path through a small per-lane ring in shared memory filled
+// by asynchronous copies (a lane only reads what it copied itself), otherwise in registers.
 //
 // Selection.  Scores are L = (w*w)*c_q in binary32 (Eq. 8); they are non-negative, so they are
 // compared through their bit patterns as unsigned integers, which also ranks NaN above every
@@ -26,6 +27,9 @@ namespace sp {
 #endif
 #ifndef SP_NM_MIN_BLOCKS
 #define SP_NM_MIN_BLOCKS 8
+#endif
+#ifndef SP_NM_RING
+#define SP_NM_RING 4  // ring stages of the aligned path (0 = rows prefetched in registers)
 #endif
 #ifndef SP_NM_THREADS
 #define SP_NM_THREADS 128
@@ -99,6 +103,36 @@ select_nm_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int64_t n,
     uint32_t *mp = mask != nullptr ? mask + static_cast<int64_t>(row_begin) * mask_words + (col >> 5)
                                    : nullptr;
 
+#if SP_NM_RING
+    if constexpr (VEC) {
+        // rows streamed through a per-lane shared-memory ring with asynchronous copies
+        constexpr int kStages = SP_NM_RING;  // a power of two
+        __shared__ __align__(16) uint4 ring[kNmWarps * kStages * 32];
+        uint4 *my_ring = ring + (threadIdx.x >> 5) * kStages * 32 + lane;
+        const uint16_t *src = wp + (left > 0 ? col : 0);
+        auto issue = [&](int rr) {
+            if (rr < rows)
+                cp_async16(my_ring + (rr & (kStages - 1)) * 32, src + static_cast<int64_t>(rr) * ldw,
+                           left > 0 ? 16 : 0);
+            cp_async_commit();
+        };
+#pragma unroll
+        for (int rr = 0; rr < kStages - 1; ++rr) issue(rr);
+        for (int rr = 0; rr < rows; ++rr) {
+            issue(rr + kStages - 1);
+            cp_async_wait<kStages - 1>();
+            const uint4 v = my_ring[(rr & (kStages - 1)) * 32];
+            uint32_t p[4] = {v.x, v.y, v.z, v.w};
+            const uint32_t keep8 =
+                nm_process_row<BF16, VEC, M>(p, c, bias_lo, bias_hi, valid, op, col, n);
+            const uint32_t word = gather_mask_word(keep8, lane);
+            if (store_word) *mp = word;
+            if (op != nullptr) op += ldo;
+            if (mp != nullptr) mp += mask_words;
+        }
+        return;
+    }
+#endif
     int r = 0;
     for (; r + kNmRowsInFlight <= rows; r += kNmRowsInFlight) {
         uint32_t p[kNmRowsInFlight][4];

@@ -31,12 +31,16 @@ namespace sp {
 #ifndef SP_NM_RING
 #define SP_NM_RING 4  // ring stages of the aligned path (0 = rows prefetched in registers)
 #endif
+#ifndef SP_NM_RING_UNROLL
+#define SP_NM_RING_UNROLL 4
+#endif
 #ifndef SP_NM_THREADS
 #define SP_NM_THREADS 128
 #endif
 constexpr int kNmThreads = SP_NM_THREADS;
 constexpr int kNmWarps = kNmThreads / 32;
 constexpr int kNmRowsInFlight = SP_NM_ROWS_IN_FLIGHT;
+constexpr int kNmRingUnroll = SP_NM_RING_UNROLL;
 
 // One row of one lane: score, rank, masks, write-back.  Returns the 8 keep bits.
 template <bool BF16, bool VEC, int M>
@@ -118,6 +122,7 @@ select_nm_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int64_t n,
         };
 #pragma unroll
         for (int rr = 0; rr < kStages - 1; ++rr) issue(rr);
+#pragma unroll kNmRingUnroll
         for (int rr = 0; rr < rows; ++rr) {
             issue(rr + kStages - 1);
             cp_async_wait<kStages - 1>();

@@ -97,12 +97,13 @@ sp_status sp_create(sp_ctx **out, int64_t d_in, int device) {
     ctx->calib_blocks_per_sm = calib_query_blocks_per_sm();
 
     const size_t np = static_cast<size_t>(ctx->n_pad);
-    void *ptrs[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
-    const size_t sizes[5] = {sizeof(double) * np * kMaxSlabs, sizeof(double) * np,
+    void *ptrs[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+    const size_t sizes[6] = {sizeof(double) * np * kMaxSlabs, sizeof(double) * np,
                              sizeof(double) * static_cast<size_t>(ctx->strips),
                              sizeof(float) * (np + kStripChannels),
-                             sizeof(DeviceScalars)};
-    for (int i = 0; i < 5; ++i) {
+                             sizeof(DeviceScalars),
+                             sizeof(float) * (np + kStripChannels)};
+    for (int i = 0; i < 6; ++i) {
         e = cudaMalloc(&ptrs[i], sizes[i]);
         if (e == cudaSuccess) e = cudaMemset(ptrs[i], 0, sizes[i]);
         if (e != cudaSuccess) {
@@ -116,6 +117,7 @@ sp_status sp_create(sp_ctx **out, int64_t d_in, int device) {
     ctx->strip_sum = static_cast<double *>(ptrs[2]);
     ctx->factor = static_cast<float *>(ptrs[3]);
     ctx->scalars = static_cast<DeviceScalars *>(ptrs[4]);
+    ctx->factor_pairs = static_cast<float *>(ptrs[5]);
     e = cudaDeviceSynchronize();
     if (e != cudaSuccess) { sp_destroy(ctx); return cuda_fail(e); }
     *out = ctx;
@@ -131,6 +133,7 @@ sp_status sp_destroy(sp_ctx *ctx) {
     cudaFree(ctx->colsq);
     cudaFree(ctx->strip_sum);
     cudaFree(ctx->factor);
+    cudaFree(ctx->factor_pairs);
     cudaFree(ctx->scalars);
     delete ctx;
     return SP_OK;

@@ -97,7 +97,8 @@ calib_accumulate_kernel(const uint16_t *__restrict__ X, int64_t ldx, int64_t n_t
 __global__ void __launch_bounds__(kFinalThreads)
 finalize_kernel(const double *__restrict__ partial, int slabs_valid, int64_t n, int64_t n_pad,
                 int strips, double *__restrict__ colsq, double *__restrict__ strip_sum,
-                float *__restrict__ factor, DeviceScalars *__restrict__ scalars) {
+                float *__restrict__ factor, float *__restrict__ factor_pairs,
+                DeviceScalars *__restrict__ scalars) {
     __shared__ double part[kFinalGroups][kStripChannels];
     __shared__ double red[kStripChannels];
     __shared__ bool is_last;
@@ -197,6 +198,11 @@ finalize_kernel(const double *__restrict__ partial, int slabs_valid, int64_t n, 
                     c = __fdiv_rn(0.5f, den);
                 }
                 factor[q] = c;
+                // second copy for kernels that pair column j with column j+4 of a chunk of 8
+                if (factor_pairs != nullptr) {
+                    const int64_t e = q & 7;
+                    factor_pairs[(q & ~int64_t(7)) | (e < 4 ? 2 * e : 2 * (e - 4) + 1)] = c;
+                }
             }
         }
     }
@@ -260,7 +266,8 @@ sp_status launch_finalize(sp_ctx *ctx, cudaStream_t stream) {
     const double *partial = ctx->partial;
     cudaError_t e = cudaLaunchKernelEx(&pdl.cfg, finalize_kernel, partial, ctx->slabs_valid,
                                        ctx->d_in, ctx->n_pad, ctx->strips, ctx->colsq,
-                                       ctx->strip_sum, ctx->factor, ctx->scalars);
+                                       ctx->strip_sum, ctx->factor, ctx->factor_pairs,
+                                       ctx->scalars);
     if (e != cudaSuccess) return cuda_fail(e);
     sp_status st = check_launch();
     if (st == SP_OK) ctx->dirty = false;
@@ -365,7 +372,7 @@ sp_status launch_calib_stats_static(int device, const void *X, sp_dtype dtype, i
     if (status != SP_OK) return status;
     finalize_kernel<<<strips, kFinalThreads, 0, stream>>>(
         sc->partial, static_cast<int>(slabs), n, n_pad, strips, sc->colsq, sc->strip_sum,
-        sc->factor, &sc->scalars);
+        sc->factor, /*factor_pairs=*/nullptr, &sc->scalars);
     status = check_launch();
     if (status != SP_OK) return status;
 

@@ -279,6 +279,261 @@ ewma_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
     }
 }
 
+// Paired-chain variant of the scan kernel for rows that allow 16-byte access.
+//
+// Same decomposition (warp per row, 8 consecutive weights per lane, two lane scans per tile),
+// but the lane's 8 elements are treated as two chains of 4 (elements 0-3 and 4-7) that advance
+// together in the two halves of packed binary32 pairs (fma.rn.f32x2: one issue slot for two
+// fused multiply-adds).  The second chain starts from the state the first one ends in, which is
+// known as soon as the first chain's zero-state total is: E(4) = a^4 E(0) + T_lo.
+//
+// Algebra used (scaled states E = est/alpha, D' = dev/(beta a)):
+//     q_i  = L_i - alpha E_{i-1}                  (score minus the estimate it is tested against)
+//     E_i  = a E_{i-1} + L_i
+//     est_i - L_i = -a q_i   =>   D'_i = b D'_{i-1} + |q_i|
+//     prune  <=>  q_i + kappa D'_{i-1} < 0 ,  kappa = la beta a .
+// D' is a linear recurrence, so the state before element j of a chain entered with D'_in is
+// Dloc_{j-1} + b^j D'_in (Dloc: the chain run from a zero state); the decision value is
+// (q_j + kappa Dloc_{j-1}) + (kappa b^j) D'_in, whose first term is formed before the D scan
+// and whose second needs one packed multiply-add per pair after it.
+//
+// The tile loop carries no special cases: the state before column 0 (est = L_0, Table 2) is set
+// up before the loop such that the decision value of column 0 cannot be negative, the scan
+// steps take their "has a partner lane" predicate from the shuffle itself, and
+// when the row is a whole number of tiles (FULL) there are no column guards.  Four tiles are
+// processed per trip so that ring slots and address offsets are compile-time constants.
+struct PairConstants {
+    float a4, b4;       // a^4, b^4: chain 0-3 -> chain 4-7
+    float kappa;        // la * beta * a
+    float kappa_b[4];   // kappa * b^j
+};
+
+// One step of the inclusive lane scan: x += m * (x of the lane `delta` below), for lanes that
+// have such a lane.  The shuffle's own predicate output says whether the source lane exists, so
+// no comparison on the lane index is needed.
+template <int DELTA>
+__device__ __forceinline__ float lane_scan_step(float x, float m) {
+    float r;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        ".reg .f32 y;\n\t"
+        "shfl.sync.up.b32 y|p, %1, %2, 0, 0xffffffff;\n\t"
+        "mov.f32 %0, %1;\n\t"
+        "@p fma.rn.f32 %0, %3, y, %1;\n\t"
+        "}"
+        : "=&f"(r)
+        : "f"(x), "n"(DELTA), "f"(m));
+    return r;
+}
+__device__ __forceinline__ float lane_affine_scan_pred(float x, const float (&step)[5]) {
+    x = lane_scan_step<1>(x, step[0]);
+    x = lane_scan_step<2>(x, step[1]);
+    x = lane_scan_step<4>(x, step[2]);
+    x = lane_scan_step<8>(x, step[3]);
+    x = lane_scan_step<16>(x, step[4]);
+    return x;
+}
+// Value of the lane below, zero in lane 0.
+__device__ __forceinline__ float lane_below_or_zero(float x) {
+    float r;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "shfl.sync.up.b32 %0|p, %1, 1, 0, 0xffffffff;\n\t"
+        "@!p mov.f32 %0, 0f00000000;\n\t"
+        "}"
+        : "=&f"(r)
+        : "f"(x));
+    return r;
+}
+
+template <bool BF16>
+__device__ __forceinline__ float unpack_lo(uint32_t u) {
+    if constexpr (BF16) return __uint_as_float(u << 16);
+    else return __half2float(__ushort_as_half(static_cast<unsigned short>(u & 0xffffu)));
+}
+template <bool BF16>
+__device__ __forceinline__ float unpack_hi(uint32_t u) {
+    if constexpr (BF16) return __uint_as_float(u & 0xffff0000u);
+    else return __half2float(__ushort_as_half(static_cast<unsigned short>(u >> 16)));
+}
+
+template <bool BF16, bool FULL, bool COUNT>
+__global__ void __launch_bounds__(kEwmaThreads, SP_EWMA_MIN_BLOCKS)
+ewma_pair_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
+                      const float *__restrict__ factor_pairs,
+                      const DeviceScalars *__restrict__ scalars,
+                      const __grid_constant__ ScanConstants sc,
+                      const __grid_constant__ PairConstants pc, uint32_t *__restrict__ mask,
+                      int mask_words, uint16_t *__restrict__ W_out, int ldo,
+                      unsigned long long *__restrict__ counters) {
+    static_assert(kEwmaPerLane == 8, "8 weights per lane");
+    pdl_launch_dependents();
+    pdl_wait();  // the per-channel factors come from an earlier kernel of the stream
+    const int lane = threadIdx.x & 31;
+    const int row = blockIdx.x * kEwmaWarps + (threadIdx.x >> 5);
+    if (row >= n_rows) return;  // warp-uniform
+    const uint16_t *wlane = W + static_cast<int64_t>(row) * ldw + lane * 8;
+    uint16_t *olane = W_out != nullptr ? W_out + static_cast<int64_t>(row) * ldo + lane * 8 : nullptr;
+    uint8_t *mlane = mask != nullptr
+                         ? reinterpret_cast<uint8_t *>(mask + static_cast<int64_t>(row) * mask_words) + lane
+                         : nullptr;
+    const float *flane = factor_pairs + lane * 8;
+    const int mask_bytes = mask_words * 4;
+
+    const float b = pinned(sc.b);
+    const float2 a2 = make_float2(pinned(sc.a), pinned(sc.a));
+    const float2 neg_alpha2 = make_float2(pinned(-sc.alpha), pinned(-sc.alpha));
+    const float a_lane = pinned(sc.a_lane[lane]), b_lane = pinned(sc.b_lane[lane]);
+    const float a4 = pinned(pc.a4), b4 = pinned(pc.b4), b8 = pinned(sc.b_step[0]);
+    const float kappa = pinned(pc.kappa);
+    float2 kappa_b2[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) kappa_b2[j] = make_float2(pinned(pc.kappa_b[j]), pinned(pc.kappa_b[j]));
+    uint32_t kept = 0;
+    uint32_t wmax = 0;
+
+    constexpr int kSlot = 32;  // uint4 per warp and stage
+    __shared__ __align__(16) uint4 ring[kEwmaWarps * kEwmaStages * kSlot];
+    uint4 *my_ring = ring + (threadIdx.x >> 5) * kEwmaStages * kSlot + lane;
+    const int tiles = (n + kEwmaTile - 1) / kEwmaTile;
+    const int n_lane = n - lane * 8;  // columns of the row at and after this lane's first one
+    auto issue_tile = [&](int t, int slot) {
+        if (FULL ? t < tiles : t * kEwmaTile < n_lane)
+            cp_async16(my_ring + slot * kSlot, wlane + t * kEwmaTile, 16);
+        cp_async_commit();
+    };
+#pragma unroll
+    for (int t = 0; t < kEwmaStages - 1; ++t) issue_tile(t, t);
+
+    // State before column 0: est = L_0, i.e. E = L_0 / alpha, lowered by one ulp when rounding
+    // would make  L_0 - alpha E  negative, so that column 0 is never pruned (Table 2).  Lane 0
+    // takes w_0 from its own first copy.
+    float carry_E, carry_D = 0.0f;
+    {
+        cp_async_wait<kEwmaStages - 2>();
+        const float w0 = unpack_lo<BF16>(my_ring[0].x);
+        const float L0 = __fmul_rn(__fmul_rn(w0, w0), __ldg(factor_pairs));
+        float e = L0 / sc.alpha;
+        if (fmaf(-sc.alpha, e, L0) < 0.0f) e = __uint_as_float(__float_as_uint(e) - 1u);
+        carry_E = __shfl_sync(kFullWarp, e, 0);
+    }
+
+    for (int t0 = 0; t0 < tiles; t0 += kEwmaStages) {
+#pragma unroll
+        for (int u = 0; u < kEwmaStages; ++u) {
+            const int tile = t0 + u;
+            if (tile >= tiles) break;  // warp-uniform
+            const int off = tile * kEwmaTile;  // column of lane 0
+            const bool in_row = FULL || off < n_lane;
+            issue_tile(tile + kEwmaStages - 1, (u + kEwmaStages - 1) & (kEwmaStages - 1));
+            cp_async_wait<kEwmaStages - 1>();
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (in_row) v = my_ring[u * kSlot];
+            uint32_t p[4] = {v.x, v.y, v.z, v.w};
+            // factors of columns (0,4,1,5 | 2,6,3,7) of the chunk, zero past d_in
+            const float4 c01 = __ldg(reinterpret_cast<const float4 *>(flane + off));
+            const float4 c23 = __ldg(reinterpret_cast<const float4 *>(flane + off) + 1);
+            float2 L2[4];  // (L_j, L_{j+4}), binary32 with one rounding per multiplication
+            {
+                float2 w2;
+                w2 = make_float2(unpack_lo<BF16>(p[0]), unpack_lo<BF16>(p[2]));
+                L2[0] = __fmul2_rn(__fmul2_rn(w2, w2), make_float2(c01.x, c01.y));
+                w2 = make_float2(unpack_hi<BF16>(p[0]), unpack_hi<BF16>(p[2]));
+                L2[1] = __fmul2_rn(__fmul2_rn(w2, w2), make_float2(c01.z, c01.w));
+                w2 = make_float2(unpack_lo<BF16>(p[1]), unpack_lo<BF16>(p[3]));
+                L2[2] = __fmul2_rn(__fmul2_rn(w2, w2), make_float2(c23.x, c23.y));
+                w2 = make_float2(unpack_hi<BF16>(p[1]), unpack_hi<BF16>(p[3]));
+                L2[3] = __fmul2_rn(__fmul2_rn(w2, w2), make_float2(c23.z, c23.w));
+            }
+            if constexpr (COUNT) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k) wmax = packed_abs_max<BF16>(wmax, p[k]);
+            }
+
+            // E: both chains from a zero state -> chain totals -> lane total -> scan over lanes.
+            float2 acc = L2[0];
+#pragma unroll
+            for (int j = 1; j < 4; ++j) acc = __ffma2_rn(a2, acc, L2[j]);
+            float incl = lane_affine_scan_pred(fmaf(a4, acc.x, acc.y), sc.a_step);
+            float excl = lane_below_or_zero(incl);
+            float2 E2;
+            E2.x = fmaf(a_lane, carry_E, excl);  // E before element 0
+            E2.y = fmaf(a4, E2.x, acc.x);        // E before element 4
+
+            // q and the true E along both chains.
+            float2 q2[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                q2[j] = __ffma2_rn(neg_alpha2, E2, L2[j]);
+                E2 = __ffma2_rn(a2, E2, L2[j]);
+            }
+            // D' of both chains from a zero state, and the part of the decision value known now.
+            float2 r2[4];
+            r2[0] = q2[0];
+            r2[1].x = fmaf(kappa, fabsf(q2[0].x), q2[1].x);
+            r2[1].y = fmaf(kappa, fabsf(q2[0].y), q2[1].y);
+            float2 dl;
+            dl.x = fmaf(b, fabsf(q2[0].x), fabsf(q2[1].x));
+            dl.y = fmaf(b, fabsf(q2[0].y), fabsf(q2[1].y));
+#pragma unroll
+            for (int j = 2; j < 4; ++j) {
+                r2[j] = __ffma2_rn(make_float2(kappa, kappa), dl, q2[j]);
+                dl.x = fmaf(b, dl.x, fabsf(q2[j].x));
+                dl.y = fmaf(b, dl.y, fabsf(q2[j].y));
+            }
+            const float d_total = fmaf(b4, dl.x, dl.y);
+            incl = lane_affine_scan_pred(d_total, sc.b_step);
+            excl = lane_below_or_zero(incl);
+            float2 D2;
+            D2.x = fmaf(b_lane, carry_D, excl);  // D' before element 0
+            D2.y = fmaf(b4, D2.x, dl.x);         // D' before element 4
+            const float D_end = fmaf(b8, D2.x, d_total);  // D' after element 7
+
+            // Decision values; their sign bits are the prune flags (a NaN is the positive
+            // canonical NaN: kept, as "L < threshold" is false).
+            float2 diff2[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) diff2[j] = __ffma2_rn(kappa_b2[j], D2, r2[j]);
+            uint32_t pm[4];
+            pm[0] = prmt(__float_as_uint(diff2[0].x), __float_as_uint(diff2[1].x), 0xffbbu);
+            pm[1] = prmt(__float_as_uint(diff2[2].x), __float_as_uint(diff2[3].x), 0xffbbu);
+            pm[2] = prmt(__float_as_uint(diff2[0].y), __float_as_uint(diff2[1].y), 0xffbbu);
+            pm[3] = prmt(__float_as_uint(diff2[2].y), __float_as_uint(diff2[3].y), 0xffbbu);
+            uint32_t keep8 = ~halfmasks_to_bits(pm) & 0xffu;
+            if (!in_row) keep8 = 0u;
+            if constexpr (COUNT) kept += __popc(keep8);
+
+            carry_E = __shfl_sync(kFullWarp, E2.y, 31);
+            carry_D = __shfl_sync(kFullWarp, D_end, 31);
+
+            if (olane != nullptr && in_row) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k) p[k] &= ~pm[k];
+                __stcs(reinterpret_cast<uint4 *>(olane + off), make_uint4(p[0], p[1], p[2], p[3]));
+            }
+            // one mask byte per lane: byte k of a little-endian word holds columns 8k .. 8k+7
+            if (mlane != nullptr && (FULL || (off >> 3) + lane < mask_bytes))
+                mlane[off >> 3] = static_cast<uint8_t>(keep8);
+        }
+    }
+
+    if constexpr (COUNT) {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) kept += __shfl_xor_sync(kFullWarp, kept, off);
+        float2 m2 = unpack2<BF16>(wmax);
+        float bound = fmaxf(m2.x, m2.y);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1)
+            bound = fmaxf(bound, __shfl_xor_sync(kFullWarp, bound, off));
+        if (lane == 0) {
+            atomicAdd(counters + SP_COUNTER_KEPT, static_cast<unsigned long long>(kept));
+            if (!(bound * bound < scalars->hazard_w2)) atomicAdd(counters + SP_COUNTER_S_HAZARD, 1ULL);
+        }
+    }
+}
+
 // Algorithm 1 exactly as printed, one thread per row, binary32 with one rounding per operation.
 // The row is read and written in chunks of 8 weights (16 bytes when aligned).  While S still
 // has its initial value the per-channel factor computed at finalisation is used: it was formed
@@ -472,11 +727,35 @@ sp_status launch_select_ewma(const sp_ctx *ctx, const void *W, sp_dtype dtype, i
     const float *factor = ctx->factor;
     const DeviceScalars *scalars = ctx->scalars;
     cudaError_t launch_err = cudaSuccess;
-#define SP_LAUNCH_C(B, V, C)                                                                 \
-    launch_err = cudaLaunchKernelEx(&pdl.cfg, ewma_scan_kernel<B, V, C>, Wp,                  \
+    PairConstants pc;
+    {
+        const double b = static_cast<double>(sc.b);
+        pc.a4 = static_cast<float>(pow(static_cast<double>(sc.a), 4.0));
+        pc.b4 = static_cast<float>(pow(b, 4.0));
+        const double kappa = static_cast<double>(p.la) * p.beta * sc.a;
+        pc.kappa = static_cast<float>(kappa);
+        for (int j = 0; j < 4; ++j) pc.kappa_b[j] = static_cast<float>(kappa * pow(b, j));
+    }
+    const bool full = n % kEwmaTile == 0;
+    const float *factor_pairs = ctx->factor_pairs;
+#define SP_LAUNCH_P(B, F, C)                                                                 \
+    launch_err = cudaLaunchKernelEx(&pdl.cfg, ewma_pair_scan_kernel<B, F, C>, Wp,             \
+                                    static_cast<int>(ldw), static_cast<int>(n_rows),          \
+                                    static_cast<int>(n), factor_pairs, scalars, sc, pc, mask, \
+                                    static_cast<int>(words), Op, static_cast<int>(ldo), counters)
+#define SP_LAUNCH_S(B, C)                                                                    \
+    launch_err = cudaLaunchKernelEx(&pdl.cfg, ewma_scan_kernel<B, false, C>, Wp,              \
                                     static_cast<int>(ldw), static_cast<int>(n_rows),          \
                                     static_cast<int>(n), factor, scalars, sc, mask,           \
                                     static_cast<int>(words), Op, static_cast<int>(ldo), counters)
+#define SP_LAUNCH_C(B, V, C)                                                                 \
+    do {                                                                                     \
+        if (V) {                                                                             \
+            if (full) SP_LAUNCH_P(B, true, C); else SP_LAUNCH_P(B, false, C);                \
+        } else {                                                                             \
+            SP_LAUNCH_S(B, C);                                                               \
+        }                                                                                    \
+    } while (0)
 #define SP_LAUNCH(B, V)                                                                      \
     do {                                                                                     \
         if (counters != nullptr) SP_LAUNCH_C(B, V, true); else SP_LAUNCH_C(B, V, false);     \
@@ -488,6 +767,8 @@ sp_status launch_select_ewma(const sp_ctx *ctx, const void *W, sp_dtype dtype, i
     }
 #undef SP_LAUNCH
 #undef SP_LAUNCH_C
+#undef SP_LAUNCH_S
+#undef SP_LAUNCH_P
     if (launch_err != cudaSuccess) return cuda_fail(launch_err);
     return check_launch();
 }

@@ -1,20 +1,19 @@
 // EWMA running-threshold selection (Algorithm 1; state rules of Table 2) fused with score,
 // mask emission and write-back.
 //
-// Frozen-S path (scan kernel).  With S fixed, est and dev do not depend on the prune
+// Frozen-S path (scan kernels).  With S fixed, est and dev do not depend on the prune
 // decisions: est_i = a est_{i-1} + alpha L_i and dev_i = b dev_{i-1} + beta |est_i - L_i|
 // (a = 1-alpha, b = 1-beta) are first-order linear recurrences, evaluated as affine scans.
-// One warp owns one row and walks it in tiles of 32*P weights; a lane owns P consecutive
-// weights (P = 8 by default, 16 as a build option).  Per tile and recurrence: the lane runs the
-// recurrence over its P elements from a zero state to get its total, a 5-step shuffle scan with
-// the constant multipliers a^(P*2^k) combines the lane totals, and the lane runs the recurrence
-// again from the state entering it (the scan's exclusive prefix plus a^(P*lane) times the state
-// carried in from the previous tile), which needs no per-element constants and keeps few values
-// live.  Element i is
-// tested against the state before its own update, est_{i-1} - la*dev_{i-1}; est_{-1} = L_0 and
-// dev_{-1} = 0 (Table 2), so column 0 is never pruned.  The weights of the next few tiles are
-// already on their way into shared memory (asynchronous copies) while a tile is processed; only
-// the two carried scalars serialise the tiles.
+// One warp owns one row and walks it in tiles of 256 weights; a lane owns 8 consecutive
+// weights.  Per tile and recurrence: the lane runs the recurrence over its elements from a zero
+// state to get its total, a 5-step shuffle scan with the constant multipliers a^(8*2^k)
+// combines the lane totals, and the lane obtains its true states from the state entering it
+// (the scan's exclusive prefix plus a^(8*lane) times the state carried in from the previous
+// tile).  Element i is tested against the state before its own update,
+// est_{i-1} - la*dev_{i-1}; est_{-1} = L_0 and dev_{-1} = 0 (Table 2), so column 0 is never
+// pruned.  Two kernels: ewma_pair_scan_kernel for rows that allow 16-byte access (the fast
+// path: packed binary32 pairs, weights streamed through a shared-memory ring of asynchronous
+// copies) and ewma_scan_kernel for any other pointer, stride or width.
 //
 // Literal-S path (sequential kernel).  Algorithm 1's "S = S - w_i^2" makes L_i depend on
 // earlier decisions, so the row is evaluated in order by one thread, every operation in
@@ -31,23 +30,11 @@ namespace sp {
 #endif
 constexpr int kEwmaThreads = 256;
 constexpr int kEwmaWarps = kEwmaThreads / 32;
-#ifndef SP_EWMA_PER_LANE
-#define SP_EWMA_PER_LANE 8
-#endif
-#ifndef SP_EWMA_RING
-#define SP_EWMA_RING 1
-#endif
-constexpr int kEwmaPerLane = SP_EWMA_PER_LANE;    // consecutive weights per lane (8 or 16)
-constexpr int kEwmaHalves = kEwmaPerLane / 8;     // 16-byte pieces per lane and tile
-constexpr bool kEwmaRing = SP_EWMA_RING != 0;     // stage tiles through shared memory
+constexpr int kEwmaPerLane = 8;                   // consecutive weights per lane
 constexpr int kEwmaTile = 32 * kEwmaPerLane;      // weights per warp tile
 #ifndef SP_EWMA_STAGES
 #define SP_EWMA_STAGES 4
 #endif
-#ifndef SP_EWMA_UNROLL
-#define SP_EWMA_UNROLL 1
-#endif
-constexpr int kEwmaUnroll = SP_EWMA_UNROLL;       // tiles per iteration of the tile loop
 constexpr int kEwmaStages = SP_EWMA_STAGES;       // ring slots per warp (a power of two)
 static_assert((kEwmaStages & (kEwmaStages - 1)) == 0, "ring size must be a power of two");
 
@@ -88,8 +75,9 @@ __device__ __forceinline__ float pinned(float v) {
     return r;
 }
 
+// General scan kernel: element-wise access with bounds checks, any alignment, stride or width.
 // COUNT: also produce the kept-weight count and the S-hazard flag of the row.
-template <bool BF16, bool VEC, bool COUNT>
+template <bool BF16, bool COUNT>
 __global__ void __launch_bounds__(kEwmaThreads, SP_EWMA_MIN_BLOCKS)
 ewma_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
                  const float *__restrict__ factor, const DeviceScalars *__restrict__ scalars,
@@ -117,72 +105,24 @@ ewma_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
     float carry_E = 0.0f, carry_D = 0.0f;
     uint32_t kept = 0;
     uint32_t wmax = 0;  // packed running max of |w| over this lane's elements
+    uint32_t p_next[4];
+    load8<false, true>(wrow, lane * kEwmaPerLane, n, p_next);
 
-    // Aligned path: every lane streams its own 16*kEwmaHalves bytes of each tile through a private
-    // slot of a shared-memory ring with asynchronous copies, kEwmaStages-1 tiles ahead of the tile
-    // being processed; a lane only ever reads what it copied itself, so waiting on its own copy
-    // groups is the only synchronisation.  (Layout: the 16-byte pieces of the 32 lanes are stored
-    // as contiguous 512-byte rows, which keeps the 16-byte shared loads conflict-free.)
-    constexpr bool RING = VEC && kEwmaRing;
-    constexpr int kSlot = 32 * kEwmaHalves;  // uint4 per warp and stage
-    __shared__ __align__(16) uint4 ring[RING ? kEwmaWarps * kEwmaStages * kSlot : 1];
-    uint4 *my_ring = ring + (RING ? (threadIdx.x >> 5) * kEwmaStages * kSlot + lane : 0);
-    auto issue_tile = [&](int t) {
-        if constexpr (RING) {
-            if (t < tiles) {
-                const int c0 = t * kEwmaTile + lane * kEwmaPerLane;
-                uint4 *slot = my_ring + (t & (kEwmaStages - 1)) * kSlot;
-#pragma unroll
-                for (int h = 0; h < kEwmaHalves; ++h)
-                    cp_async16(slot + 32 * h, wrow + min(c0 + 8 * h, n - 8),
-                               c0 + 8 * h < n ? 16 : 0);
-            }
-            cp_async_commit();
-        }
-    };
-#pragma unroll
-    for (int t = 0; t < kEwmaStages - 1; ++t) issue_tile(t);
-    uint32_t p_next[kEwmaHalves][4];
-    if constexpr (!RING) {
-#pragma unroll
-        for (int h = 0; h < kEwmaHalves; ++h)
-            load8<VEC, true>(wrow, lane * kEwmaPerLane + 8 * h, n, p_next[h]);
-    }
-
-#pragma unroll kEwmaUnroll
     for (int tile = 0; tile < tiles; ++tile) {
         const int col = tile * kEwmaTile + lane * kEwmaPerLane;
-        uint32_t p[kEwmaHalves][4];
-        if constexpr (RING) {
-            issue_tile(tile + kEwmaStages - 1);
-            cp_async_wait<kEwmaStages - 1>();
-            const uint4 *slot = my_ring + (tile & (kEwmaStages - 1)) * kSlot;
+        uint32_t p[4];
 #pragma unroll
-            for (int h = 0; h < kEwmaHalves; ++h) {
-                const uint4 v = slot[32 * h];
-                p[h][0] = v.x; p[h][1] = v.y; p[h][2] = v.z; p[h][3] = v.w;
-            }
-        } else {
-#pragma unroll
-            for (int h = 0; h < kEwmaHalves; ++h) {
-#pragma unroll
-                for (int k = 0; k < 4; ++k) p[h][k] = p_next[h][k];
-                if (tile + 1 < tiles) load8<VEC, true>(wrow, col + kEwmaTile + 8 * h, n, p_next[h]);
-            }
-        }
+        for (int k = 0; k < 4; ++k) p[k] = p_next[k];
+        if (tile + 1 < tiles) load8<false, true>(wrow, col + kEwmaTile, n, p_next);
 
-        float L[kEwmaPerLane];
+        float L[kEwmaPerLane], w[8], c[8];
+        unpack8<BF16>(p, w);
+        load_factor8(factor, col, c);  // zero past d_in: scores of padding are 0
 #pragma unroll
-        for (int h = 0; h < kEwmaHalves; ++h) {
-            float w[8], c[8];
-            unpack8<BF16>(p[h], w);
-            load_factor8(factor, col + 8 * h, c);  // zero past d_in: scores of padding are 0
+        for (int j = 0; j < 8; ++j) L[j] = __fmul_rn(__fmul_rn(w[j], w[j]), c[j]);
+        if constexpr (COUNT) {
 #pragma unroll
-            for (int j = 0; j < 8; ++j) L[8 * h + j] = __fmul_rn(__fmul_rn(w[j], w[j]), c[j]);
-            if constexpr (COUNT) {
-#pragma unroll
-                for (int k = 0; k < 4; ++k) wmax = packed_abs_max<BF16>(wmax, p[h][k]);
-            }
+            for (int k = 0; k < 4; ++k) wmax = packed_abs_max<BF16>(wmax, p[k]);
         }
 
         if (tile == 0) carry_E = __shfl_sync(kFullWarp, L[0], 0) / alpha;  // est starts at L_0
@@ -224,44 +164,30 @@ ewma_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
             diff[j] = fmaf(la_beta, D_run, q[j]);
             D_run = fmaf(b, D_run, dabs[j]);
         }
-        uint32_t pm[kEwmaHalves][4];
+        uint32_t pm[4];
 #pragma unroll
-        for (int h = 0; h < kEwmaHalves; ++h)
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-                pm[h][k] = prmt(__float_as_uint(diff[8 * h + 2 * k]),
-                                __float_as_uint(diff[8 * h + 2 * k + 1]), 0xffbbu);
-        uint32_t pruned = halfmasks_to_bits(pm[0]);
-        if constexpr (kEwmaHalves == 2) pruned |= halfmasks_to_bits(pm[kEwmaHalves - 1]) << 8;
-        uint32_t keep16 = ~pruned & ((1u << kEwmaPerLane) - 1u);
-        if (tile == 0 && lane == 0 && (keep16 & 1u) == 0u) {
+        for (int k = 0; k < 4; ++k)
+            pm[k] = prmt(__float_as_uint(diff[2 * k]), __float_as_uint(diff[2 * k + 1]), 0xffbbu);
+        uint32_t keep8 = ~halfmasks_to_bits(pm) & 0xffu;
+        if (tile == 0 && lane == 0 && (keep8 & 1u) == 0u) {
             // column 0 is kept by definition (est starts at L_0); alpha*(L_0/alpha) may round up
-            keep16 |= 1u;
-            pm[0][0] &= 0xffff0000u;
+            keep8 |= 1u;
+            pm[0] &= 0xffff0000u;
         }
         const int left = n - col;
-        if (left < kEwmaPerLane) keep16 &= left > 0 ? ((1u << left) - 1u) : 0u;
-        if constexpr (COUNT) kept += __popc(keep16);
+        if (left < kEwmaPerLane) keep8 &= left > 0 ? ((1u << left) - 1u) : 0u;
+        if constexpr (COUNT) kept += __popc(keep8);
 
         carry_E = __shfl_sync(kFullWarp, E_run, 31);
         carry_D = __shfl_sync(kFullWarp, D_run, 31);
 
         if (orow != nullptr) {
 #pragma unroll
-            for (int h = 0; h < kEwmaHalves; ++h) {
-#pragma unroll
-                for (int k = 0; k < 4; ++k) p[h][k] &= ~pm[h][k];
-                store8<VEC>(orow, col + 8 * h, n, p[h]);
-            }
+            for (int k = 0; k < 4; ++k) p[k] &= ~pm[k];
+            store8<false>(orow, col, n, p);
         }
-        if constexpr (kEwmaPerLane == 16) {  // two lanes share a 32-bit mask word
-            uint32_t word = keep16 << (16 * (lane & 1));
-            word |= __shfl_xor_sync(kFullWarp, word, 1);
-            if (mrow != nullptr && (lane & 1) == 0 && col < n) mrow[col >> 5] = word;
-        } else {                             // four lanes share one
-            const uint32_t word = gather_mask_word(keep16, lane);
-            if (mrow != nullptr && (lane & 3) == 0 && col < n) mrow[col >> 5] = word;
-        }
+        const uint32_t word = gather_mask_word(keep8, lane);  // four lanes share a mask word
+        if (mrow != nullptr && (lane & 3) == 0 && col < n) mrow[col >> 5] = word;
     }
 
     if constexpr (COUNT) {
@@ -420,6 +346,8 @@ ewma_pair_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n
         carry_E = __shfl_sync(kFullWarp, e, 0);
     }
 
+    float4 c01_next = __ldg(reinterpret_cast<const float4 *>(flane));
+    float4 c23_next = __ldg(reinterpret_cast<const float4 *>(flane) + 1);
     for (int t0 = 0; t0 < tiles; t0 += kEwmaStages) {
 #pragma unroll
         for (int u = 0; u < kEwmaStages; ++u) {
@@ -427,14 +355,16 @@ ewma_pair_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n
             if (tile >= tiles) break;  // warp-uniform
             const int off = tile * kEwmaTile;  // column of lane 0
             const bool in_row = FULL || off < n_lane;
+            // factors of columns (0,4,1,5 | 2,6,3,7) of the chunk, zero past d_in; those of
+            // the next tile are requested now (the array is padded by one tile of zeros)
+            const float4 c01 = c01_next, c23 = c23_next;
+            c01_next = __ldg(reinterpret_cast<const float4 *>(flane + off + kEwmaTile));
+            c23_next = __ldg(reinterpret_cast<const float4 *>(flane + off + kEwmaTile) + 1);
             issue_tile(tile + kEwmaStages - 1, (u + kEwmaStages - 1) & (kEwmaStages - 1));
             cp_async_wait<kEwmaStages - 1>();
             uint4 v = make_uint4(0u, 0u, 0u, 0u);
             if (in_row) v = my_ring[u * kSlot];
             uint32_t p[4] = {v.x, v.y, v.z, v.w};
-            // factors of columns (0,4,1,5 | 2,6,3,7) of the chunk, zero past d_in
-            const float4 c01 = __ldg(reinterpret_cast<const float4 *>(flane + off));
-            const float4 c23 = __ldg(reinterpret_cast<const float4 *>(flane + off) + 1);
             float2 L2[4];  // (L_j, L_{j+4}), binary32 with one rounding per multiplication
             {
                 float2 w2;
@@ -739,12 +669,12 @@ sp_status launch_select_ewma(const sp_ctx *ctx, const void *W, sp_dtype dtype, i
     const bool full = n % kEwmaTile == 0;
     const float *factor_pairs = ctx->factor_pairs;
 #define SP_LAUNCH_P(B, F, C)                                                                 \
-    launch_err = cudaLaunchKernelEx(&pdl.cfg, ewma_pair_scan_kernel<B, F, C>, Wp,             \
+    launch_err = cudaLaunchKernelEx(&pdl.cfg, ewma_pair_scan_kernel<B, F, C>, Wp,            \
                                     static_cast<int>(ldw), static_cast<int>(n_rows),          \
                                     static_cast<int>(n), factor_pairs, scalars, sc, pc, mask, \
                                     static_cast<int>(words), Op, static_cast<int>(ldo), counters)
 #define SP_LAUNCH_S(B, C)                                                                    \
-    launch_err = cudaLaunchKernelEx(&pdl.cfg, ewma_scan_kernel<B, false, C>, Wp,              \
+    launch_err = cudaLaunchKernelEx(&pdl.cfg, ewma_scan_kernel<B, C>, Wp,              \
                                     static_cast<int>(ldw), static_cast<int>(n_rows),          \
                                     static_cast<int>(n), factor, scalars, sc, mask,           \
                                     static_cast<int>(words), Op, static_cast<int>(ldo), counters)

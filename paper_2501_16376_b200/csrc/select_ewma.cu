@@ -260,20 +260,6 @@ __device__ __forceinline__ float lane_affine_scan_pred(float x, const float (&st
     x = lane_scan_step<16>(x, step[4]);
     return x;
 }
-// Value of the lane below, zero in lane 0.
-__device__ __forceinline__ float lane_below_or_zero(float x) {
-    float r;
-    asm volatile(
-        "{\n\t"
-        ".reg .pred p;\n\t"
-        "shfl.sync.up.b32 %0|p, %1, 1, 0, 0xffffffff;\n\t"
-        "@!p mov.f32 %0, 0f00000000;\n\t"
-        "}"
-        : "=&f"(r)
-        : "f"(x));
-    return r;
-}
-
 template <bool BF16>
 __device__ __forceinline__ float unpack_lo(uint32_t u) {
     if constexpr (BF16) return __uint_as_float(u << 16);
@@ -311,8 +297,12 @@ ewma_pair_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n
     const float b = pinned(sc.b);
     const float2 a2 = make_float2(pinned(sc.a), pinned(sc.a));
     const float2 neg_alpha2 = make_float2(pinned(-sc.alpha), pinned(-sc.alpha));
-    const float a_lane = pinned(sc.a_lane[lane]), b_lane = pinned(sc.b_lane[lane]);
-    const float a4 = pinned(pc.a4), b4 = pinned(pc.b4), b8 = pinned(sc.b_step[0]);
+    const float a4 = pinned(pc.a4), b4 = pinned(pc.b4);
+    // lane 0 folds the state carried in from the previous tile into its total before the scan
+    const float a8_lane0 = pinned(lane == 0 ? sc.a_step[0] : 0.0f);
+    const float b8_lane0 = pinned(lane == 0 ? sc.b_step[0] : 0.0f);
+    const int lane_below = (lane + 31) & 31;
+    const bool is_lane0 = lane == 0;
     const float kappa = pinned(pc.kappa);
     float2 kappa_b2[4];
 #pragma unroll
@@ -343,7 +333,7 @@ ewma_pair_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n
         const float L0 = __fmul_rn(__fmul_rn(w0, w0), __ldg(factor_pairs));
         float e = L0 / sc.alpha;
         if (fmaf(-sc.alpha, e, L0) < 0.0f) e = __uint_as_float(__float_as_uint(e) - 1u);
-        carry_E = __shfl_sync(kFullWarp, e, 0);
+        carry_E = is_lane0 ? e : 0.0f;  // only lane 0's copy of the carried states is used
     }
 
     float4 c01_next = __ldg(reinterpret_cast<const float4 *>(flane));
@@ -386,11 +376,16 @@ ewma_pair_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n
             float2 acc = L2[0];
 #pragma unroll
             for (int j = 1; j < 4; ++j) acc = __ffma2_rn(a2, acc, L2[j]);
-            float incl = lane_affine_scan_pred(fmaf(a4, acc.x, acc.y), sc.a_step);
-            float excl = lane_below_or_zero(incl);
+            // (lane 0 adds a^8 times the state carried in, so the scanned values are true states)
+            float incl = lane_affine_scan_pred(
+                fmaf(a8_lane0, carry_E, fmaf(a4, acc.x, acc.y)), sc.a_step);
+            // one rotation hands every lane the state before its first element (the end state of
+            // the lane below) and lane 0 the end state of the tile, which it carries on
+            float rot = __shfl_sync(kFullWarp, incl, lane_below);
             float2 E2;
-            E2.x = fmaf(a_lane, carry_E, excl);  // E before element 0
-            E2.y = fmaf(a4, E2.x, acc.x);        // E before element 4
+            E2.x = is_lane0 ? carry_E : rot;  // E before element 0
+            E2.y = fmaf(a4, E2.x, acc.x);     // E before element 4
+            carry_E = rot;
 
             // q and the true E along both chains.
             float2 q2[4];
@@ -414,12 +409,12 @@ ewma_pair_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n
                 dl.y = fmaf(b, dl.y, fabsf(q2[j].y));
             }
             const float d_total = fmaf(b4, dl.x, dl.y);
-            incl = lane_affine_scan_pred(d_total, sc.b_step);
-            excl = lane_below_or_zero(incl);
+            incl = lane_affine_scan_pred(fmaf(b8_lane0, carry_D, d_total), sc.b_step);
+            rot = __shfl_sync(kFullWarp, incl, lane_below);
             float2 D2;
-            D2.x = fmaf(b_lane, carry_D, excl);  // D' before element 0
-            D2.y = fmaf(b4, D2.x, dl.x);         // D' before element 4
-            const float D_end = fmaf(b8, D2.x, d_total);  // D' after element 7
+            D2.x = is_lane0 ? carry_D : rot;  // D' before element 0
+            D2.y = fmaf(b4, D2.x, dl.x);      // D' before element 4
+            carry_D = rot;
 
             // Decision values; their sign bits are the prune flags (a NaN is the positive
             // canonical NaN: kept, as "L < threshold" is false).
@@ -434,9 +429,6 @@ ewma_pair_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n
             uint32_t keep8 = ~halfmasks_to_bits(pm) & 0xffu;
             if (!in_row) keep8 = 0u;
             if constexpr (COUNT) kept += __popc(keep8);
-
-            carry_E = __shfl_sync(kFullWarp, E2.y, 31);
-            carry_D = __shfl_sync(kFullWarp, D_end, 31);
 
             if (olane != nullptr && in_row) {
 #pragma unroll

@@ -102,7 +102,7 @@ sp_status sp_create(sp_ctx **out, int64_t d_in, int device) {
                              sizeof(double) * static_cast<size_t>(ctx->strips),
                              sizeof(float) * (np + kStripChannels),
                              sizeof(DeviceScalars),
-                             sizeof(float) * (np + kStripChannels)};
+                             sizeof(float) * ((np + 511) / 512 * 512 + 512)};
     for (int i = 0; i < 6; ++i) {
         e = cudaMalloc(&ptrs[i], sizes[i]);
         if (e == cudaSuccess) e = cudaMemset(ptrs[i], 0, sizes[i]);

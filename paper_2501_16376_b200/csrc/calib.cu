@@ -198,10 +198,15 @@ finalize_kernel(const double *__restrict__ partial, int slabs_valid, int64_t n, 
                     c = __fdiv_rn(0.5f, den);
                 }
                 factor[q] = c;
-                // second copy for kernels that pair column j with column j+4 of a chunk of 8
+                // Second copy for the EWMA pair kernel, whose lanes own 16 consecutive columns
+                // of a 512-column tile and pair column j of a chunk of 8 with column j + 4:
+                // [tile][float4 i = 2 * chunk + pos / 4][lane][pos % 4], pos = place of the
+                // column in the order 0,4,1,5,2,6,3,7.
                 if (factor_pairs != nullptr) {
                     const int64_t e = q & 7;
-                    factor_pairs[(q & ~int64_t(7)) | (e < 4 ? 2 * e : 2 * (e - 4) + 1)] = c;
+                    const int64_t pos = e < 4 ? 2 * e : 2 * (e - 4) + 1;
+                    const int64_t r = q & 511, ln = r >> 4, ch = (r >> 3) & 1;
+                    factor_pairs[(q & ~int64_t(511)) + (2 * ch + (pos >> 2)) * 128 + ln * 4 + (pos & 3)] = c;
                 }
             }
         }

@@ -32,6 +32,14 @@ constexpr int kEwmaThreads = 256;
 constexpr int kEwmaWarps = kEwmaThreads / 32;
 constexpr int kEwmaPerLane = 8;                   // consecutive weights per lane
 constexpr int kEwmaTile = 32 * kEwmaPerLane;      // weights per warp tile
+#ifndef SP_EWMA_PAIR_THREADS
+#define SP_EWMA_PAIR_THREADS 128
+#endif
+#ifndef SP_EWMA_PAIR_MIN_BLOCKS
+#define SP_EWMA_PAIR_MIN_BLOCKS 8
+#endif
+constexpr int kPairThreads = SP_EWMA_PAIR_THREADS;
+constexpr int kPairWarps = kPairThreads / 32;
 #ifndef SP_EWMA_STAGES
 #define SP_EWMA_STAGES 4
 #endif
@@ -205,13 +213,15 @@ ewma_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
     }
 }
 
-// Paired-chain variant of the scan kernel for rows that allow 16-byte access.
+// Paired-chain scan kernel for rows that allow 16-byte access.
 //
-// Same decomposition (warp per row, 8 consecutive weights per lane, two lane scans per tile),
-// but the lane's 8 elements are treated as two chains of 4 (elements 0-3 and 4-7) that advance
-// together in the two halves of packed binary32 pairs (fma.rn.f32x2: one issue slot for two
-// fused multiply-adds).  The second chain starts from the state the first one ends in, which is
-// known as soon as the first chain's zero-state total is: E(4) = a^4 E(0) + T_lo.
+// Same decomposition as ewma_scan_kernel (warp per row, two lane scans per tile), but a lane
+// owns 16 consecutive weights (two 16-byte chunks) and a tile is 512 weights.  Each chunk is
+// treated as two chains of 4 (elements 0-3 and 4-7) that advance together in the two halves of
+// packed binary32 pairs (fma.rn.f32x2: one issue slot for two fused multiply-adds); the two
+// chunks give every warp two independent instruction streams.  A later chain starts from the
+// state the previous one ends in, which is known as soon as the previous chain's zero-state
+// total is: E(4) = a^4 E(0) + T_0, E(8) = a^8 E(0) + (a^4 T_0 + T_1), ...
 //
 // Algebra used (scaled states E = est/alpha, D' = dev/(beta a)):
 //     q_i  = L_i - alpha E_{i-1}                  (score minus the estimate it is tested against)
@@ -225,9 +235,20 @@ ewma_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
 //
 // The tile loop carries no special cases: the state before column 0 (est = L_0, Table 2) is set
 // up before the loop such that the decision value of column 0 cannot be negative, the scan
-// steps take their "has a partner lane" predicate from the shuffle itself, and
-// when the row is a whole number of tiles (FULL) there are no column guards.  Four tiles are
+// steps take their "has a partner lane" predicate from the shuffle itself, lane 0 folds the
+// state carried in from the previous tile into its total before the scan (one lane rotation
+// then gives every lane the state it starts from and lane 0 the state to carry on), and when
+// the row is a whole number of tiles (FULL) there are no column guards.  Four tiles are
 // processed per trip so that ring slots and address offsets are compile-time constants.
+//
+// Shared-memory ring: the copies of a tile are issued coalesced (instruction h moves the
+// 16-byte chunk 32h + lane), while a lane reads chunks 2*lane and 2*lane + 1.  Chunk g is kept
+// at position g ^ ((g >> 3) & 1): both the coalesced writes and the strided reads then touch
+// eight different bank groups per quarter warp.
+//
+// The per-channel factors come from a copy of the factor array laid out for this kernel (see
+// finalize_kernel): per 512-column tile, four 16-byte loads per lane, each contiguous across
+// the warp, deliver the lane's 16 factors in pair order (columns 0,4,1,5 | 2,6,3,7 of a chunk).
 struct PairConstants {
     float a4, b4;       // a^4, b^4: chain 0-3 -> chain 4-7
     float kappa;        // la * beta * a
@@ -271,173 +292,201 @@ __device__ __forceinline__ float unpack_hi(uint32_t u) {
     else return __half2float(__ushort_as_half(static_cast<unsigned short>(u >> 16)));
 }
 
+struct TileConstants {
+    float a_step[5], b_step[5];  // a^(16*2^k), b^(16*2^k)
+    float a8, b8;
+};
+
 template <bool BF16, bool FULL, bool COUNT>
-__global__ void __launch_bounds__(kEwmaThreads, SP_EWMA_MIN_BLOCKS)
+__global__ void __launch_bounds__(kPairThreads, SP_EWMA_PAIR_MIN_BLOCKS)
 ewma_pair_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
                       const float *__restrict__ factor_pairs,
                       const DeviceScalars *__restrict__ scalars,
                       const __grid_constant__ ScanConstants sc,
-                      const __grid_constant__ PairConstants pc, uint32_t *__restrict__ mask,
+                      const __grid_constant__ PairConstants pc,
+                      const __grid_constant__ TileConstants wc, uint32_t *__restrict__ mask,
                       int mask_words, uint16_t *__restrict__ W_out, int ldo,
                       unsigned long long *__restrict__ counters) {
-    static_assert(kEwmaPerLane == 8, "8 weights per lane");
+    constexpr int kTile = 512;
     pdl_launch_dependents();
     pdl_wait();  // the per-channel factors come from an earlier kernel of the stream
     const int lane = threadIdx.x & 31;
-    const int row = blockIdx.x * kEwmaWarps + (threadIdx.x >> 5);
+    const int row = blockIdx.x * kPairWarps + (threadIdx.x >> 5);
     if (row >= n_rows) return;  // warp-uniform
-    const uint16_t *wlane = W + static_cast<int64_t>(row) * ldw + lane * 8;
-    uint16_t *olane = W_out != nullptr ? W_out + static_cast<int64_t>(row) * ldo + lane * 8 : nullptr;
-    uint8_t *mlane = mask != nullptr
-                         ? reinterpret_cast<uint8_t *>(mask + static_cast<int64_t>(row) * mask_words) + lane
-                         : nullptr;
-    const float *flane = factor_pairs + lane * 8;
-    const int mask_bytes = mask_words * 4;
+    const uint16_t *wrow = W + static_cast<int64_t>(row) * ldw;
+    uint16_t *olane = W_out != nullptr ? W_out + static_cast<int64_t>(row) * ldo + lane * 16 : nullptr;
+    uint16_t *mlane = mask != nullptr
+                          ? reinterpret_cast<uint16_t *>(mask + static_cast<int64_t>(row) * mask_words) + lane
+                          : nullptr;
+    const float4 *flane = reinterpret_cast<const float4 *>(factor_pairs) + lane;
+    const int mask_halves = mask_words * 2;
 
     const float b = pinned(sc.b);
     const float2 a2 = make_float2(pinned(sc.a), pinned(sc.a));
     const float2 neg_alpha2 = make_float2(pinned(-sc.alpha), pinned(-sc.alpha));
-    const float a4 = pinned(pc.a4), b4 = pinned(pc.b4);
+    const float a4 = pinned(pc.a4), b4 = pinned(pc.b4), a8 = pinned(wc.a8), b8 = pinned(wc.b8);
     // lane 0 folds the state carried in from the previous tile into its total before the scan
-    const float a8_lane0 = pinned(lane == 0 ? sc.a_step[0] : 0.0f);
-    const float b8_lane0 = pinned(lane == 0 ? sc.b_step[0] : 0.0f);
+    const float a16_lane0 = pinned(lane == 0 ? sc.a_step[1] : 0.0f);
+    const float b16_lane0 = pinned(lane == 0 ? sc.b_step[1] : 0.0f);
     const int lane_below = (lane + 31) & 31;
     const bool is_lane0 = lane == 0;
     const float kappa = pinned(pc.kappa);
+    const float2 kappa2 = make_float2(kappa, kappa);
     float2 kappa_b2[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) kappa_b2[j] = make_float2(pinned(pc.kappa_b[j]), pinned(pc.kappa_b[j]));
     uint32_t kept = 0;
     uint32_t wmax = 0;
 
-    constexpr int kSlot = 32;  // uint4 per warp and stage
-    __shared__ __align__(16) uint4 ring[kEwmaWarps * kEwmaStages * kSlot];
-    uint4 *my_ring = ring + (threadIdx.x >> 5) * kEwmaStages * kSlot + lane;
-    const int tiles = (n + kEwmaTile - 1) / kEwmaTile;
-    const int n_lane = n - lane * 8;  // columns of the row at and after this lane's first one
+    constexpr int kSlot = 64;  // uint4 per warp and stage
+    __shared__ __align__(16) uint4 ring[kPairWarps * kEwmaStages * kSlot];
+    uint4 *my_ring = ring + (threadIdx.x >> 5) * kEwmaStages * kSlot;
+    const int wpos = lane ^ ((lane >> 3) & 1);               // where this lane's copies go
+    const int rpos_a = 2 * lane + ((lane >> 2) & 1);         // where chunk 2*lane sits
+    const int rpos_b = 2 * lane + 1 - ((lane >> 2) & 1);     // where chunk 2*lane + 1 sits
+    const int tiles = (n + kTile - 1) / kTile;
     auto issue_tile = [&](int t, int slot) {
-        if (FULL ? t < tiles : t * kEwmaTile < n_lane)
-            cp_async16(my_ring + slot * kSlot, wlane + t * kEwmaTile, 16);
+        if (t < tiles) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int c = t * kTile + (32 * h + lane) * 8;
+                if (FULL || c < n) cp_async16(my_ring + slot * kSlot + 32 * h + wpos, wrow + c, 16);
+            }
+        }
         cp_async_commit();
     };
 #pragma unroll
     for (int t = 0; t < kEwmaStages - 1; ++t) issue_tile(t, t);
 
     // State before column 0: est = L_0, i.e. E = L_0 / alpha, lowered by one ulp when rounding
-    // would make  L_0 - alpha E  negative, so that column 0 is never pruned (Table 2).  Lane 0
-    // takes w_0 from its own first copy.
+    // would make  L_0 - alpha E  negative, so that column 0 is never pruned (Table 2).
     float carry_E, carry_D = 0.0f;
     {
         cp_async_wait<kEwmaStages - 2>();
-        const float w0 = unpack_lo<BF16>(my_ring[0].x);
+        const float w0 = unpack_lo<BF16>(my_ring[rpos_a].x);  // lane 0: its own copy of chunk 0
         const float L0 = __fmul_rn(__fmul_rn(w0, w0), __ldg(factor_pairs));
         float e = L0 / sc.alpha;
         if (fmaf(-sc.alpha, e, L0) < 0.0f) e = __uint_as_float(__float_as_uint(e) - 1u);
         carry_E = is_lane0 ? e : 0.0f;  // only lane 0's copy of the carried states is used
     }
 
-    float4 c01_next = __ldg(reinterpret_cast<const float4 *>(flane));
-    float4 c23_next = __ldg(reinterpret_cast<const float4 *>(flane) + 1);
     for (int t0 = 0; t0 < tiles; t0 += kEwmaStages) {
 #pragma unroll
         for (int u = 0; u < kEwmaStages; ++u) {
             const int tile = t0 + u;
             if (tile >= tiles) break;  // warp-uniform
-            const int off = tile * kEwmaTile;  // column of lane 0
-            const bool in_row = FULL || off < n_lane;
-            // factors of columns (0,4,1,5 | 2,6,3,7) of the chunk, zero past d_in; those of
-            // the next tile are requested now (the array is padded by one tile of zeros)
-            const float4 c01 = c01_next, c23 = c23_next;
-            c01_next = __ldg(reinterpret_cast<const float4 *>(flane + off + kEwmaTile));
-            c23_next = __ldg(reinterpret_cast<const float4 *>(flane + off + kEwmaTile) + 1);
+            const int col = tile * kTile + lane * 16;
+            // factors in pair order: (0,4,1,5) (2,6,3,7) of either chunk; zero past d_in
+            float4 cf[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) cf[i] = __ldg(flane + tile * 128 + 32 * i);
             issue_tile(tile + kEwmaStages - 1, (u + kEwmaStages - 1) & (kEwmaStages - 1));
             cp_async_wait<kEwmaStages - 1>();
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (in_row) v = my_ring[u * kSlot];
-            uint32_t p[4] = {v.x, v.y, v.z, v.w};
-            float2 L2[4];  // (L_j, L_{j+4}), binary32 with one rounding per multiplication
-            {
+            __syncwarp();  // the copies of this tile were made by other lanes
+            uint4 v[2];
+            v[0] = my_ring[u * kSlot + rpos_a];
+            v[1] = my_ring[u * kSlot + rpos_b];
+            bool in_row[2];
+            uint32_t p[2][4];
+            float2 L2[2][4];  // chunk x: (L_j, L_{j+4})
+            float2 acc[2];
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
+                in_row[x] = FULL || col + 8 * x < n;
+                if (!in_row[x]) v[x] = make_uint4(0u, 0u, 0u, 0u);
+                p[x][0] = v[x].x; p[x][1] = v[x].y; p[x][2] = v[x].z; p[x][3] = v[x].w;
                 float2 w2;
-                w2 = make_float2(unpack_lo<BF16>(p[0]), unpack_lo<BF16>(p[2]));
-                L2[0] = __fmul2_rn(__fmul2_rn(w2, w2), make_float2(c01.x, c01.y));
-                w2 = make_float2(unpack_hi<BF16>(p[0]), unpack_hi<BF16>(p[2]));
-                L2[1] = __fmul2_rn(__fmul2_rn(w2, w2), make_float2(c01.z, c01.w));
-                w2 = make_float2(unpack_lo<BF16>(p[1]), unpack_lo<BF16>(p[3]));
-                L2[2] = __fmul2_rn(__fmul2_rn(w2, w2), make_float2(c23.x, c23.y));
-                w2 = make_float2(unpack_hi<BF16>(p[1]), unpack_hi<BF16>(p[3]));
-                L2[3] = __fmul2_rn(__fmul2_rn(w2, w2), make_float2(c23.z, c23.w));
-            }
-            if constexpr (COUNT) {
+                w2 = make_float2(unpack_lo<BF16>(p[x][0]), unpack_lo<BF16>(p[x][2]));
+                L2[x][0] = __fmul2_rn(__fmul2_rn(w2, w2), make_float2(cf[2 * x].x, cf[2 * x].y));
+                w2 = make_float2(unpack_hi<BF16>(p[x][0]), unpack_hi<BF16>(p[x][2]));
+                L2[x][1] = __fmul2_rn(__fmul2_rn(w2, w2), make_float2(cf[2 * x].z, cf[2 * x].w));
+                w2 = make_float2(unpack_lo<BF16>(p[x][1]), unpack_lo<BF16>(p[x][3]));
+                L2[x][2] = __fmul2_rn(__fmul2_rn(w2, w2), make_float2(cf[2 * x + 1].x, cf[2 * x + 1].y));
+                w2 = make_float2(unpack_hi<BF16>(p[x][1]), unpack_hi<BF16>(p[x][3]));
+                L2[x][3] = __fmul2_rn(__fmul2_rn(w2, w2), make_float2(cf[2 * x + 1].z, cf[2 * x + 1].w));
+                if constexpr (COUNT) {
 #pragma unroll
-                for (int k = 0; k < 4; ++k) wmax = packed_abs_max<BF16>(wmax, p[k]);
-            }
-
-            // E: both chains from a zero state -> chain totals -> lane total -> scan over lanes.
-            float2 acc = L2[0];
+                    for (int k = 0; k < 4; ++k) wmax = packed_abs_max<BF16>(wmax, p[x][k]);
+                }
+                // E: the chunk's two chains from a zero state
+                acc[x] = L2[x][0];
 #pragma unroll
-            for (int j = 1; j < 4; ++j) acc = __ffma2_rn(a2, acc, L2[j]);
-            // (lane 0 adds a^8 times the state carried in, so the scanned values are true states)
+                for (int j = 1; j < 4; ++j) acc[x] = __ffma2_rn(a2, acc[x], L2[x][j]);
+            }
+            // chunk totals -> lane total (+ a^16 carry in lane 0) -> scan over lanes
+            const float tot_a = fmaf(a4, acc[0].x, acc[0].y), tot_b = fmaf(a4, acc[1].x, acc[1].y);
             float incl = lane_affine_scan_pred(
-                fmaf(a8_lane0, carry_E, fmaf(a4, acc.x, acc.y)), sc.a_step);
-            // one rotation hands every lane the state before its first element (the end state of
-            // the lane below) and lane 0 the end state of the tile, which it carries on
+                fmaf(a16_lane0, carry_E, fmaf(a8, tot_a, tot_b)), wc.a_step);
             float rot = __shfl_sync(kFullWarp, incl, lane_below);
-            float2 E2;
-            E2.x = is_lane0 ? carry_E : rot;  // E before element 0
-            E2.y = fmaf(a4, E2.x, acc.x);     // E before element 4
+            const float e0 = is_lane0 ? carry_E : rot;  // E before element 0
             carry_E = rot;
+            float2 E2[2];
+            E2[0].x = e0;
+            E2[0].y = fmaf(a4, e0, acc[0].x);           // before element 4
+            E2[1].x = fmaf(a8, e0, tot_a);              // before element 8
+            E2[1].y = fmaf(a4, E2[1].x, acc[1].x);      // before element 12
 
-            // q and the true E along both chains.
-            float2 q2[4];
+            float2 r2[2][4], dl[2];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                q2[j] = __ffma2_rn(neg_alpha2, E2, L2[j]);
-                E2 = __ffma2_rn(a2, E2, L2[j]);
-            }
-            // D' of both chains from a zero state, and the part of the decision value known now.
-            float2 r2[4];
-            r2[0] = q2[0];
-            r2[1].x = fmaf(kappa, fabsf(q2[0].x), q2[1].x);
-            r2[1].y = fmaf(kappa, fabsf(q2[0].y), q2[1].y);
-            float2 dl;
-            dl.x = fmaf(b, fabsf(q2[0].x), fabsf(q2[1].x));
-            dl.y = fmaf(b, fabsf(q2[0].y), fabsf(q2[1].y));
+            for (int x = 0; x < 2; ++x) {
+                float2 q2[4];
 #pragma unroll
-            for (int j = 2; j < 4; ++j) {
-                r2[j] = __ffma2_rn(make_float2(kappa, kappa), dl, q2[j]);
-                dl.x = fmaf(b, dl.x, fabsf(q2[j].x));
-                dl.y = fmaf(b, dl.y, fabsf(q2[j].y));
+                for (int j = 0; j < 4; ++j) {
+                    q2[j] = __ffma2_rn(neg_alpha2, E2[x], L2[x][j]);
+                    E2[x] = __ffma2_rn(a2, E2[x], L2[x][j]);
+                }
+                r2[x][0] = q2[0];
+                r2[x][1].x = fmaf(kappa, fabsf(q2[0].x), q2[1].x);
+                r2[x][1].y = fmaf(kappa, fabsf(q2[0].y), q2[1].y);
+                dl[x].x = fmaf(b, fabsf(q2[0].x), fabsf(q2[1].x));
+                dl[x].y = fmaf(b, fabsf(q2[0].y), fabsf(q2[1].y));
+#pragma unroll
+                for (int j = 2; j < 4; ++j) {
+                    r2[x][j] = __ffma2_rn(kappa2, dl[x], q2[j]);
+                    dl[x].x = fmaf(b, dl[x].x, fabsf(q2[j].x));
+                    dl[x].y = fmaf(b, dl[x].y, fabsf(q2[j].y));
+                }
             }
-            const float d_total = fmaf(b4, dl.x, dl.y);
-            incl = lane_affine_scan_pred(fmaf(b8_lane0, carry_D, d_total), sc.b_step);
+            const float dtot_a = fmaf(b4, dl[0].x, dl[0].y), dtot_b = fmaf(b4, dl[1].x, dl[1].y);
+            incl = lane_affine_scan_pred(
+                fmaf(b16_lane0, carry_D, fmaf(b8, dtot_a, dtot_b)), wc.b_step);
             rot = __shfl_sync(kFullWarp, incl, lane_below);
-            float2 D2;
-            D2.x = is_lane0 ? carry_D : rot;  // D' before element 0
-            D2.y = fmaf(b4, D2.x, dl.x);      // D' before element 4
+            const float d0 = is_lane0 ? carry_D : rot;  // D' before element 0
             carry_D = rot;
+            float2 D2[2];
+            D2[0].x = d0;
+            D2[0].y = fmaf(b4, d0, dl[0].x);
+            D2[1].x = fmaf(b8, d0, dtot_a);
+            D2[1].y = fmaf(b4, D2[1].x, dl[1].x);
 
-            // Decision values; their sign bits are the prune flags (a NaN is the positive
-            // canonical NaN: kept, as "L < threshold" is false).
-            float2 diff2[4];
+            uint32_t keep16 = 0;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) diff2[j] = __ffma2_rn(kappa_b2[j], D2, r2[j]);
-            uint32_t pm[4];
-            pm[0] = prmt(__float_as_uint(diff2[0].x), __float_as_uint(diff2[1].x), 0xffbbu);
-            pm[1] = prmt(__float_as_uint(diff2[2].x), __float_as_uint(diff2[3].x), 0xffbbu);
-            pm[2] = prmt(__float_as_uint(diff2[0].y), __float_as_uint(diff2[1].y), 0xffbbu);
-            pm[3] = prmt(__float_as_uint(diff2[2].y), __float_as_uint(diff2[3].y), 0xffbbu);
-            uint32_t keep8 = ~halfmasks_to_bits(pm) & 0xffu;
-            if (!in_row) keep8 = 0u;
-            if constexpr (COUNT) kept += __popc(keep8);
-
-            if (olane != nullptr && in_row) {
+            for (int x = 0; x < 2; ++x) {
+                // Decision values; their sign bits are the prune flags (a NaN is the positive
+                // canonical NaN: kept, as "L < threshold" is false).
+                float2 diff2[4];
 #pragma unroll
-                for (int k = 0; k < 4; ++k) p[k] &= ~pm[k];
-                __stcs(reinterpret_cast<uint4 *>(olane + off), make_uint4(p[0], p[1], p[2], p[3]));
+                for (int j = 0; j < 4; ++j) diff2[j] = __ffma2_rn(kappa_b2[j], D2[x], r2[x][j]);
+                uint32_t pm[4];
+                pm[0] = prmt(__float_as_uint(diff2[0].x), __float_as_uint(diff2[1].x), 0xffbbu);
+                pm[1] = prmt(__float_as_uint(diff2[2].x), __float_as_uint(diff2[3].x), 0xffbbu);
+                pm[2] = prmt(__float_as_uint(diff2[0].y), __float_as_uint(diff2[1].y), 0xffbbu);
+                pm[3] = prmt(__float_as_uint(diff2[2].y), __float_as_uint(diff2[3].y), 0xffbbu);
+                uint32_t keep8 = ~halfmasks_to_bits(pm) & 0xffu;
+                if (!in_row[x]) keep8 = 0u;
+                keep16 |= keep8 << (8 * x);
+                if (olane != nullptr && in_row[x]) {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) p[x][k] &= ~pm[k];
+                    __stcs(reinterpret_cast<uint4 *>(olane + tile * kTile + 8 * x),
+                           make_uint4(p[x][0], p[x][1], p[x][2], p[x][3]));
+                }
             }
-            // one mask byte per lane: byte k of a little-endian word holds columns 8k .. 8k+7
-            if (mlane != nullptr && (FULL || (off >> 3) + lane < mask_bytes))
-                mlane[off >> 3] = static_cast<uint8_t>(keep8);
+            if constexpr (COUNT) kept += __popc(keep16);
+            // two mask bytes per lane: a little-endian half word holds columns 16k .. 16k+15
+            if (mlane != nullptr && (FULL || tile * 32 + lane < mask_halves))
+                mlane[tile * 32] = static_cast<uint16_t>(keep16);
+            __syncwarp();  // all lanes have read this slot before it is refilled
         }
     }
 
@@ -658,13 +707,23 @@ sp_status launch_select_ewma(const sp_ctx *ctx, const void *W, sp_dtype dtype, i
         pc.kappa = static_cast<float>(kappa);
         for (int j = 0; j < 4; ++j) pc.kappa_b[j] = static_cast<float>(kappa * pow(b, j));
     }
-    const bool full = n % kEwmaTile == 0;
+    TileConstants wc;
+    for (int k = 0; k < 5; ++k) {
+        wc.a_step[k] = static_cast<float>(pow(static_cast<double>(sc.a), 16.0 * (1 << k)));
+        wc.b_step[k] = static_cast<float>(pow(static_cast<double>(sc.b), 16.0 * (1 << k)));
+    }
+    wc.a8 = sc.a_step[0];
+    wc.b8 = sc.b_step[0];
+    const bool full_tiles = n % 512 == 0;
+    PdlConfig pdlp(dim3(static_cast<unsigned>((n_rows + kPairWarps - 1) / kPairWarps)),
+                   dim3(kPairThreads), stream);
     const float *factor_pairs = ctx->factor_pairs;
 #define SP_LAUNCH_P(B, F, C)                                                                 \
-    launch_err = cudaLaunchKernelEx(&pdl.cfg, ewma_pair_scan_kernel<B, F, C>, Wp,            \
+    launch_err = cudaLaunchKernelEx(&pdlp.cfg, ewma_pair_scan_kernel<B, F, C>, Wp,            \
                                     static_cast<int>(ldw), static_cast<int>(n_rows),          \
-                                    static_cast<int>(n), factor_pairs, scalars, sc, pc, mask, \
-                                    static_cast<int>(words), Op, static_cast<int>(ldo), counters)
+                                    static_cast<int>(n), factor_pairs, scalars, sc, pc, wc,   \
+                                    mask, static_cast<int>(words), Op, static_cast<int>(ldo), \
+                                    counters)
 #define SP_LAUNCH_S(B, C)                                                                    \
     launch_err = cudaLaunchKernelEx(&pdl.cfg, ewma_scan_kernel<B, C>, Wp,              \
                                     static_cast<int>(ldw), static_cast<int>(n_rows),          \
@@ -673,7 +732,7 @@ sp_status launch_select_ewma(const sp_ctx *ctx, const void *W, sp_dtype dtype, i
 #define SP_LAUNCH_C(B, V, C)                                                                 \
     do {                                                                                     \
         if (V) {                                                                             \
-            if (full) SP_LAUNCH_P(B, true, C); else SP_LAUNCH_P(B, false, C);                \
+            if (full_tiles) SP_LAUNCH_P(B, true, C); else SP_LAUNCH_P(B, false, C);          \
         } else {                                                                             \
             SP_LAUNCH_S(B, C);                                                               \
         }                                                                                    \

@@ -55,7 +55,7 @@ struct sp_ctx {
     double *colsq;             // [n_pad]
     double *strip_sum;         // [strips]
     float *factor;             // [n_pad + 256] c_q, zero in the padding
-    float *factor_pairs;       // the same values with every chunk of 8 stored as 0,4,1,5,2,6,3,7
+    float *factor_pairs;       // the same values in the layout of the EWMA pair kernel (calib.cu)
     sp::DeviceScalars *scalars;
     sp::HostPipe *host_pipe;   // created by the first host-buffer call
 };

@@ -36,7 +36,7 @@ constexpr int kEwmaTile = 32 * kEwmaPerLane;      // weights per warp tile
 #define SP_EWMA_PAIR_THREADS 128
 #endif
 #ifndef SP_EWMA_PAIR_MIN_BLOCKS
-#define SP_EWMA_PAIR_MIN_BLOCKS 8
+#define SP_EWMA_PAIR_MIN_BLOCKS 7
 #endif
 constexpr int kPairThreads = SP_EWMA_PAIR_THREADS;
 constexpr int kPairWarps = kPairThreads / 32;
@@ -370,6 +370,9 @@ ewma_pair_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n
         carry_E = is_lane0 ? e : 0.0f;  // only lane 0's copy of the carried states is used
     }
 
+    float4 cf_next[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) cf_next[i] = __ldg(flane + 32 * i);
     for (int t0 = 0; t0 < tiles; t0 += kEwmaStages) {
 #pragma unroll
         for (int u = 0; u < kEwmaStages; ++u) {
@@ -379,7 +382,10 @@ ewma_pair_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n
             // factors in pair order: (0,4,1,5) (2,6,3,7) of either chunk; zero past d_in
             float4 cf[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) cf[i] = __ldg(flane + tile * 128 + 32 * i);
+            for (int i = 0; i < 4; ++i) {  // those of the next tile are requested now
+                cf[i] = cf_next[i];
+                cf_next[i] = __ldg(flane + (tile + 1) * 128 + 32 * i);  // padded by one tile
+            }
             issue_tile(tile + kEwmaStages - 1, (u + kEwmaStages - 1) & (kEwmaStages - 1));
             cp_async_wait<kEwmaStages - 1>();
             __syncwarp();  // the copies of this tile were made by other lanes

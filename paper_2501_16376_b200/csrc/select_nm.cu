@@ -5,8 +5,9 @@
 // per row), i.e. two groups of four or one group of eight: a group never straddles lanes, so
 // the selection needs no cross-lane traffic.  The 8 per-channel factors c_q of the lane's
 // columns are loaded once and stay in registers for the whole slab, and several rows are kept
-// in flight per lane: on the aligned path through a small per-lane ring in shared memory filled
-// by asynchronous copies (a lane only reads what it copied itself), otherwise in registers.
+// in flight per lane: in select_nm_stream_kernel (rows that allow 16-byte access) through a
+// small per-lane ring in shared memory filled by asynchronous copies (a lane only reads what it
+// copied itself), in select_nm_kernel (any other layout, element-wise access) in registers.
 //
 // Selection.  Scores are L = (w*w)*c_q in binary32 (Eq. 8); they are non-negative, so they are
 // compared through their bit patterns as unsigned integers, which also ranks NaN above every
@@ -28,22 +29,15 @@ namespace sp {
 #ifndef SP_NM_MIN_BLOCKS
 #define SP_NM_MIN_BLOCKS 8
 #endif
-#ifndef SP_NM_RING
-#define SP_NM_RING 4  // ring stages of the aligned path (0 = rows prefetched in registers)
-#endif
-#ifndef SP_NM_RING_UNROLL
-#define SP_NM_RING_UNROLL 4
-#endif
 #ifndef SP_NM_THREADS
 #define SP_NM_THREADS 128
 #endif
 constexpr int kNmThreads = SP_NM_THREADS;
 constexpr int kNmWarps = kNmThreads / 32;
 constexpr int kNmRowsInFlight = SP_NM_ROWS_IN_FLIGHT;
-constexpr int kNmRingUnroll = SP_NM_RING_UNROLL;
 
 // One row of one lane: score, rank, masks, write-back.  Returns the 8 keep bits.
-template <bool BF16, bool VEC, int M>
+template <bool BF16, int M>
 __device__ __forceinline__ uint32_t nm_process_row(uint32_t (&p)[4], const float (&c)[8],
                                                    uint32_t bias_lo, uint32_t bias_hi,
                                                    uint32_t valid, uint16_t *out_row, int64_t col,
@@ -68,12 +62,12 @@ __device__ __forceinline__ uint32_t nm_process_row(uint32_t (&p)[4], const float
     if (out_row != nullptr) {
 #pragma unroll
         for (int k = 0; k < 4; ++k) p[k] &= m[k];
-        store8<VEC>(out_row, col, n, p);
+        store8<false>(out_row, col, n, p);
     }
     return halfmasks_to_bits(m) & valid;
 }
 
-template <bool BF16, bool VEC, int M>
+template <bool BF16, int M>
 __global__ void __launch_bounds__(kNmThreads, SP_NM_MIN_BLOCKS)
 select_nm_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int64_t n,
                  int rows_per_warp, const float *__restrict__ factor, int prune_count,
@@ -107,48 +101,17 @@ select_nm_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int64_t n,
     uint32_t *mp = mask != nullptr ? mask + static_cast<int64_t>(row_begin) * mask_words + (col >> 5)
                                    : nullptr;
 
-#if SP_NM_RING
-    if constexpr (VEC) {
-        // rows streamed through a per-lane shared-memory ring with asynchronous copies
-        constexpr int kStages = SP_NM_RING;  // a power of two
-        __shared__ __align__(16) uint4 ring[kNmWarps * kStages * 32];
-        uint4 *my_ring = ring + (threadIdx.x >> 5) * kStages * 32 + lane;
-        const uint16_t *src = wp + (left > 0 ? col : 0);
-        auto issue = [&](int rr) {
-            if (rr < rows)
-                cp_async16(my_ring + (rr & (kStages - 1)) * 32, src + static_cast<int64_t>(rr) * ldw,
-                           left > 0 ? 16 : 0);
-            cp_async_commit();
-        };
-#pragma unroll
-        for (int rr = 0; rr < kStages - 1; ++rr) issue(rr);
-#pragma unroll kNmRingUnroll
-        for (int rr = 0; rr < rows; ++rr) {
-            issue(rr + kStages - 1);
-            cp_async_wait<kStages - 1>();
-            const uint4 v = my_ring[(rr & (kStages - 1)) * 32];
-            uint32_t p[4] = {v.x, v.y, v.z, v.w};
-            const uint32_t keep8 =
-                nm_process_row<BF16, VEC, M>(p, c, bias_lo, bias_hi, valid, op, col, n);
-            const uint32_t word = gather_mask_word(keep8, lane);
-            if (store_word) *mp = word;
-            if (op != nullptr) op += ldo;
-            if (mp != nullptr) mp += mask_words;
-        }
-        return;
-    }
-#endif
     int r = 0;
     for (; r + kNmRowsInFlight <= rows; r += kNmRowsInFlight) {
         uint32_t p[kNmRowsInFlight][4];
 #pragma unroll
         for (int u = 0; u < kNmRowsInFlight; ++u)
-            load8<VEC, true>(wp + static_cast<int64_t>(u) * ldw, col, n, p[u]);
+            load8<false, true>(wp + static_cast<int64_t>(u) * ldw, col, n, p[u]);
 #pragma unroll
         for (int u = 0; u < kNmRowsInFlight; ++u) {
             uint16_t *orow = op != nullptr ? op + static_cast<int64_t>(u) * ldo : nullptr;
             const uint32_t keep8 =
-                nm_process_row<BF16, VEC, M>(p[u], c, bias_lo, bias_hi, valid, orow, col, n);
+                nm_process_row<BF16, M>(p[u], c, bias_lo, bias_hi, valid, orow, col, n);
             const uint32_t word = gather_mask_word(keep8, lane);
             if (store_word) mp[static_cast<int64_t>(u) * mask_words] = word;
         }
@@ -158,14 +121,112 @@ select_nm_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int64_t n,
     }
     for (; r < rows; ++r) {  // fewer than kNmRowsInFlight rows left in the slab
         uint32_t p[4];
-        load8<VEC, true>(wp, col, n, p);
+        load8<false, true>(wp, col, n, p);
         const uint32_t keep8 =
-            nm_process_row<BF16, VEC, M>(p, c, bias_lo, bias_hi, valid, op, col, n);
+            nm_process_row<BF16, M>(p, c, bias_lo, bias_hi, valid, op, col, n);
         const uint32_t word = gather_mask_word(keep8, lane);
         if (store_word) *mp = word;
         wp += ldw;
         if (op != nullptr) op += ldo;
         if (mp != nullptr) mp += mask_words;
+    }
+}
+
+// Streaming kernel for rows that allow 16-byte access (the fast path).  Same work layout and
+// selection as select_nm_kernel; what differs is the bookkeeping around it: scores are formed
+// two at a time in packed binary32 pairs (mul.rn.f32x2, each half rounded like a scalar
+// product), the rows run through a four-slot per-lane ring whose slots are compile-time
+// constants (four rows per trip), every lane stores its own mask byte (byte k of a
+// little-endian mask word holds columns 8k .. 8k+7) instead of assembling words across lanes,
+// and when the strip is whole (FULL: d_in a multiple of 256) there are no column guards.
+template <bool BF16, bool FULL, int M>
+__global__ void __launch_bounds__(kNmThreads, SP_NM_MIN_BLOCKS)
+select_nm_stream_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
+                        int rows_per_warp, const float *__restrict__ factor, int prune_count,
+                        uint32_t *__restrict__ mask, int mask_words,
+                        uint16_t *__restrict__ W_out, int ldo) {
+    pdl_launch_dependents();
+    pdl_wait();  // the per-channel factors come from an earlier kernel of the stream
+    const int lane = threadIdx.x & 31;
+    const int col = blockIdx.x * kStripChannels + lane * 8;
+    const int slab = blockIdx.y * kNmWarps + (threadIdx.x >> 5);
+    const int64_t row_begin64 = static_cast<int64_t>(slab) * rows_per_warp;
+    if (row_begin64 >= n_rows) return;  // warp-uniform
+    const int row_begin = static_cast<int>(row_begin64);
+    const int rows = min(n_rows - row_begin, rows_per_warp);
+    const bool in_row = FULL || col < n;  // d_in % 8 == 0: a chunk is inside or outside as a whole
+
+    float2 cp[4];  // factors of columns (0,1) (2,3) (4,5) (6,7) of the chunk, zero past d_in
+    {
+        float c[8];
+        load_factor8(factor, col, c);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) cp[k] = make_float2(c[2 * k], c[2 * k + 1]);
+    }
+    // M == 4: rank bytes in two registers; M == 8: rank nibbles in one (see nm_rank.cuh)
+    const uint32_t bias =
+        M == 4 ? static_cast<uint32_t>(0x80 - prune_count) * 0x01010101u + 0x03020100u
+               : static_cast<uint32_t>(8 - prune_count) * 0x11111111u + 0x76543210u;
+
+    const uint16_t *src = W + static_cast<int64_t>(row_begin) * ldw + (in_row ? col : 0);
+    uint16_t *dst = W_out != nullptr && in_row
+                        ? W_out + static_cast<int64_t>(row_begin) * ldo + col
+                        : nullptr;
+    const int mask_pitch = mask_words * 4;  // bytes per mask row
+    uint8_t *mdst = mask != nullptr && (FULL || (col >> 3) < mask_pitch)
+                        ? reinterpret_cast<uint8_t *>(mask + static_cast<int64_t>(row_begin) * mask_words) + (col >> 3)
+                        : nullptr;
+
+    constexpr int kStages = 4;
+    __shared__ __align__(16) uint4 ring[kNmWarps * kStages * 32];
+    uint4 *my_ring = ring + (threadIdx.x >> 5) * kStages * 32 + lane;
+    auto issue = [&](int rr, int slot) {
+        if (rr < rows && in_row)
+            cp_async16(my_ring + slot * 32, src + static_cast<int64_t>(rr) * ldw, 16);
+        cp_async_commit();
+    };
+#pragma unroll
+    for (int rr = 0; rr < kStages - 1; ++rr) issue(rr, rr);
+
+    for (int r0 = 0; r0 < rows; r0 += kStages) {
+#pragma unroll
+        for (int u = 0; u < kStages; ++u) {
+            const int rr = r0 + u;
+            if (rr >= rows) break;  // warp-uniform
+            issue(rr + kStages - 1, (u + kStages - 1) & (kStages - 1));
+            cp_async_wait<kStages - 1>();
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (in_row) v = my_ring[u * 32];
+            uint32_t p[4] = {v.x, v.y, v.z, v.w};
+            uint32_t key[8];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float2 w2 = unpack2<BF16>(p[k]);
+                const float2 L2 = __fmul2_rn(__fmul2_rn(w2, w2), cp[k]);
+                key[2 * k] = __float_as_uint(L2.x);
+                key[2 * k + 1] = __float_as_uint(L2.y);
+            }
+            // half-word masks from the top bit of each rank field (sign replication)
+            uint32_t m[4];
+            if constexpr (M == 4) {
+                uint32_t ra, rb;
+                nm_rank_bytes<4>(key, bias, bias, ra, rb);
+                m[0] = prmt(ra, 0u, 0x9988u);
+                m[1] = prmt(ra, 0u, 0xbbaau);
+                m[2] = prmt(rb, 0u, 0x9988u);
+                m[3] = prmt(rb, 0u, 0xbbaau);
+            } else {
+                masks_from_nibbles(nm_rank_nibbles8(key, bias), m);
+            }
+            if (dst != nullptr) {
+                __stcs(reinterpret_cast<uint4 *>(dst + static_cast<int64_t>(rr) * ldo),
+                       make_uint4(p[0] & m[0], p[1] & m[1], p[2] & m[2], p[3] & m[3]));
+            }
+            if (mdst != nullptr) {
+                const uint32_t keep8 = in_row ? halfmasks_to_bits(m) & 0xffu : 0u;
+                mdst[static_cast<int64_t>(rr) * mask_pitch] = static_cast<uint8_t>(keep8);
+            }
+        }
     }
 }
 
@@ -202,20 +263,38 @@ sp_status launch_select_nm(const sp_ctx *ctx, const void *W, sp_dtype dtype, int
     PdlConfig pdl(grid, dim3(kNmThreads), stream);
     const float *factor = ctx->factor;
     cudaError_t launch_err = cudaSuccess;
-#define SP_LAUNCH(B, V, MM)                                                                  \
-    launch_err = cudaLaunchKernelEx(&pdl.cfg, select_nm_kernel<B, V, MM>, Wp,                 \
+#define SP_LAUNCH(B, MM)                                                                     \
+    launch_err = cudaLaunchKernelEx(&pdl.cfg, select_nm_kernel<B, MM>, Wp,                    \
                                     static_cast<int>(ldw), static_cast<int>(n_rows), n, rpw,  \
                                     factor, prune_count, mask, static_cast<int>(words), Op,   \
                                     static_cast<int>(ldo))
-#define SP_LAUNCH_M(B, V)                                                                     \
+#define SP_LAUNCH_M(B)                                                                        \
     do {                                                                                      \
-        if (M == 8) SP_LAUNCH(B, V, 8); else SP_LAUNCH(B, V, 4);                              \
+        if (M == 8) SP_LAUNCH(B, 8); else SP_LAUNCH(B, 4);                                    \
     } while (0)
-    if (dtype == SP_BF16) {
-        if (vec) SP_LAUNCH_M(true, true); else SP_LAUNCH_M(true, false);
+#define SP_LAUNCH_ST(B, F, MM)                                                               \
+    launch_err = cudaLaunchKernelEx(&pdl.cfg, select_nm_stream_kernel<B, F, MM>, Wp,          \
+                                    static_cast<int>(ldw), static_cast<int>(n_rows),          \
+                                    static_cast<int>(n), rpw, factor, prune_count, mask,      \
+                                    static_cast<int>(words), Op, static_cast<int>(ldo))
+#define SP_LAUNCH_STM(B, F)                                                                   \
+    do {                                                                                      \
+        if (M == 8) SP_LAUNCH_ST(B, F, 8); else SP_LAUNCH_ST(B, F, 4);                        \
+    } while (0)
+    const bool full = n % kStripChannels == 0;
+    if (vec) {
+        if (dtype == SP_BF16) {
+            if (full) SP_LAUNCH_STM(true, true); else SP_LAUNCH_STM(true, false);
+        } else {
+            if (full) SP_LAUNCH_STM(false, true); else SP_LAUNCH_STM(false, false);
+        }
+    } else if (dtype == SP_BF16) {
+        SP_LAUNCH_M(true);
     } else {
-        if (vec) SP_LAUNCH_M(false, true); else SP_LAUNCH_M(false, false);
+        SP_LAUNCH_M(false);
     }
+#undef SP_LAUNCH_STM
+#undef SP_LAUNCH_ST
 #undef SP_LAUNCH_M
 #undef SP_LAUNCH
     if (launch_err != cudaSuccess) return cuda_fail(launch_err);

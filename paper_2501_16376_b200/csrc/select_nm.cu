@@ -139,7 +139,8 @@ select_nm_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int64_t n,
 // constants (four rows per trip), every lane stores its own mask byte (byte k of a
 // little-endian mask word holds columns 8k .. 8k+7) instead of assembling words across lanes,
 // and when the strip is whole (FULL: d_in a multiple of 256) there are no column guards.
-template <bool BF16, bool FULL, int M>
+// OUT / MASK: the pruned weights / the keep mask are requested.
+template <bool BF16, bool FULL, int M, bool OUT, bool MASK>
 __global__ void __launch_bounds__(kNmThreads, SP_NM_MIN_BLOCKS)
 select_nm_stream_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
                         int rows_per_warp, const float *__restrict__ factor, int prune_count,
@@ -169,13 +170,12 @@ select_nm_stream_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int
                : static_cast<uint32_t>(8 - prune_count) * 0x11111111u + 0x76543210u;
 
     const uint16_t *src = W + static_cast<int64_t>(row_begin) * ldw + (in_row ? col : 0);
-    uint16_t *dst = W_out != nullptr && in_row
-                        ? W_out + static_cast<int64_t>(row_begin) * ldo + col
-                        : nullptr;
+    uint16_t *dst = OUT ? W_out + static_cast<int64_t>(row_begin) * ldo + (in_row ? col : 0) : nullptr;
     const int mask_pitch = mask_words * 4;  // bytes per mask row
-    uint8_t *mdst = mask != nullptr && (FULL || (col >> 3) < mask_pitch)
-                        ? reinterpret_cast<uint8_t *>(mask + static_cast<int64_t>(row_begin) * mask_words) + (col >> 3)
-                        : nullptr;
+    const bool in_mask = FULL || (col >> 3) < mask_pitch;
+    uint8_t *mdst = MASK ? reinterpret_cast<uint8_t *>(mask + static_cast<int64_t>(row_begin) * mask_words) +
+                               (in_mask ? col >> 3 : 0)
+                         : nullptr;
 
     constexpr int kStages = 4;
     __shared__ __align__(16) uint4 ring[kNmWarps * kStages * 32];
@@ -188,46 +188,48 @@ select_nm_stream_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int
 #pragma unroll
     for (int rr = 0; rr < kStages - 1; ++rr) issue(rr, rr);
 
-    for (int r0 = 0; r0 < rows; r0 += kStages) {
+    // One row of this lane: wait for its copy, score, rank, masks, write-back.
+    auto process = [&](int rr, int slot) {
+        issue(rr + kStages - 1, (slot + kStages - 1) & (kStages - 1));
+        cp_async_wait<kStages - 1>();
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (in_row) v = my_ring[slot * 32];
+        uint32_t p[4] = {v.x, v.y, v.z, v.w};
+        uint32_t key[8];
 #pragma unroll
-        for (int u = 0; u < kStages; ++u) {
-            const int rr = r0 + u;
-            if (rr >= rows) break;  // warp-uniform
-            issue(rr + kStages - 1, (u + kStages - 1) & (kStages - 1));
-            cp_async_wait<kStages - 1>();
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (in_row) v = my_ring[u * 32];
-            uint32_t p[4] = {v.x, v.y, v.z, v.w};
-            uint32_t key[8];
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const float2 w2 = unpack2<BF16>(p[k]);
-                const float2 L2 = __fmul2_rn(__fmul2_rn(w2, w2), cp[k]);
-                key[2 * k] = __float_as_uint(L2.x);
-                key[2 * k + 1] = __float_as_uint(L2.y);
-            }
-            // half-word masks from the top bit of each rank field (sign replication)
-            uint32_t m[4];
-            if constexpr (M == 4) {
-                uint32_t ra, rb;
-                nm_rank_bytes<4>(key, bias, bias, ra, rb);
-                m[0] = prmt(ra, 0u, 0x9988u);
-                m[1] = prmt(ra, 0u, 0xbbaau);
-                m[2] = prmt(rb, 0u, 0x9988u);
-                m[3] = prmt(rb, 0u, 0xbbaau);
-            } else {
-                masks_from_nibbles(nm_rank_nibbles8(key, bias), m);
-            }
-            if (dst != nullptr) {
-                __stcs(reinterpret_cast<uint4 *>(dst + static_cast<int64_t>(rr) * ldo),
-                       make_uint4(p[0] & m[0], p[1] & m[1], p[2] & m[2], p[3] & m[3]));
-            }
-            if (mdst != nullptr) {
-                const uint32_t keep8 = in_row ? halfmasks_to_bits(m) & 0xffu : 0u;
-                mdst[static_cast<int64_t>(rr) * mask_pitch] = static_cast<uint8_t>(keep8);
-            }
+        for (int k = 0; k < 4; ++k) {
+            const float2 w2 = unpack2<BF16>(p[k]);
+            const float2 L2 = __fmul2_rn(__fmul2_rn(w2, w2), cp[k]);
+            key[2 * k] = __float_as_uint(L2.x);
+            key[2 * k + 1] = __float_as_uint(L2.y);
         }
+        // half-word masks from the top bit of each rank field (sign replication)
+        uint32_t m[4];
+        if constexpr (M == 4) {
+            uint32_t ra, rb;
+            nm_rank_bytes<4>(key, bias, bias, ra, rb);
+            m[0] = prmt(ra, 0u, 0x9988u);
+            m[1] = prmt(ra, 0u, 0xbbaau);
+            m[2] = prmt(rb, 0u, 0x9988u);
+            m[3] = prmt(rb, 0u, 0xbbaau);
+        } else {
+            masks_from_nibbles(nm_rank_nibbles8(key, bias), m);
+        }
+        if (OUT && in_row) {
+            __stcs(reinterpret_cast<uint4 *>(dst + static_cast<int64_t>(rr) * ldo),
+                   make_uint4(p[0] & m[0], p[1] & m[1], p[2] & m[2], p[3] & m[3]));
+        }
+        if (MASK && in_mask) {
+            const uint32_t keep8 = in_row ? halfmasks_to_bits(m) & 0xffu : 0u;
+            mdst[static_cast<int64_t>(rr) * mask_pitch] = static_cast<uint8_t>(keep8);
+        }
+    };
+    int r0 = 0;
+    for (; r0 + kStages <= rows; r0 += kStages) {  // four rows per trip: static ring slots
+#pragma unroll
+        for (int u = 0; u < kStages; ++u) process(r0 + u, u);
     }
+    for (int rr = r0; rr < rows; ++rr) process(rr, rr & (kStages - 1));  // r0 % kStages == 0
 }
 
 sp_status launch_select_nm(const sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
@@ -272,14 +274,20 @@ sp_status launch_select_nm(const sp_ctx *ctx, const void *W, sp_dtype dtype, int
     do {                                                                                      \
         if (M == 8) SP_LAUNCH(B, 8); else SP_LAUNCH(B, 4);                                    \
     } while (0)
-#define SP_LAUNCH_ST(B, F, MM)                                                               \
-    launch_err = cudaLaunchKernelEx(&pdl.cfg, select_nm_stream_kernel<B, F, MM>, Wp,          \
+#define SP_LAUNCH_ST(B, F, MM, O, K)                                                         \
+    launch_err = cudaLaunchKernelEx(&pdl.cfg, select_nm_stream_kernel<B, F, MM, O, K>, Wp,    \
                                     static_cast<int>(ldw), static_cast<int>(n_rows),          \
                                     static_cast<int>(n), rpw, factor, prune_count, mask,      \
                                     static_cast<int>(words), Op, static_cast<int>(ldo))
+#define SP_LAUNCH_STO(B, F, MM)                                                               \
+    do {                                                                                      \
+        if (Op != nullptr && mask != nullptr) SP_LAUNCH_ST(B, F, MM, true, true);             \
+        else if (Op != nullptr) SP_LAUNCH_ST(B, F, MM, true, false);                          \
+        else SP_LAUNCH_ST(B, F, MM, false, true);                                             \
+    } while (0)
 #define SP_LAUNCH_STM(B, F)                                                                   \
     do {                                                                                      \
-        if (M == 8) SP_LAUNCH_ST(B, F, 8); else SP_LAUNCH_ST(B, F, 4);                        \
+        if (M == 8) SP_LAUNCH_STO(B, F, 8); else SP_LAUNCH_STO(B, F, 4);                      \
     } while (0)
     const bool full = n % kStripChannels == 0;
     if (vec) {
@@ -294,6 +302,7 @@ sp_status launch_select_nm(const sp_ctx *ctx, const void *W, sp_dtype dtype, int
         SP_LAUNCH_M(false);
     }
 #undef SP_LAUNCH_STM
+#undef SP_LAUNCH_STO
 #undef SP_LAUNCH_ST
 #undef SP_LAUNCH_M
 #undef SP_LAUNCH

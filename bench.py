@@ -43,9 +43,10 @@ CALIB_BYTES_PER_ELEMENT = 2.0
 # Valid for the kernels as committed with that capture; other shapes report null.
 NCU_CALIB_TRAFFIC = {4096: 269.85e6, 11008: 722.67e6, 14336: 941.03e6}
 NCU_SELECT_TRAFFIC = {
-    "select_nm_kernel": {(4096, 4096): 33.68e6, (11008, 4096): 131.77e6, (4096, 11008): 131.10e6},
-    "ewma_pair_scan_kernel": {(4096, 4096): 34.5e6, (1024, 4096): 8.42e6,
-                              (14336, 4096): 189.1e6, (4096, 14336): 191.2e6},
+    "select_nm_stream_kernel": {(4096, 4096): 34.3e6, (11008, 4096): 132.7e6,
+                                (4096, 11008): 133.0e6},
+    "ewma_pair_scan_kernel": {(4096, 4096): 34.1e6, (1024, 4096): 8.43e6,
+                              (14336, 4096): 187.3e6, (4096, 14336): 188.0e6},
 }
 
 
@@ -323,7 +324,7 @@ def gpu_arm(args):
     if batch_tokens == 32768 and w.tokens % batch_tokens == 0 and \
             all(d in NCU_CALIB_TRAFFIC for d in widths):
         calib_traffic = sum(NCU_CALIB_TRAFFIC[d] for d in widths) / len(widths)
-    sel_kernel = "select_nm_kernel" if w.mode == "nm" else "ewma_pair_scan_kernel"
+    sel_kernel = "select_nm_stream_kernel" if w.mode == "nm" else "ewma_pair_scan_kernel"
     sel_traffic = None
     shapes = [(l.d_out, l.d_in) for l in w.layers]
     table = NCU_SELECT_TRAFFIC[sel_kernel]

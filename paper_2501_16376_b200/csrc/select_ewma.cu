@@ -15,9 +15,10 @@
 // path: packed binary32 pairs, weights streamed through a shared-memory ring of asynchronous
 // copies) and ewma_scan_kernel for any other pointer, stride or width.
 //
-// Literal-S path (sequential kernel).  Algorithm 1's "S = S - w_i^2" makes L_i depend on
-// earlier decisions, so the row is evaluated in order by one thread, every operation in
-// binary32 with one rounding each.  It is a correctness path, not a fast one.
+// Literal-S path (sequential kernels, here and in select_ewma_tiled.cu).  Algorithm 1's
+// "S = S - w_i^2" makes L_i depend on earlier decisions, so the row is evaluated in order by one
+// thread, every operation in binary32 with one rounding each.  It is the exact path, bound by
+// the latency of one dependent chain per row.
 #include <math.h>
 
 #include "sp_device.cuh"
@@ -512,11 +513,12 @@ ewma_pair_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n
 }
 
 // Algorithm 1 exactly as printed, one thread per row, binary32 with one rounding per operation.
-// The row is read and written in chunks of 8 weights (16 bytes when aligned).  While S still
+// Element-wise access with bounds checks: the path for rows that do not allow 16-byte access
+// (ewma_literal_tiled_kernel handles those that do).  While S still
 // has its initial value the per-channel factor computed at finalisation is used: it was formed
 // by the same three operations from the same S, so the result is bit-identical to recomputing
 // it; once a pruned weight has changed S the factor is recomputed for every element.
-template <bool BF16, bool VEC>
+template <bool BF16>
 __global__ void __launch_bounds__(128)
 ewma_literal_kernel(const uint16_t *__restrict__ W, int64_t ldw, int64_t n_rows, int64_t n,
                     const double *__restrict__ colsq, const float *__restrict__ factor,
@@ -538,8 +540,8 @@ ewma_literal_kernel(const uint16_t *__restrict__ W, int64_t ldw, int64_t n_rows,
     unsigned long long kept = 0;
     // two chunks are kept in flight ahead of the one being evaluated
     uint32_t ahead[2][4];
-    load8<VEC, true>(wrow, 0, n, ahead[0]);
-    load8<VEC, true>(wrow, 8, n, ahead[1]);
+    load8<false, true>(wrow, 0, n, ahead[0]);
+    load8<false, true>(wrow, 8, n, ahead[1]);
     for (int64_t i0 = 0; i0 < n; i0 += 8) {
         uint32_t p[4];
 #pragma unroll
@@ -547,7 +549,7 @@ ewma_literal_kernel(const uint16_t *__restrict__ W, int64_t ldw, int64_t n_rows,
             p[k] = ahead[0][k];
             ahead[0][k] = ahead[1][k];
         }
-        load8<VEC, true>(wrow, i0 + 16, n, ahead[1]);
+        load8<false, true>(wrow, i0 + 16, n, ahead[1]);
         float w[8];
         unpack8<BF16>(p, w);
         uint32_t keep8 = 0;
@@ -579,7 +581,7 @@ ewma_literal_kernel(const uint16_t *__restrict__ W, int64_t ldw, int64_t n_rows,
         kept += __popc(keep8);
         if (orow != nullptr) {
             zero_pruned(p, keep8);
-            store8<VEC>(orow, i0, n, p);
+            store8<false>(orow, i0, n, p);
         }
         word |= keep8 << (i0 & 31);
         if ((i0 & 31) == 24 || i0 + 8 >= n) {
@@ -679,16 +681,15 @@ sp_status launch_select_ewma(const sp_ctx *ctx, const void *W, sp_dtype dtype, i
         if (blocks > 0x7fffffffLL) return SP_ERR_SHAPE;
         const bool lvec = aligned16(W) && ldw % 8 == 0 && n % 8 == 0 &&
                           (W_out == nullptr || (aligned16(W_out) && ldo % 8 == 0));
+        if (lvec)  // rows that allow 16-byte access: the same arithmetic, rows moved in tiles
+            return launch_ewma_literal_tiled(ctx, W, dtype, n_rows, ldw, p, mask, W_out, ldo,
+                                             counters, stream);
         const unsigned lgrid = static_cast<unsigned>(blocks);
-#define SP_LAUNCH_L(B, V)                                                                    \
-    ewma_literal_kernel<B, V><<<lgrid, 128, 0, stream>>>(                                    \
+#define SP_LAUNCH_L(B)                                                                       \
+    ewma_literal_kernel<B><<<lgrid, 128, 0, stream>>>(                                       \
         Wp, ldw, n_rows, n, ctx->colsq, ctx->factor, ctx->scalars, p.alpha, p.beta, p.la, mask, \
         words, Op, ldo, counters)
-        if (bf16) {
-            if (lvec) SP_LAUNCH_L(true, true); else SP_LAUNCH_L(true, false);
-        } else {
-            if (lvec) SP_LAUNCH_L(false, true); else SP_LAUNCH_L(false, false);
-        }
+        if (bf16) SP_LAUNCH_L(true); else SP_LAUNCH_L(false);
 #undef SP_LAUNCH_L
         return check_launch();
     }

@@ -104,6 +104,12 @@ sp_status launch_select_ewma(const sp_ctx *ctx, const void *W, sp_dtype dtype, i
                              int64_t ldw, const sp_ewma_params &p, uint32_t *mask, void *W_out,
                              int64_t ldo, unsigned long long *counters, cudaStream_t stream);
 
+// select_ewma_tiled.cu
+sp_status launch_ewma_literal_tiled(const sp_ctx *ctx, const void *W, sp_dtype dtype,
+                                    int64_t n_rows, int64_t ldw, const sp_ewma_params &p,
+                                    uint32_t *mask, void *W_out, int64_t ldo,
+                                    unsigned long long *counters, cudaStream_t stream);
+
 // host_pipe.cu
 void host_pipe_destroy(HostPipe *hp);
 sp_status host_calib_accumulate(sp_ctx *ctx, const void *X_host, sp_dtype dtype, int64_t n_tokens,

@@ -53,6 +53,11 @@ def test_nm_stream_kernel_on_partial_strips(sp, n, dtype):
                                          torch.cuda.current_stream().cuda_stream)
                 assert st == sp.SP_OK
                 assert np.array_equal(P.mask_np(mask_only), P.mask_np(mask))
+                if (N, M) == (2, 4):  # the same selection, emitted as values + index records
+                    values, meta = ctx.sp_select_24_compressed(W_ref)
+                    v, m = so.compress_24(P.bits(W_ref), sel.keep_bool(n))
+                    assert np.array_equal(P.bits(values), v)
+                    assert np.array_equal(P.mask_np(meta), m)
 
 @pytest.mark.parametrize("n", WIDTHS)
 @pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])

@@ -66,8 +66,7 @@ def parse_args():
                     help="which of the workload's sparsities / N:M patterns to run")
     ap.add_argument("--graph", action="store_true",
                     help="replay the whole-model pass as one CUDA graph in the timed region "
-                         "(for launch-bound small models); the per-kernel breakdown then comes "
-                         "from one instrumented pass after it")
+                         "(for launch-bound small models)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
 
@@ -292,18 +291,21 @@ def gpu_arm(args):
     else:
         counts = None
         for _ in range(args.steps):
-            counts = pipeline.prune_model(mb, arg, batch_tokens, phase_events)
+            counts = pipeline.prune_model(mb, arg, batch_tokens)
     stop.record()
     barrier()
+    clocks = sampler.stop()
     elapsed_ms = start.elapsed_time(stop)
     if graph is not None:
         launches = sum(counts.values()) * args.steps
-        for _ in range(args.steps):        # instrumented passes, outside the timed region
-            pipeline.prune_model(mb, arg, batch_tokens, phase_events)
-        torch.cuda.synchronize()
     else:
         launches = sp.sp_launch_count() - launches_before
-    clocks = sampler.stop()
+    # The per-phase breakdown and the per-kernel rates come from instrumented passes after the
+    # timed region: the event records between phases would otherwise sit inside it (they keep a
+    # kernel from overlapping the tail of its predecessor).
+    for _ in range(args.steps):
+        pipeline.prune_model(mb, arg, batch_tokens, phase_events)
+    torch.cuda.synchronize()
 
     elapsed_ms = sharding.max_over_ranks(elapsed_ms, world, device)
     total_weights = w.total_weights() * world
@@ -366,6 +368,9 @@ def gpu_arm(args):
                                 "finalize": final_ms / args.steps * 1e-3,
                                 "select_apply": select_ms / args.steps * 1e-3,
                                 "total": elapsed_ms / args.steps * 1e-3},
+        "phase_note": "calib / finalize / select_apply are event brackets from instrumented passes "
+                      "run after the timed region (the brackets stop kernels from overlapping "
+                      "their predecessors' tails); total is the timed region",
         "roofline": roofline, "roofline_select": roofline_select,
         "clocks": clocks, "gpu_launches": int(launches),
     }

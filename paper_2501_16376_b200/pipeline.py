@@ -93,8 +93,10 @@ def prune_model(mb: ModelBuffers, mode_arg, batch_tokens: int, phase_events=None
     layer that reads this input.  phase_events, if given, is a list that receives
     (kind, start_event, end_event, units) tuples per layer input: "calib" (units = activation
     elements, brackets its back-to-back accumulate launches), "finalize", and "select" (units =
-    weights, brackets the back-to-back selection launches of the layers reading this input).
-    Returns launch counts."""
+    weights, brackets the back-to-back selection launches of the layers reading this input);
+    with phase_events the calls are issued strictly input by input so that the brackets are
+    clean, without it the next input's calibration is enqueued ahead of the current input's
+    selections (same calls, same results).  Returns launch counts."""
     w = mb.workload
     n_calib = n_select = n_final = 0
 
@@ -103,32 +105,54 @@ def prune_model(mb: ModelBuffers, mode_arg, batch_tokens: int, phase_events=None
         e.record(stream)
         return e
 
-    last = mark() if phase_events is not None else None
+    def select_input(b, name, ctx):
+        nonlocal n_select
+        weights = 0
+        for li, layer in enumerate(w.layers):
+            if layer.input != name:
+                continue
+            select_layer(ctx, w, mb.weights[b][li], mb.masks[b][li], mb.outputs[b][li],
+                         mode_arg, stream)
+            n_select += 1
+            weights += layer.d_out * layer.d_in
+        return weights
+
+    if phase_events is None:
+        # Plain pass.  The calibration of the next input is enqueued between an input's
+        # finalisation and its selections: the accumulate kernel only waits for its predecessor
+        # before it writes its partial sums, so it streams its activations while the few CTAs
+        # of the finalisation run (inputs of different widths have different contexts; with a
+        # single input the order is simply calibrate, finalise, select).
+        units = [(b, name) for b in range(w.blocks) for name in w.input_widths()]
+        distinct = len(w.input_widths()) > 1
+        for i, (b, name) in enumerate(units):
+            ctx = mb.ctxs[name]
+            if i == 0 or not distinct:
+                n_calib += calibrate_input(ctx, mb.acts[name], batch_tokens, stream)
+            ctx.sp_score(None, stream=stream)          # finalisation only
+            n_final += 1
+            if distinct and i + 1 < len(units):
+                nxt = units[i + 1][1]
+                n_calib += calibrate_input(mb.ctxs[nxt], mb.acts[nxt], batch_tokens, stream)
+            select_input(b, name, ctx)
+        return {"calib": n_calib, "finalize": n_final, "select": n_select}
+
+    last = mark()
     for b in range(w.blocks):
         for name, d_in in w.input_widths().items():
             ctx = mb.ctxs[name]
             X = mb.acts[name]
             e0 = last
             n_calib += calibrate_input(ctx, X, batch_tokens, stream)
-            if phase_events is not None:
-                e1 = mark()
+            e1 = mark()
             ctx.sp_score(None, stream=stream)          # finalisation only
             n_final += 1
-            if phase_events is not None:
-                e2 = mark()
-                phase_events.append(("calib", e0, e1, X.shape[0] * d_in))
-                phase_events.append(("finalize", e1, e2, d_in))
-            sel_weights = 0
-            for li, layer in enumerate(w.layers):
-                if layer.input != name:
-                    continue
-                select_layer(ctx, w, mb.weights[b][li], mb.masks[b][li], mb.outputs[b][li],
-                             mode_arg, stream)
-                n_select += 1
-                sel_weights += layer.d_out * layer.d_in
-            if phase_events is not None:
-                last = mark()
-                phase_events.append(("select", e2, last, sel_weights))
+            e2 = mark()
+            phase_events.append(("calib", e0, e1, X.shape[0] * d_in))
+            phase_events.append(("finalize", e1, e2, d_in))
+            sel_weights = select_input(b, name, ctx)
+            last = mark()
+            phase_events.append(("select", e2, last, sel_weights))
     return {"calib": n_calib, "finalize": n_final, "select": n_select}
 
 

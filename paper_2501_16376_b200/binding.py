@@ -114,7 +114,7 @@ def _matrix(t: torch.Tensor, what: str, host: bool = False):
 
 def _stream(stream) -> int:
     if stream is None:
-        stream = torch.cuda.current_stream()
+        return torch._C._cuda_getCurrentRawStream(torch.cuda.current_device())
     return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
 
 

@@ -99,6 +99,8 @@ def prune_model(mb: ModelBuffers, mode_arg, batch_tokens: int, phase_events=None
     selections (same calls, same results).  Returns launch counts."""
     w = mb.workload
     n_calib = n_select = n_final = 0
+    if stream is None:
+        stream = torch.cuda.current_stream()   # looked up once, not once per call
 
     def mark():
         e = torch.cuda.Event(enable_timing=True)

@@ -350,6 +350,31 @@ def gpu_arm(args):
                 "while the kernel runs (part of the output is still in L2 when it ends)",
     }
 
+    # The same select kernel timed alone on the largest layer shape: back-to-back launches over
+    # every block's own weights / outputs (distinct buffers, far more than L2), statistics in place.
+    li = max(range(len(w.layers)), key=lambda i: w.layers[i].d_out * w.layers[i].d_in)
+    big = w.layers[li]
+    if w.blocks * big.d_out * big.d_in * 4 > 256e6:
+        ctx_big = mb.ctxs[big.input]
+        t0 = torch.cuda.Event(enable_timing=True)
+        t1 = torch.cuda.Event(enable_timing=True)
+        for rep in range(2):   # the first repetition warms up
+            t0.record()
+            for b in range(w.blocks):
+                pipeline.select_layer(ctx_big, w, mb.weights[b][li], mb.masks[b][li],
+                                      mb.outputs[b][li], arg)
+            t1.record()
+            torch.cuda.synchronize()
+        alone_ms = t0.elapsed_time(t1) / w.blocks
+        alone_gbs = SELECT_BYTES_PER_WEIGHT * big.d_out * big.d_in / (alone_ms * 1e-3) / 1e9
+        roofline_select["alone"] = {
+            "layer": "%dx%d" % (big.d_out, big.d_in), "launches": w.blocks,
+            "avg_launch_ms": alone_ms, "achieved": alone_gbs, "frac": alone_gbs / peak,
+            "frac_of_8TBs": alone_gbs / 8000.0,
+            "note": "select launches only, back to back over all blocks (no calibration traffic "
+                    "in between, so the SM clock is not held down by the power cap)",
+        }
+
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": elapsed_ms / args.steps,

@@ -22,7 +22,8 @@
 
 namespace sp {
 
-// Tuning knobs (compile-time): rows kept in flight per lane, resident CTAs per SM asked of ptxas.
+// Tuning knobs (compile-time): rows kept in flight per lane (general kernel), resident CTAs per
+// SM asked of ptxas, the fewest rows a warp gets and the warps per SM the launcher aims for.
 #ifndef SP_NM_ROWS_IN_FLIGHT
 #define SP_NM_ROWS_IN_FLIGHT 4
 #endif

@@ -11,6 +11,8 @@
 // loads.  The walk is one dependent chain per row (about 25 instructions per weight, each
 // waiting for the one before it): with a few thousand rows there is at most one warp per
 // scheduler to run, so the kernel is bound by instruction latency, not by memory.
+#include <type_traits>
+
 #include "sp_device.cuh"
 #include "sp_internal.h"
 
@@ -87,28 +89,48 @@ ewma_literal_tiled_kernel(const uint16_t *__restrict__ W, int64_t ldw, int n_row
             const float4 c0 = __ldg(reinterpret_cast<const float4 *>(factor + i0));
             const float4 c1 = __ldg(reinterpret_cast<const float4 *>(factor + i0) + 1);
             const float cf[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
-            uint32_t keep8 = 0;
+            // The 8 elements of the chunk, in order.  FOLLOW_S: recompute the factor of an
+            // element from the current S once a pruned weight has changed it (a lane whose S
+            // still has its initial value keeps the finalised factor, which is the same three
+            // operations on the same operands).
+            uint32_t keep8;
+            auto walk = [&](auto follow_s) {
+                keep8 = 0;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                float c = cf[j];
-                // Once a pruned weight has changed S the factor follows it.  The test is made
-                // warp-wide so that the usual case (no lane's S has moved) takes no divergent
-                // branch; a lane whose S still has its initial value recomputes the identical
-                // factor (same three operations on the same operands).
-                if (__any_sync(kFullWarp, S != S0)) {
-                    const float u = __fdiv_rn(static_cast<float>(colsq[i0 + j]), S);
-                    c = __fdiv_rn(0.5f, __fsub_rn(1.0f, u));
+                for (int j = 0; j < 8; ++j) {
+                    float c = cf[j];
+                    if (decltype(follow_s)::value) {
+                        if (S != S0) {
+                            const float u = __fdiv_rn(static_cast<float>(colsq[i0 + j]), S);
+                            c = __fdiv_rn(0.5f, __fsub_rn(1.0f, u));
+                        }
+                    }
+                    const float w2 = __fmul_rn(w[j], w[j]);
+                    const float L = __fmul_rn(w2, c);
+                    if (k == 0 && j == 0 && tile == 0) est = L;
+                    const float thr = __fsub_rn(est, __fmul_rn(la, dev));
+                    const bool prune = L < thr;
+                    S = prune ? __fsub_rn(S, w2) : S;
+                    keep8 |= prune ? 0u : 1u << j;
+                    est = __fadd_rn(__fmul_rn(one_minus_alpha, est), __fmul_rn(alpha, L));
+                    dev = __fadd_rn(__fmul_rn(one_minus_beta, dev),
+                                    __fmul_rn(beta, fabsf(__fsub_rn(est, L))));
                 }
-                const float w2 = __fmul_rn(w[j], w[j]);
-                const float L = __fmul_rn(w2, c);
-                if (k == 0 && j == 0 && tile == 0) est = L;
-                const float thr = __fsub_rn(est, __fmul_rn(la, dev));
-                const bool prune = L < thr;
-                S = prune ? __fsub_rn(S, w2) : S;
-                keep8 |= prune ? 0u : 1u << j;
-                est = __fadd_rn(__fmul_rn(one_minus_alpha, est), __fmul_rn(alpha, L));
-                dev = __fadd_rn(__fmul_rn(one_minus_beta, dev),
-                                __fmul_rn(beta, fabsf(__fsub_rn(est, L))));
+            };
+            // Usual case: no lane's S has moved, and none moves inside the chunk - the chunk is
+            // straight-line code with the finalised factors.  Otherwise the chunk is walked
+            // (again) from the state it started in, following S element by element.
+            const float est_in = est, dev_in = dev, S_in = S;
+            bool follow = __any_sync(kFullWarp, S_in != S0);
+            if (!follow) {
+                walk(std::false_type{});
+                follow = __any_sync(kFullWarp, S != S_in);
+            }
+            if (follow) {
+                est = est_in;
+                dev = dev_in;
+                S = S_in;
+                walk(std::true_type{});
             }
             word |= keep8 << (8 * k);
             if (dst != nullptr) {

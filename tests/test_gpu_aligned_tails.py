@@ -87,3 +87,22 @@ def test_ewma_pair_kernel_on_partial_tiles(sp, n, dtype):
                 assert not (words[:, -1] >> np.uint32(n % 32)).any()
             if counters is not None:
                 assert int(counters[sp.SP_COUNTER_KEPT]) == int(keep.sum())
+
+
+@pytest.mark.parametrize("alpha,beta", [(1.0, 1.0), (1.0, 0.125), (0.01, 0.02), (0.5, 0.03125)])
+def test_ewma_pair_kernel_parameter_extremes(sp, alpha, beta):
+    # a = 1 - alpha = 0 makes every power in the lane scans vanish; a small alpha gives the state
+    # a memory of hundreds of columns, i.e. many tiles
+    R, n = 24, 2048
+    W, colsq = _inputs(4242, R, n, torch.bfloat16)
+    for la in (0.5, -0.9):
+        with sp.Context(n) as ctx:
+            ctx.sp_set_stats(torch.from_numpy(colsq), 5)
+            mask, out = ctx.sp_select_unstructured(W, params=sp.EwmaParams(alpha, beta, la, 0))
+            sel = so.select_ewma(P.bits(W), P.odtype(W), so.Stats(colsq.copy(), 5), la, alpha, beta,
+                                 s_update=so.S_FROZEN, want_trace=True)
+            keep = so.unpack_mask(P.mask_np(mask), n)
+            diff = keep != sel.keep_bool(n)
+            assert not (diff & ~P.ewma_allowed_flips(sel)).any()
+            assert diff.sum() <= 1
+            assert np.array_equal(P.bits(out), np.where(keep, P.bits(W), 0))

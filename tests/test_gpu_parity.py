@@ -467,6 +467,33 @@ def test_la_search_matches_oracle_bisection(sp, target):
         assert abs((1.0 - keep.mean()) - achieved) < 1e-12
 
 
+# ------------------------------------------------------------------ token-sharded calibration
+
+def test_token_shards_merge_into_the_statistics_of_all_tokens(sp):
+    # what two ranks that each saw half the tokens would do, in one process: the column sums of
+    # squares add up, so the merged context selects exactly like one that saw every token
+    from paper_2501_16376_b200 import sharding
+    n, T = 1024, 4096
+    X = _activations(77, T, n, torch.float16)
+    W = _gen(78, (64, n), torch.float16, 0.02)
+    with sp.Context(n) as whole, sp.Context(n) as a, sp.Context(n) as b:
+        whole.sp_calib_accumulate(X)
+        a.sp_calib_accumulate(X[:T // 2])
+        b.sp_calib_accumulate(X[T // 2:])
+        ca, _, _, ta = a.sp_get_stats()
+        cb, _, _, tb = b.sp_get_stats()
+        a.sp_set_stats(ca + cb, ta + tb)                    # the all-reduce, written out
+        assert sharding.merge_calibration(b, world=1) == T // 2   # one rank: nothing to add
+        cw, Sw, fw, tw = whole.sp_get_stats()
+        cm, Sm, fm, tm = a.sp_get_stats()
+        assert tm == tw == T
+        assert torch.allclose(cm, cw, rtol=1e-13, atol=0.0)
+        assert abs(Sm - Sw) <= 1e-12 * Sw
+        m1, o1 = whole.sp_select_nm(W, 2, 4)
+        m2, o2 = a.sp_select_nm(W, 2, 4)
+        assert torch.equal(m1, m2) and torch.equal(o1, o2)
+
+
 # ------------------------------------------------------------------ CUDA graph capture
 
 def test_whole_pass_can_be_captured_and_replayed_as_a_cuda_graph(sp):

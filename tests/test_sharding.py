@@ -41,8 +41,11 @@ def _worker(rank, world, port, out):
         blocks = list(sharding.assign_units(7, world, rank))
         gathered = [None] * world
         dist.all_gather_object(gathered, blocks)
+        # token-sharded calibration: per-rank column sums of squares add up
+        colsq = torch.arange(5, dtype=torch.float64) * (rank + 1) + 0.25
+        merged, tokens = sharding.allreduce_colsq(colsq, 100 + rank, world)
         if rank == 0:
-            out.put((slowest, total, gathered))
+            out.put((slowest, total, gathered, merged.tolist(), tokens))
     finally:
         dist.destroy_process_group()
 
@@ -54,16 +57,23 @@ def test_two_gloo_ranks_reduce_timing_and_partition_units():
     procs = [ctx.Process(target=_worker, args=(r, 2, port, out)) for r in range(2)]
     for p in procs:
         p.start()
-    slowest, total, gathered = out.get(timeout=120)
+    slowest, total, gathered, merged, tokens = out.get(timeout=120)
     for p in procs:
         p.join(timeout=120)
         assert p.exitcode == 0
     assert slowest == 15.0                 # value = total work / slowest rank's time
     assert total == 3000.0
     assert gathered == [[0, 1, 2, 3], [4, 5, 6]]
+    assert merged == [0.5 + 3.0 * k for k in range(5)]     # (k + 0.25) + (2k + 0.25)
+    assert tokens == 201
 
 
 def test_single_process_reductions_are_identity():
     assert sharding.max_over_ranks(3.5, 1) == 3.5
     assert sharding.sum_over_ranks(3.5, 1) == 3.5
     assert sharding.unit_of_rank(0, 1) == 0
+    c = torch.tensor([1.0, 2.0], dtype=torch.float64)
+    merged, tokens = sharding.allreduce_colsq(c, 7, 1)
+    assert merged.tolist() == [1.0, 2.0] and tokens == 7
+    with pytest.raises(ValueError):
+        sharding.allreduce_colsq(c.float(), 7, 1)

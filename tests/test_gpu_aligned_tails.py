@@ -106,3 +106,45 @@ def test_ewma_pair_kernel_parameter_extremes(sp, alpha, beta):
             assert not (diff & ~P.ewma_allowed_flips(sel)).any()
             assert diff.sum() <= 1
             assert np.array_equal(P.bits(out), np.where(keep, P.bits(W), 0))
+
+
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+def test_fast_kernels_with_padded_row_strides(sp, dtype):
+    # rows that allow 16-byte access but are not contiguous: input and output are column slices of
+    # wider matrices with different (aligned) leading dimensions
+    R, n = 37, 1032
+    g = torch.Generator(device="cuda").manual_seed(99)
+    big_in = (torch.randn(R, n + 24, generator=g, device="cuda") * 0.02).to(dtype)
+    W = big_in[:, 8:8 + n]
+    big_out = torch.full((R, n + 40), 7.0, device="cuda").to(dtype)
+    W_out = big_out[:, 16:16 + n]
+    assert W.data_ptr() % 16 == 0 and W_out.data_ptr() % 16 == 0
+    rng = np.random.default_rng(5)
+    colsq = rng.uniform(0.5, 2.0, n) * 1e4
+    W_ref = W.clone()
+    with sp.Context(n) as ctx:
+        ctx.sp_set_stats(torch.from_numpy(colsq), 5)
+        st = so.Stats(colsq.copy(), 5)
+        mask, out = ctx.sp_select_nm(W, 2, 4, W_out=W_out)
+        sel = so.select_nm(P.bits(W_ref), P.odtype(W_ref), st, 2, 4)
+        P.check_selection(mask, out, W_ref, sel, None, strict=True)
+        values, meta = ctx.sp_select_24_compressed(W)
+        v, m = so.compress_24(P.bits(W_ref), sel.keep_bool(n))
+        assert np.array_equal(P.bits(values), v) and np.array_equal(P.mask_np(meta), m)
+        for literal in (0, 1):
+            big_out.fill_(7.0)
+            mask, out = ctx.sp_select_unstructured(W, params=sp.EwmaParams(0.125, 0.125, 0.5, literal),
+                                                   W_out=W_out)
+            sel = so.select_ewma(P.bits(W_ref), P.odtype(W_ref), st, 0.5, 0.125, 0.125,
+                                 s_update=so.S_LITERAL_W2 if literal else so.S_FROZEN,
+                                 want_trace=True)
+            keep = so.unpack_mask(P.mask_np(mask), n)
+            diff = keep != sel.keep_bool(n)
+            if literal:
+                assert not diff.any()
+            else:
+                assert not (diff & ~P.ewma_allowed_flips(sel)).any() and diff.sum() <= 1
+            assert np.array_equal(P.bits(out), np.where(keep, P.bits(W_ref), 0))
+            # nothing outside the output slice was touched
+            assert (big_out[:, :16] == 7.0).all() and (big_out[:, 16 + n:] == 7.0).all()
+    assert np.array_equal(P.bits(W), P.bits(W_ref))   # the input was not modified

@@ -326,6 +326,11 @@ sp_status sp_search_la(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_row
     if (st != SP_OK) return st;
     // The pruned fraction never increases with la (the threshold est - la*dev only moves down
     // and, with S frozen, est and dev do not depend on the decisions): bisection on [-8, 8].
+    // Rows that allow 16-byte access: the whole bisection runs on the device, one
+    // synchronisation at the end.
+    if (ewma_pair_path_applies(W, ldw, ctx->d_in))
+        return launch_search_la_device(ctx, W, dtype, n_rows, ldw, target_sparsity, alpha, beta,
+                                       iterations, la_out, achieved_out, s);
     const double total = static_cast<double>(n_rows) * static_cast<double>(ctx->d_in);
     float lo = -8.0f, hi = 8.0f, best_la = 0.0f;
     double best_gap = 2.0, best_frac = 0.0;

@@ -251,9 +251,11 @@ ewma_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
 // finalize_kernel): per 512-column tile, four 16-byte loads per lane, each contiguous across
 // the warp, deliver the lane's 16 factors in pair order (columns 0,4,1,5 | 2,6,3,7 of a chunk).
 struct PairConstants {
-    float a4, b4;       // a^4, b^4: chain 0-3 -> chain 4-7
-    float kappa;        // la * beta * a
-    float kappa_b[4];   // kappa * b^j
+    float a4, b4;        // a^4, b^4: chain 0-3 -> chain 4-7
+    float kappa;         // la * beta * a
+    float kappa_b[4];    // kappa * b^j
+    float unit_b[4];     // beta * a * b^j (kappa_b for la = 1)
+    int la_from_device;  // counting passes of the la search: la is DeviceScalars::search_la
 };
 
 // One step of the inclusive lane scan: x += m * (x of the lane `delta` below), for lanes that
@@ -331,11 +333,21 @@ ewma_pair_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n
     const float b16_lane0 = pinned(lane == 0 ? sc.b_step[1] : 0.0f);
     const int lane_below = (lane + 31) & 31;
     const bool is_lane0 = lane == 0;
-    const float kappa = pinned(pc.kappa);
+    float kappa_b[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) kappa_b[j] = pc.kappa_b[j];
+    if constexpr (COUNT) {
+        if (pc.la_from_device) {  // the bisection of sp_search_la keeps its current la on the device
+            const float la = scalars->search_la;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) kappa_b[j] = la * pc.unit_b[j];
+        }
+    }
+    const float kappa = pinned(kappa_b[0]);
     const float2 kappa2 = make_float2(kappa, kappa);
     float2 kappa_b2[4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) kappa_b2[j] = make_float2(pinned(pc.kappa_b[j]), pinned(pc.kappa_b[j]));
+    for (int j = 0; j < 4; ++j) kappa_b2[j] = make_float2(pinned(kappa_b[j]), pinned(kappa_b[j]));
     uint32_t kept = 0;
     uint32_t wmax = 0;
 
@@ -665,9 +677,14 @@ static void fill_scan_constants(const sp_ewma_params &p, ScanConstants &sc) {
     }
 }
 
+bool ewma_pair_path_applies(const void *W, int64_t ldw, int64_t n) {
+    return aligned16(W) && ldw % 8 == 0 && n % 8 == 0;
+}
+
 sp_status launch_select_ewma(const sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
                              int64_t ldw, const sp_ewma_params &p, uint32_t *mask, void *W_out,
-                             int64_t ldo, unsigned long long *counters, cudaStream_t stream) {
+                             int64_t ldo, unsigned long long *counters, cudaStream_t stream,
+                             bool la_from_device) {
     const int64_t n = ctx->d_in;
     if (n_rows == 0) return SP_OK;
     if (n_rows > 0x7fffffffLL || ldw > 0x7fffffffLL || ldo > 0x7fffffffLL) return SP_ERR_SHAPE;
@@ -712,7 +729,11 @@ sp_status launch_select_ewma(const sp_ctx *ctx, const void *W, sp_dtype dtype, i
         pc.b4 = static_cast<float>(pow(b, 4.0));
         const double kappa = static_cast<double>(p.la) * p.beta * sc.a;
         pc.kappa = static_cast<float>(kappa);
-        for (int j = 0; j < 4; ++j) pc.kappa_b[j] = static_cast<float>(kappa * pow(b, j));
+        for (int j = 0; j < 4; ++j) {
+            pc.kappa_b[j] = static_cast<float>(kappa * pow(b, j));
+            pc.unit_b[j] = static_cast<float>(static_cast<double>(p.beta) * sc.a * pow(b, j));
+        }
+        pc.la_from_device = la_from_device ? 1 : 0;
     }
     TileConstants wc;
     for (int k = 0; k < 5; ++k) {
@@ -759,6 +780,70 @@ sp_status launch_select_ewma(const sp_ctx *ctx, const void *W, sp_dtype dtype, i
 #undef SP_LAUNCH_P
     if (launch_err != cudaSuccess) return cuda_fail(launch_err);
     return check_launch();
+}
+
+// Bisection of la on the device: no host round trip between the counting passes.
+__global__ void search_init_kernel(DeviceScalars *s, float lo, float hi) {
+    s->search_lo = lo;
+    s->search_hi = hi;
+    s->search_la = 0.5f * (lo + hi);
+    s->search_best_la = 0.0f;
+    s->search_best_gap = 2.0;
+    s->search_best_frac = 0.0;
+    for (int i = 0; i < SP_NUM_COUNTERS; ++i) s->search_counters[i] = 0ULL;
+}
+
+__global__ void search_step_kernel(DeviceScalars *s, double total, double target) {
+    const float la = s->search_la;
+    const double pruned = 1.0 - static_cast<double>(s->search_counters[SP_COUNTER_KEPT]) / total;
+    const double gap = fabs(pruned - target);
+    if (gap < s->search_best_gap) {
+        s->search_best_gap = gap;
+        s->search_best_la = la;
+        s->search_best_frac = pruned;
+    }
+    if (pruned > target)
+        s->search_lo = la;  // too much pruned: raise la
+    else
+        s->search_hi = la;
+    s->search_la = 0.5f * (s->search_lo + s->search_hi);
+    for (int i = 0; i < SP_NUM_COUNTERS; ++i) s->search_counters[i] = 0ULL;
+}
+
+sp_status launch_search_la_device(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
+                                  int64_t ldw, float target, float alpha, float beta,
+                                  int iterations, float *la_out, double *achieved_out,
+                                  cudaStream_t stream) {
+    DeviceScalars *sc = ctx->scalars;
+    const double total = static_cast<double>(n_rows) * static_cast<double>(ctx->d_in);
+    search_init_kernel<<<1, 1, 0, stream>>>(sc, -8.0f, 8.0f);
+    sp_status st = check_launch();
+    if (st != SP_OK) return st;
+    sp_ewma_params p;
+    p.alpha = alpha;
+    p.beta = beta;
+    p.la = 0.0f;  // unused: the kernel reads DeviceScalars::search_la
+    p.s_update = SP_S_FROZEN;
+    for (int it = 0; it < iterations; ++it) {
+        st = launch_select_ewma(ctx, W, dtype, n_rows, ldw, p, nullptr, nullptr, ldw,
+                                sc->search_counters, stream, /*la_from_device=*/true);
+        if (st != SP_OK) return st;
+        search_step_kernel<<<1, 1, 0, stream>>>(sc, total, static_cast<double>(target));
+        st = check_launch();
+        if (st != SP_OK) return st;
+    }
+    float best_la = 0.0f;
+    double best_frac = 0.0;
+    cudaError_t e = cudaMemcpyAsync(&best_la, &sc->search_best_la, sizeof(float),
+                                    cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(&best_frac, &sc->search_best_frac, sizeof(double),
+                            cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+    *la_out = best_la;
+    if (achieved_out != nullptr) *achieved_out = best_frac;
+    return SP_OK;
 }
 
 }  // namespace sp

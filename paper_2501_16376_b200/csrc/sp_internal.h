@@ -24,6 +24,9 @@ struct DeviceScalars {
     int flags;            // kFlag*
     unsigned int ticket;  // arrival counter of the finalisation kernel (returns to 0)
     unsigned long long search_counters[SP_NUM_COUNTERS];  // scratch of sp_search_la
+    // state of sp_search_la's bisection when it runs on the device
+    float search_la, search_lo, search_hi, search_best_la;
+    double search_best_gap, search_best_frac;
 };
 
 // Powers of a = 1-alpha and b = 1-beta that the scan kernel needs (a lane owns P consecutive
@@ -102,7 +105,14 @@ sp_status launch_select_24_compressed(const sp_ctx *ctx, const void *W, sp_dtype
 // select_ewma.cu
 sp_status launch_select_ewma(const sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
                              int64_t ldw, const sp_ewma_params &p, uint32_t *mask, void *W_out,
-                             int64_t ldo, unsigned long long *counters, cudaStream_t stream);
+                             int64_t ldo, unsigned long long *counters, cudaStream_t stream,
+                             bool la_from_device = false);
+// True when launch_select_ewma would take the kernel that can read la from DeviceScalars.
+bool ewma_pair_path_applies(const void *W, int64_t ldw, int64_t n);
+sp_status launch_search_la_device(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
+                                  int64_t ldw, float target, float alpha, float beta,
+                                  int iterations, float *la_out, double *achieved_out,
+                                  cudaStream_t stream);
 
 // select_ewma_tiled.cu
 sp_status launch_ewma_literal_tiled(const sp_ctx *ctx, const void *W, sp_dtype dtype,

@@ -219,8 +219,10 @@ sp_status sp_ewma_trace(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_ro
  * names "finding the optimal sparsity" and frequent re-pruning as the use, Sections 1 and 4.2).
  * With S frozen the pruned fraction is a non-increasing function of la, so the call bisects
  * la on [-8, 8]: each of the `iterations` (1..64) steps runs Algorithm 1 over W at the midpoint
- * in count-only mode (W is read, nothing is written) and reads the kept count back, i.e. the
- * call SYNCHRONISES the stream once per step.  *la_out (host) receives the visited la whose
+ * in count-only mode (W is read, nothing is written).  For rows that allow 16-byte access
+ * (W 16-byte aligned, ldw and d_in multiples of 8) the bisection state stays on the device and
+ * the call SYNCHRONISES the stream once, at the end; otherwise the kept count is read back after
+ * every step (one synchronisation per step).  *la_out (host) receives the visited la whose
  * pruned fraction is closest to target_sparsity, *achieved_out (host, nullable) that fraction.
  * Follow with sp_select_unstructured_ex(la) to prune.
  */

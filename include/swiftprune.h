@@ -60,10 +60,16 @@ typedef enum {
 
 typedef enum { SP_F16 = 0, SP_BF16 = 1 } sp_dtype;
 
-/* How the EWMA selection treats Algorithm 1's step "S = S - w_i^2" (Table 2, row S). */
+/* How the EWMA selection treats Algorithm 1's step "S = S - w_i^2" (Table 2, row S).
+ * In binary32 the subtraction changes S only if w_i^2 reaches a quarter of the spacing of
+ * floats at S, which calibration-scale statistics (S ~ tokens * d_in) never allow. */
 typedef enum {
-    SP_S_FROZEN = 0,    /* S keeps its initial value; rows are scanned in parallel */
-    SP_S_LITERAL_W2 = 1 /* the printed update, evaluated sequentially along each row */
+    SP_S_GATED = 0,      /* Algorithm 1 as printed, at scan speed: rows are scanned in parallel with
+                            S at its initial value; a row holding a weight that could change S is
+                            detected and re-evaluated sequentially in the same call, so the
+                            result is that of SP_S_LITERAL_W2 for every row (the default) */
+    SP_S_LITERAL_W2 = 1, /* the printed update, evaluated sequentially along every row */
+    SP_S_FROZEN = 2      /* S keeps its initial value whatever is pruned */
 } sp_s_update;
 
 /* Parameters of Algorithm 1 (alpha, beta: Table 2; la: Table 3). */
@@ -179,17 +185,19 @@ sp_status sp_la_for_sparsity(float sparsity, float *la_out);
  *     (dev uses the updated est, as Algorithm 1 orders the two steps).
  * Column 0 of every row is therefore never pruned.
  *   sparsity   nominal pruning ratio; la = sp_la_for_sparsity(sparsity),
- *              alpha = beta = 0.125 (Section 4.2), S frozen.  The achieved ratio
+ *              alpha = beta = 0.125 (Section 4.2), SP_S_GATED.  The achieved ratio
  *              is only approximately the nominal one.
  *   mask_out   nullable; mask as described above.
  *   W_out      nullable; pruned copy of W with leading dimension ldo; may alias W
  *              exactly (same pointer, same ld) for in-place pruning.
  *   counters   nullable; SP_NUM_COUNTERS device uint64 the call ADDS to:
- *              [SP_COUNTER_KEPT] kept weights, [SP_COUNTER_S_HAZARD] rows in which
- *              Algorithm 1's "S = S - w_i^2" could have changed S in binary32
- *              (when 0, SP_S_FROZEN and SP_S_LITERAL_W2 give identical results).
- * The frozen-S path evaluates the two recurrences as warp-level affine scans in
- * fp32; results differ from a sequential fp32 evaluation by re-association only.
+ *              [SP_COUNTER_KEPT] kept weights, [SP_COUNTER_S_HAZARD] rows that held a weight
+ *              able to change S in binary32 and were therefore finished sequentially
+ *              (SP_S_GATED only; 0 at calibration scale).
+ * The scan evaluates the two recurrences as warp-level affine scans in fp32; results differ
+ * from a sequential fp32 evaluation by re-association only.  A row that SP_S_GATED finishes
+ * sequentially costs about as much as a thousand scanned rows: when the statistics are so
+ * small that most rows need it, SP_S_LITERAL_W2 is the faster way to the same result.
  */
 sp_status sp_select_unstructured(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
                                  int64_t ldw, float sparsity, uint32_t *mask_out, void *W_out,

@@ -97,13 +97,14 @@ sp_status sp_create(sp_ctx **out, int64_t d_in, int device) {
     ctx->calib_blocks_per_sm = calib_query_blocks_per_sm();
 
     const size_t np = static_cast<size_t>(ctx->n_pad);
-    void *ptrs[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
-    const size_t sizes[6] = {sizeof(double) * np * kMaxSlabs, sizeof(double) * np,
-                             sizeof(double) * static_cast<size_t>(ctx->strips),
-                             sizeof(float) * (np + kStripChannels),
-                             sizeof(DeviceScalars),
-                             sizeof(float) * ((np + 511) / 512 * 512 + 512)};
-    for (int i = 0; i < 6; ++i) {
+    constexpr int kBuffers = 6;
+    void *ptrs[kBuffers] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+    const size_t sizes[kBuffers] = {sizeof(double) * np * kMaxSlabs, sizeof(double) * np,
+                                    sizeof(double) * static_cast<size_t>(ctx->strips),
+                                    sizeof(float) * (np + kStripChannels),
+                                    sizeof(DeviceScalars),
+                                    sizeof(float) * ((np + 511) / 512 * 512 + 512)};
+    for (int i = 0; i < kBuffers; ++i) {
         e = cudaMalloc(&ptrs[i], sizes[i]);
         if (e == cudaSuccess) e = cudaMemset(ptrs[i], 0, sizes[i]);
         if (e != cudaSuccess) {
@@ -266,7 +267,8 @@ sp_status sp_select_unstructured_ex(sp_ctx *ctx, const void *W, sp_dtype dtype, 
     if (!(params->alpha > 0.0f) || !(params->alpha <= 1.0f) || !(params->beta > 0.0f) ||
         !(params->beta <= 1.0f) || !std::isfinite(params->la))
         return SP_ERR_INVALID_ARG;
-    if (params->s_update != SP_S_FROZEN && params->s_update != SP_S_LITERAL_W2)
+    if (params->s_update != SP_S_GATED && params->s_update != SP_S_FROZEN &&
+        params->s_update != SP_S_LITERAL_W2)
         return SP_ERR_INVALID_ARG;
     if (ctx->n_tokens <= 0) return SP_ERR_STATE;
     DeviceGuard guard(ctx->device);
@@ -283,7 +285,7 @@ sp_status sp_select_unstructured(sp_ctx *ctx, const void *W, sp_dtype dtype, int
     sp_ewma_params p;
     p.alpha = 0.125f;  // Section 4.2
     p.beta = 0.125f;
-    p.s_update = SP_S_FROZEN;
+    p.s_update = SP_S_GATED;
     sp_status st = sp_la_for_sparsity(sparsity, &p.la);
     if (st != SP_OK) return st;
     return sp_select_unstructured_ex(ctx, W, dtype, n_rows, ldw, &p, mask_out, W_out, ldo, counters,
@@ -298,7 +300,8 @@ sp_status sp_ewma_trace(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_ro
     if (params == nullptr || !(params->alpha > 0.0f) || !(params->alpha <= 1.0f) ||
         !(params->beta > 0.0f) || !(params->beta <= 1.0f) || !std::isfinite(params->la))
         return SP_ERR_INVALID_ARG;
-    if (params->s_update != SP_S_FROZEN && params->s_update != SP_S_LITERAL_W2)
+    if (params->s_update != SP_S_GATED && params->s_update != SP_S_FROZEN &&
+        params->s_update != SP_S_LITERAL_W2)
         return SP_ERR_INVALID_ARG;
     if (ctx->n_tokens <= 0) return SP_ERR_STATE;
     DeviceGuard guard(ctx->device);
@@ -450,7 +453,7 @@ sp_status sp_select_unstructured_host(sp_ctx *ctx, const void *W_host, sp_dtype 
     sp_ewma_params p;
     p.alpha = 0.125f;
     p.beta = 0.125f;
-    p.s_update = SP_S_FROZEN;
+    p.s_update = SP_S_GATED;
     st = sp_la_for_sparsity(sparsity, &p.la);
     if (st != SP_OK) return st;
     if (ctx->n_tokens <= 0) return SP_ERR_STATE;

@@ -15,14 +15,24 @@
 // path: packed binary32 pairs, weights streamed through a shared-memory ring of asynchronous
 // copies) and ewma_scan_kernel for any other pointer, stride or width.
 //
+// Drift gate (SP_S_GATED).  "S = S - w_i^2" (Table 2, row S) changes S in binary32 only when a
+// pruned weight has w_i^2 >= DeviceScalars::hazard_w2.  The scan kernels test every tile for
+// such a weight before they store anything of it; at the first tile that may hold one, the warp
+// notes the column and the state of Algorithm 1 before it and stops storing, and once its scan
+// loop has ended one of its lanes takes the row up again at that column and walks it
+// sequentially with the printed update (literal_walk).  Up to that column the frozen and the
+// printed rule are the same rule, so the result is Algorithm 1 as printed; the input is never
+// overwritten ahead of the sequential walk, so pruning in place works as well.  A row that is
+// walked this way costs about as much as a thousand scanned ones: the gate is a safety net for
+// stray rows, and SP_S_LITERAL_W2 the mode for statistics so small that every row needs it.
+//
 // Literal-S path (sequential kernels, here and in select_ewma_tiled.cu).  Algorithm 1's
 // "S = S - w_i^2" makes L_i depend on earlier decisions, so the row is evaluated in order by one
 // thread, every operation in binary32 with one rounding each.  It is the exact path, bound by
 // the latency of one dependent chain per row.
 #include <math.h>
 
-#include "sp_device.cuh"
-#include "sp_internal.h"
+#include "ewma_common.cuh"
 
 namespace sp {
 
@@ -47,22 +57,6 @@ constexpr int kPairWarps = kPairThreads / 32;
 constexpr int kEwmaStages = SP_EWMA_STAGES;       // ring slots per warp (a power of two)
 static_assert((kEwmaStages & (kEwmaStages - 1)) == 0, "ring size must be a power of two");
 
-// Running packed maximum of |w| (two 16-bit floats per word).
-template <bool BF16>
-__device__ __forceinline__ uint32_t packed_abs_max(uint32_t acc, uint32_t v) {
-    if constexpr (BF16) {
-        __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162 *>(&acc);
-        __nv_bfloat162 b = __habs2(*reinterpret_cast<__nv_bfloat162 *>(&v));
-        __nv_bfloat162 m = __hmax2(a, b);
-        return *reinterpret_cast<uint32_t *>(&m);
-    } else {
-        __half2 a = *reinterpret_cast<__half2 *>(&acc);
-        __half2 b = __habs2(*reinterpret_cast<__half2 *>(&v));
-        __half2 m = __hmax2(a, b);
-        return *reinterpret_cast<uint32_t *>(&m);
-    }
-}
-
 // Inclusive scan over lanes of x with the recurrence multiplier step[k] = m^(P*2^k).
 __device__ __forceinline__ float lane_affine_scan(float x, const float (&step)[5], int lane) {
 #pragma unroll
@@ -73,26 +67,115 @@ __device__ __forceinline__ float lane_affine_scan(float x, const float (&step)[5
     return x;
 }
 
+// The matrices of one launch.  Rows are numbered through all jobs.
+struct EwmaJob {
+    const uint16_t *W;
+    uint16_t *W_out;  // nullable
+    uint32_t *mask;   // nullable
+    int ldw, ldo, n_rows;
+    int first_row;
+};
+struct EwmaJobTable {
+    int count;
+    int total_rows;
+    EwmaJob job[kEwmaMaxJobs];
+};
+
+// Algorithm 1 exactly as printed along one row from column i_begin (a multiple of 32) on, by
+// one thread, binary32 with one rounding per operation; est / dev are the state before that
+// column (ignored for column 0, where est starts at L_0).  Element-wise access with bounds
+// checks.  While S still has its initial value the per-channel factor computed at finalisation
+// is used: it was formed by the same three operations from the same S, so the result is
+// bit-identical to recomputing it; once a pruned weight has changed S the factor is recomputed
+// for every element.  Returns the number of kept weights.
+template <bool BF16>
+__device__ __forceinline__ unsigned long long literal_walk(
+    const uint16_t *__restrict__ wrow, uint16_t *__restrict__ orow, uint32_t *__restrict__ mrow,
+    int64_t n, int64_t i_begin, float est, float dev, const double *__restrict__ colsq,
+    const float *__restrict__ factor, float S0, float alpha, float beta, float la) {
+    const float one_minus_alpha = __fsub_rn(1.0f, alpha);
+    const float one_minus_beta = __fsub_rn(1.0f, beta);
+    float S = S0;
+    uint32_t word = 0;
+    unsigned long long kept = 0;
+    // two chunks are kept in flight ahead of the one being evaluated
+    uint32_t ahead[2][4];
+    load8<false, true>(wrow, i_begin, n, ahead[0]);
+    load8<false, true>(wrow, i_begin + 8, n, ahead[1]);
+    for (int64_t i0 = i_begin; i0 < n; i0 += 8) {
+        uint32_t p[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            p[k] = ahead[0][k];
+            ahead[0][k] = ahead[1][k];
+        }
+        load8<false, true>(wrow, i0 + 16, n, ahead[1]);
+        float w[8];
+        unpack8<BF16>(p, w);
+        uint32_t keep8 = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int64_t i = i0 + j;
+            if (i < n) {
+                float c;
+                if (S == S0) {
+                    c = __ldg(factor + i);
+                } else {
+                    const float u = __fdiv_rn(static_cast<float>(colsq[i]), S);
+                    c = __fdiv_rn(0.5f, __fsub_rn(1.0f, u));
+                }
+                const float w2 = __fmul_rn(w[j], w[j]);
+                const float L = __fmul_rn(w2, c);
+                if (i == 0) est = L;
+                const float thr = __fsub_rn(est, __fmul_rn(la, dev));
+                if (L < thr) {
+                    S = __fsub_rn(S, w2);
+                } else {
+                    keep8 |= 1u << j;
+                }
+                est = __fadd_rn(__fmul_rn(one_minus_alpha, est), __fmul_rn(alpha, L));
+                dev = __fadd_rn(__fmul_rn(one_minus_beta, dev),
+                                __fmul_rn(beta, fabsf(__fsub_rn(est, L))));
+            }
+        }
+        kept += __popc(keep8);
+        if (orow != nullptr) {
+            zero_pruned(p, keep8);
+            store8<false>(orow, i0, n, p);
+        }
+        word |= keep8 << (i0 & 31);
+        if ((i0 & 31) == 24 || i0 + 8 >= n) {
+            if (mrow != nullptr) mrow[i0 >> 5] = word;
+            word = 0;
+        }
+    }
+    return kept;
+}
+
+// Drift gate: the rest of a row, from column `col` on, for a scan kernel that had to leave it
+// (est, dev: the state of Algorithm 1 before that column).  Rarely taken, kept out of line.
+template <bool BF16>
+__device__ __noinline__ unsigned long long gate_walk(
+    const uint16_t *wrow, uint16_t *orow, uint32_t *mrow, int n, int col, float est, float dev,
+    const double *colsq, const float *factor, const DeviceScalars *scalars, float alpha, float beta,
+    float la, unsigned long long *counters) {
+    if (counters != nullptr) atomicAdd(counters + SP_COUNTER_S_HAZARD, 1ULL);
+    return literal_walk<BF16>(wrow, orow, mrow, n, col, est, dev, colsq, factor, scalars->S32,
+                              alpha, beta, la);
+}
+
 // The kernel carries the two states in scaled form, E = est/alpha and D = dev/beta:
 //     E_i = a E_{i-1} + L_i ,   D_i = b D_{i-1} + |alpha E_i - L_i| ,
 // and element i is pruned iff  L_i - alpha E_{i-1} + (la beta) D_{i-1} < 0.
-// Keeps a kernel parameter in a register for the whole kernel (the compiler would otherwise be
-// free to re-read it from the constant bank at every use).
-__device__ __forceinline__ float pinned(float v) {
-    float r;
-    asm volatile("mov.f32 %0, %1;" : "=f"(r) : "f"(v));
-    return r;
-}
-
 // General scan kernel: element-wise access with bounds checks, any alignment, stride or width.
-// COUNT: also produce the kept-weight count and the S-hazard flag of the row.
-template <bool BF16, bool COUNT>
+// COUNT: also produce the kept-weight count.  GATE: the drift gate described above.
+template <bool BF16, bool COUNT, bool GATE>
 __global__ void __launch_bounds__(kEwmaThreads, SP_EWMA_MIN_BLOCKS)
 ewma_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
                  const float *__restrict__ factor, const DeviceScalars *__restrict__ scalars,
                  const __grid_constant__ ScanConstants sc, uint32_t *__restrict__ mask,
                  int mask_words, uint16_t *__restrict__ W_out, int ldo,
-                 unsigned long long *__restrict__ counters) {
+                 unsigned long long *__restrict__ counters, const double *__restrict__ colsq) {
     pdl_launch_dependents();
     pdl_wait();  // the per-channel factors come from an earlier kernel of the stream
     const int lane = threadIdx.x & 31;
@@ -113,7 +196,8 @@ ewma_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
     const int tiles = (n + kEwmaTile - 1) / kEwmaTile;
     float carry_E = 0.0f, carry_D = 0.0f;
     uint32_t kept = 0;
-    uint32_t wmax = 0;  // packed running max of |w| over this lane's elements
+    int left_at = -1;  // GATE: column from which the row is walked sequentially
+    const float hazard_w2 = GATE ? scalars->hazard_w2 : 0.0f;
     uint32_t p_next[4];
     load8<false, true>(wrow, lane * kEwmaPerLane, n, p_next);
 
@@ -129,12 +213,24 @@ ewma_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
         load_factor8(factor, col, c);  // zero past d_in: scores of padding are 0
 #pragma unroll
         for (int j = 0; j < 8; ++j) L[j] = __fmul_rn(__fmul_rn(w[j], w[j]), c[j]);
-        if constexpr (COUNT) {
-#pragma unroll
-            for (int k = 0; k < 4; ++k) wmax = packed_abs_max<BF16>(wmax, p[k]);
-        }
 
         if (tile == 0) carry_E = __shfl_sync(kFullWarp, L[0], 0) / alpha;  // est starts at L_0
+        if constexpr (GATE) {
+            // a weight of this tile could change S if it were pruned: the sequential kernel
+            // takes the row up from here (nothing of the tile has been stored yet)
+            float w2max = 0.0f;
+            bool odd = false;  // a NaN weight
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float w2 = __fmul_rn(w[j], w[j]);
+                odd = odd || !(w2 == w2);
+                w2max = fmaxf(w2max, w2);
+            }
+            if (__any_sync(kFullWarp, odd || !(w2max < hazard_w2))) {
+                left_at = tile * kEwmaTile;
+                break;
+            }
+        }
 
         // Pass A: E over the lane's elements from a zero state -> lane total -> scan.
         float acc = L[0];
@@ -199,18 +295,18 @@ ewma_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
         if (mrow != nullptr && (lane & 3) == 0 && col < n) mrow[col >> 5] = word;
     }
 
+    unsigned long long walked = 0;
+    if constexpr (GATE) {
+        if (left_at >= 0 && lane == 0)
+            walked = gate_walk<BF16>(wrow, orow, mrow, n, left_at, __fmul_rn(alpha, carry_E),
+                                     __fmul_rn(sc.beta, carry_D), colsq, factor, scalars, sc.alpha,
+                                     sc.beta, sc.la, counters);
+    }
     if constexpr (COUNT) {
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) kept += __shfl_xor_sync(kFullWarp, kept, off);
-        float2 m2 = unpack2<BF16>(wmax);
-        float bound = fmaxf(m2.x, m2.y);
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1)
-            bound = fmaxf(bound, __shfl_xor_sync(kFullWarp, bound, off));
-        if (lane == 0) {
-            atomicAdd(counters + SP_COUNTER_KEPT, static_cast<unsigned long long>(kept));
-            if (!(bound * bound < scalars->hazard_w2)) atomicAdd(counters + SP_COUNTER_S_HAZARD, 1ULL);
-        }
+        if (lane == 0 && kept + walked != 0ULL)
+            atomicAdd(counters + SP_COUNTER_KEPT, static_cast<unsigned long long>(kept) + walked);
     }
 }
 
@@ -252,72 +348,41 @@ ewma_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
 // the warp, deliver the lane's 16 factors in pair order (columns 0,4,1,5 | 2,6,3,7 of a chunk).
 struct PairConstants {
     float a4, b4;        // a^4, b^4: chain 0-3 -> chain 4-7
-    float kappa;         // la * beta * a
-    float kappa_b[4];    // kappa * b^j
-    float unit_b[4];     // beta * a * b^j (kappa_b for la = 1)
+    float la;            // the decision constants kappa * b^j are formed on the device as
+    float unit_b[4];     // la * (beta * a * b^j), the same way wherever la comes from
     int la_from_device;  // counting passes of the la search: la is DeviceScalars::search_la
+    float hazard_scale;  // a^3 / 2, a little lowered (gate test on the chain totals)
 };
-
-// One step of the inclusive lane scan: x += m * (x of the lane `delta` below), for lanes that
-// have such a lane.  The shuffle's own predicate output says whether the source lane exists, so
-// no comparison on the lane index is needed.
-template <int DELTA>
-__device__ __forceinline__ float lane_scan_step(float x, float m) {
-    float r;
-    asm volatile(
-        "{\n\t"
-        ".reg .pred p;\n\t"
-        ".reg .f32 y;\n\t"
-        "shfl.sync.up.b32 y|p, %1, %2, 0, 0xffffffff;\n\t"
-        "mov.f32 %0, %1;\n\t"
-        "@p fma.rn.f32 %0, %3, y, %1;\n\t"
-        "}"
-        : "=&f"(r)
-        : "f"(x), "n"(DELTA), "f"(m));
-    return r;
-}
-__device__ __forceinline__ float lane_affine_scan_pred(float x, const float (&step)[5]) {
-    x = lane_scan_step<1>(x, step[0]);
-    x = lane_scan_step<2>(x, step[1]);
-    x = lane_scan_step<4>(x, step[2]);
-    x = lane_scan_step<8>(x, step[3]);
-    x = lane_scan_step<16>(x, step[4]);
-    return x;
-}
-template <bool BF16>
-__device__ __forceinline__ float unpack_lo(uint32_t u) {
-    if constexpr (BF16) return __uint_as_float(u << 16);
-    else return __half2float(__ushort_as_half(static_cast<unsigned short>(u & 0xffffu)));
-}
-template <bool BF16>
-__device__ __forceinline__ float unpack_hi(uint32_t u) {
-    if constexpr (BF16) return __uint_as_float(u & 0xffff0000u);
-    else return __half2float(__ushort_as_half(static_cast<unsigned short>(u >> 16)));
-}
 
 struct TileConstants {
     float a_step[5], b_step[5];  // a^(16*2^k), b^(16*2^k)
     float a8, b8;
 };
 
-template <bool BF16, bool FULL, bool COUNT>
+template <bool BF16, bool FULL, bool COUNT, bool GATE>
 __global__ void __launch_bounds__(kPairThreads, SP_EWMA_PAIR_MIN_BLOCKS)
-ewma_pair_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
+ewma_pair_scan_kernel(const __grid_constant__ EwmaJobTable jobs, int n,
                       const float *__restrict__ factor_pairs,
                       const DeviceScalars *__restrict__ scalars,
                       const __grid_constant__ ScanConstants sc,
                       const __grid_constant__ PairConstants pc,
-                      const __grid_constant__ TileConstants wc, uint32_t *__restrict__ mask,
-                      int mask_words, uint16_t *__restrict__ W_out, int ldo,
-                      unsigned long long *__restrict__ counters) {
+                      const __grid_constant__ TileConstants wc, int mask_words,
+                      unsigned long long *__restrict__ counters,
+                      const double *__restrict__ colsq, const float *__restrict__ factor) {
     constexpr int kTile = 512;
     pdl_launch_dependents();
     pdl_wait();  // the per-channel factors come from an earlier kernel of the stream
     const int lane = threadIdx.x & 31;
-    const int row = blockIdx.x * kPairWarps + (threadIdx.x >> 5);
-    if (row >= n_rows) return;  // warp-uniform
-    const uint16_t *wrow = W + static_cast<int64_t>(row) * ldw;
-    uint16_t *olane = W_out != nullptr ? W_out + static_cast<int64_t>(row) * ldo + lane * 16 : nullptr;
+    const int grow = blockIdx.x * kPairWarps + (threadIdx.x >> 5);  // row among all jobs
+    if (grow >= jobs.total_rows) return;  // warp-uniform
+    int jk = 0;
+    while (jk + 1 < jobs.count && grow >= jobs.job[jk + 1].first_row) ++jk;
+    const int row = grow - jobs.job[jk].first_row;
+    const int ldw = jobs.job[jk].ldw;
+    const uint16_t *wrow = jobs.job[jk].W + static_cast<int64_t>(row) * ldw;
+    uint16_t *const W_out = jobs.job[jk].W_out;
+    uint32_t *const mask = jobs.job[jk].mask;
+    uint16_t *olane = W_out != nullptr ? W_out + static_cast<int64_t>(row) * jobs.job[jk].ldo + lane * 16 : nullptr;
     uint16_t *mlane = mask != nullptr
                           ? reinterpret_cast<uint16_t *>(mask + static_cast<int64_t>(row) * mask_words) + lane
                           : nullptr;
@@ -333,26 +398,26 @@ ewma_pair_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n
     const float b16_lane0 = pinned(lane == 0 ? sc.b_step[1] : 0.0f);
     const int lane_below = (lane + 31) & 31;
     const bool is_lane0 = lane == 0;
+    float la = pc.la;
+    if constexpr (COUNT) {
+        // the bisection of sp_search_la keeps its current la on the device
+        if (pc.la_from_device) la = scalars->search_la;
+    }
     float kappa_b[4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) kappa_b[j] = pc.kappa_b[j];
-    if constexpr (COUNT) {
-        if (pc.la_from_device) {  // the bisection of sp_search_la keeps its current la on the device
-            const float la = scalars->search_la;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) kappa_b[j] = la * pc.unit_b[j];
-        }
-    }
+    for (int j = 0; j < 4; ++j) kappa_b[j] = __fmul_rn(la, pc.unit_b[j]);
     const float kappa = pinned(kappa_b[0]);
     const float2 kappa2 = make_float2(kappa, kappa);
     float2 kappa_b2[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) kappa_b2[j] = make_float2(pinned(kappa_b[j]), pinned(kappa_b[j]));
     uint32_t kept = 0;
-    uint32_t wmax = 0;
+    float hz_thr = 0.0f;
+    if constexpr (GATE) hz_thr = scalars->hazard_w2 * pc.hazard_scale;
 
     constexpr int kSlot = 64;  // uint4 per warp and stage
     __shared__ __align__(16) uint4 ring[kPairWarps * kEwmaStages * kSlot];
+    __shared__ int gate_snap[GATE ? kPairWarps : 1][4 + 32];
     uint4 *my_ring = ring + (threadIdx.x >> 5) * kEwmaStages * kSlot;
     const int wpos = lane ^ ((lane >> 3) & 1);               // where this lane's copies go
     const int rpos_a = 2 * lane + ((lane >> 2) & 1);         // where chunk 2*lane sits
@@ -386,6 +451,9 @@ ewma_pair_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n
     float4 cf_next[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) cf_next[i] = __ldg(flane + 32 * i);
+    if constexpr (GATE) {
+        if (is_lane0) gate_snap[threadIdx.x >> 5][0] = -1;  // no column recorded yet
+    }
     for (int t0 = 0; t0 < tiles; t0 += kEwmaStages) {
 #pragma unroll
         for (int u = 0; u < kEwmaStages; ++u) {
@@ -423,10 +491,6 @@ ewma_pair_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n
                 L2[x][2] = __fmul2_rn(__fmul2_rn(w2, w2), make_float2(cf[2 * x + 1].x, cf[2 * x + 1].y));
                 w2 = make_float2(unpack_hi<BF16>(p[x][1]), unpack_hi<BF16>(p[x][3]));
                 L2[x][3] = __fmul2_rn(__fmul2_rn(w2, w2), make_float2(cf[2 * x + 1].z, cf[2 * x + 1].w));
-                if constexpr (COUNT) {
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) wmax = packed_abs_max<BF16>(wmax, p[x][k]);
-                }
                 // E: the chunk's two chains from a zero state
                 acc[x] = L2[x][0];
 #pragma unroll
@@ -434,8 +498,33 @@ ewma_pair_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n
             }
             // chunk totals -> lane total (+ a^16 carry in lane 0) -> scan over lanes
             const float tot_a = fmaf(a4, acc[0].x, acc[0].y), tot_b = fmaf(a4, acc[1].x, acc[1].y);
-            float incl = lane_affine_scan_pred(
-                fmaf(a16_lane0, carry_E, fmaf(a8, tot_a, tot_b)), wc.a_step);
+            const float lane_tot = fmaf(a8, tot_a, tot_b);
+            if constexpr (GATE) {
+                // Every score is at least w^2 / 2 and a chain's zero-state total at least a^3
+                // times any of its 4 scores, so four totals below the scaled bound rule out a
+                // weight that could change S (a NaN fails the test as well).  Otherwise the
+                // sequential kernel takes the row up from this tile: nothing of it has been
+                // stored yet, and nothing more of the row is stored or counted here.
+                const float m4 = fmaxf(fmaxf(acc[0].x, acc[0].y), fmaxf(acc[1].x, acc[1].y));
+                if (__any_sync(kFullWarp, !(lane_tot == lane_tot) || !(m4 < hz_thr))) {
+                    // (rare) remember the column, the scaled state before it and the count so
+                    // far - only the first time - and stop storing: the outputs are off from here
+                    int *snap = gate_snap[threadIdx.x >> 5];
+                    const bool first = snap[0] < 0;
+                    __syncwarp();
+                    if (first) {
+                        snap[4 + lane] = static_cast<int>(kept);
+                        if (is_lane0) {
+                            snap[0] = tile * kTile;
+                            snap[1] = __float_as_int(carry_E);
+                            snap[2] = __float_as_int(carry_D);
+                        }
+                    }
+                    olane = nullptr;
+                    mlane = nullptr;
+                }
+            }
+            float incl = lane_affine_scan_pred(fmaf(a16_lane0, carry_E, lane_tot), wc.a_step);
             float rot = __shfl_sync(kFullWarp, incl, lane_below);
             const float e0 = is_lane0 ? carry_E : rot;  // E before element 0
             carry_E = rot;
@@ -509,27 +598,31 @@ ewma_pair_scan_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n
         }
     }
 
+    unsigned long long walked = 0;
+    if constexpr (GATE) {
+        __syncwarp();
+        const int *snap = gate_snap[threadIdx.x >> 5];
+        if (snap[0] >= 0) {  // the scan stopped storing at column snap[0]: walk the rest
+            kept = static_cast<uint32_t>(snap[4 + lane]);  // kept before that column
+            if (is_lane0)
+                walked = gate_walk<BF16>(
+                    wrow, W_out != nullptr ? W_out + static_cast<int64_t>(row) * jobs.job[jk].ldo : nullptr,
+                    mask != nullptr ? mask + static_cast<int64_t>(row) * mask_words : nullptr, n,
+                    snap[0], __fmul_rn(sc.alpha, __int_as_float(snap[1])),
+                    __fmul_rn(pc.unit_b[0], __int_as_float(snap[2])), colsq, factor, scalars,
+                    sc.alpha, sc.beta, la, counters);
+        }
+    }
     if constexpr (COUNT) {
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) kept += __shfl_xor_sync(kFullWarp, kept, off);
-        float2 m2 = unpack2<BF16>(wmax);
-        float bound = fmaxf(m2.x, m2.y);
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1)
-            bound = fmaxf(bound, __shfl_xor_sync(kFullWarp, bound, off));
-        if (lane == 0) {
-            atomicAdd(counters + SP_COUNTER_KEPT, static_cast<unsigned long long>(kept));
-            if (!(bound * bound < scalars->hazard_w2)) atomicAdd(counters + SP_COUNTER_S_HAZARD, 1ULL);
-        }
+        if (lane == 0 && kept + walked != 0ULL)
+            atomicAdd(counters + SP_COUNTER_KEPT, static_cast<unsigned long long>(kept) + walked);
     }
 }
 
-// Algorithm 1 exactly as printed, one thread per row, binary32 with one rounding per operation.
-// Element-wise access with bounds checks: the path for rows that do not allow 16-byte access
-// (ewma_literal_tiled_kernel handles those that do).  While S still
-// has its initial value the per-channel factor computed at finalisation is used: it was formed
-// by the same three operations from the same S, so the result is bit-identical to recomputing
-// it; once a pruned weight has changed S the factor is recomputed for every element.
+// The sequential path for rows that do not allow 16-byte access (ewma_literal_tiled_kernel
+// handles those that do): one thread per row, whole rows.
 template <bool BF16>
 __global__ void __launch_bounds__(128)
 ewma_literal_kernel(const uint16_t *__restrict__ W, int64_t ldw, int64_t n_rows, int64_t n,
@@ -540,67 +633,10 @@ ewma_literal_kernel(const uint16_t *__restrict__ W, int64_t ldw, int64_t n_rows,
                     unsigned long long *__restrict__ counters) {
     const int64_t row = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (row >= n_rows) return;
-    const uint16_t *wrow = W + row * ldw;
-    uint16_t *orow = W_out != nullptr ? W_out + row * ldo : nullptr;
-    uint32_t *mrow = mask != nullptr ? mask + row * mask_words : nullptr;
-    const float one_minus_alpha = __fsub_rn(1.0f, alpha);
-    const float one_minus_beta = __fsub_rn(1.0f, beta);
-    const float S0 = scalars->S32;
-    float S = S0;
-    float est = 0.0f, dev = 0.0f;
-    uint32_t word = 0;
-    unsigned long long kept = 0;
-    // two chunks are kept in flight ahead of the one being evaluated
-    uint32_t ahead[2][4];
-    load8<false, true>(wrow, 0, n, ahead[0]);
-    load8<false, true>(wrow, 8, n, ahead[1]);
-    for (int64_t i0 = 0; i0 < n; i0 += 8) {
-        uint32_t p[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            p[k] = ahead[0][k];
-            ahead[0][k] = ahead[1][k];
-        }
-        load8<false, true>(wrow, i0 + 16, n, ahead[1]);
-        float w[8];
-        unpack8<BF16>(p, w);
-        uint32_t keep8 = 0;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int64_t i = i0 + j;
-            if (i < n) {
-                float c;
-                if (S == S0) {
-                    c = __ldg(factor + i);
-                } else {
-                    const float u = __fdiv_rn(static_cast<float>(colsq[i]), S);
-                    c = __fdiv_rn(0.5f, __fsub_rn(1.0f, u));
-                }
-                const float w2 = __fmul_rn(w[j], w[j]);
-                const float L = __fmul_rn(w2, c);
-                if (i == 0) est = L;
-                const float thr = __fsub_rn(est, __fmul_rn(la, dev));
-                if (L < thr) {
-                    S = __fsub_rn(S, w2);
-                } else {
-                    keep8 |= 1u << j;
-                }
-                est = __fadd_rn(__fmul_rn(one_minus_alpha, est), __fmul_rn(alpha, L));
-                dev = __fadd_rn(__fmul_rn(one_minus_beta, dev),
-                                __fmul_rn(beta, fabsf(__fsub_rn(est, L))));
-            }
-        }
-        kept += __popc(keep8);
-        if (orow != nullptr) {
-            zero_pruned(p, keep8);
-            store8<false>(orow, i0, n, p);
-        }
-        word |= keep8 << (i0 & 31);
-        if ((i0 & 31) == 24 || i0 + 8 >= n) {
-            if (mrow != nullptr) mrow[i0 >> 5] = word;
-            word = 0;
-        }
-    }
+    const unsigned long long kept = literal_walk<BF16>(
+        W + row * ldw, W_out != nullptr ? W_out + row * ldo : nullptr,
+        mask != nullptr ? mask + row * mask_words : nullptr, n, 0, 0.0f, 0.0f, colsq, factor,
+        scalars->S32, alpha, beta, la);
     if (counters != nullptr) atomicAdd(counters + SP_COUNTER_KEPT, kept);
 }
 
@@ -648,7 +684,7 @@ sp_status launch_ewma_trace(const sp_ctx *ctx, const void *W, sp_dtype dtype, in
     const int64_t blocks = (n_rows + 127) / 128;
     if (blocks > 0x7fffffffLL) return SP_ERR_SHAPE;
     const uint16_t *Wp = static_cast<const uint16_t *>(W);
-    const int literal = p.s_update == SP_S_LITERAL_W2 ? 1 : 0;
+    const int literal = p.s_update != SP_S_FROZEN ? 1 : 0;  // gated = Algorithm 1 as printed
     if (dtype == SP_BF16)
         ewma_trace_kernel<true><<<static_cast<unsigned>(blocks), 128, 0, stream>>>(
             Wp, ldw, n_rows, ctx->d_in, ctx->colsq, ctx->scalars, p.alpha, p.beta, p.la, literal,
@@ -681,105 +717,194 @@ bool ewma_pair_path_applies(const void *W, int64_t ldw, int64_t n) {
     return aligned16(W) && ldw % 8 == 0 && n % 8 == 0;
 }
 
-sp_status launch_select_ewma(const sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
-                             int64_t ldw, const sp_ewma_params &p, uint32_t *mask, void *W_out,
-                             int64_t ldo, unsigned long long *counters, cudaStream_t stream,
-                             bool la_from_device) {
-    const int64_t n = ctx->d_in;
-    if (n_rows == 0) return SP_OK;
-    if (n_rows > 0x7fffffffLL || ldw > 0x7fffffffLL || ldo > 0x7fffffffLL) return SP_ERR_SHAPE;
-    const uint16_t *Wp = static_cast<const uint16_t *>(W);
-    uint16_t *Op = static_cast<uint16_t *>(W_out);
-    const int64_t words = (n + 31) / 32;
-    const bool bf16 = dtype == SP_BF16;
+namespace {
 
-    if (p.s_update == SP_S_LITERAL_W2) {
-        const int64_t blocks = (n_rows + 127) / 128;
-        if (blocks > 0x7fffffffLL) return SP_ERR_SHAPE;
-        const bool lvec = aligned16(W) && ldw % 8 == 0 && n % 8 == 0 &&
-                          (W_out == nullptr || (aligned16(W_out) && ldo % 8 == 0));
-        if (lvec)  // rows that allow 16-byte access: the same arithmetic, rows moved in tiles
-            return launch_ewma_literal_tiled(ctx, W, dtype, n_rows, ldw, p, mask, W_out, ldo,
-                                             counters, stream);
-        const unsigned lgrid = static_cast<unsigned>(blocks);
-#define SP_LAUNCH_L(B)                                                                       \
-    ewma_literal_kernel<B><<<lgrid, 128, 0, stream>>>(                                       \
-        Wp, ldw, n_rows, n, ctx->colsq, ctx->factor, ctx->scalars, p.alpha, p.beta, p.la, mask, \
-        words, Op, ldo, counters)
-        if (bf16) SP_LAUNCH_L(true); else SP_LAUNCH_L(false);
-#undef SP_LAUNCH_L
-        return check_launch();
+bool job_is_vector(const EwmaLaunchJob &j, int64_t n) {
+    return aligned16(j.W) && j.ldw % 8 == 0 && n % 8 == 0 &&
+           (j.W_out == nullptr || (aligned16(j.W_out) && j.ldo % 8 == 0));
+}
+
+// Device-side table of the jobs [first, first + count); false if there are too many rows.
+bool fill_job_table(const EwmaLaunchJob *jobs, int first, int count, EwmaJobTable &t) {
+    t.count = count;
+    int64_t rows = 0;
+    for (int i = 0; i < count; ++i) {
+        const EwmaLaunchJob &j = jobs[first + i];
+        EwmaJob &d = t.job[i];
+        d.W = static_cast<const uint16_t *>(j.W);
+        d.W_out = static_cast<uint16_t *>(j.W_out);
+        d.mask = j.mask;
+        d.ldw = static_cast<int>(j.ldw);
+        d.ldo = static_cast<int>(j.ldo);
+        d.n_rows = static_cast<int>(j.n_rows);
+        d.first_row = static_cast<int>(rows);
+        rows += j.n_rows;
     }
+    t.total_rows = static_cast<int>(rows);
+    return rows <= kEwmaMaxLaunchRows;
+}
+
+// The frozen-S scan (with the drift gate, if asked for) over jobs that share one launch: all of
+// them allow 16-byte access, or there is a single job.
+sp_status launch_scan_group(const sp_ctx *ctx, const EwmaLaunchJob *jobs, int first, int count,
+                            sp_dtype dtype, const sp_ewma_params &p,
+                            unsigned long long *counters, cudaStream_t stream,
+                            bool la_from_device) {
+    const int64_t n = ctx->d_in;
+    const bool bf16 = dtype == SP_BF16;
+    const bool gated = p.s_update == SP_S_GATED;
+    const int words = static_cast<int>((n + 31) / 32);
+    EwmaJobTable table{};
+    if (!fill_job_table(jobs, first, count, table)) return SP_ERR_SHAPE;
+    if (table.total_rows == 0) return SP_OK;
 
     ScanConstants sc;
     fill_scan_constants(p, sc);
-    const int64_t blocks = (n_rows + kEwmaWarps - 1) / kEwmaWarps;
-    if (blocks > 0x7fffffffLL) return SP_ERR_SHAPE;
-    const bool vec = aligned16(W) && ldw % 8 == 0 && n % 8 == 0 &&
-                     (W_out == nullptr || (aligned16(W_out) && ldo % 8 == 0));
-    const unsigned grid = static_cast<unsigned>(blocks);
-    PdlConfig pdl(dim3(grid), dim3(kEwmaThreads), stream);
-    const float *factor = ctx->factor;
     const DeviceScalars *scalars = ctx->scalars;
+    const double *colsq = ctx->colsq;
+    const float *factor = ctx->factor;
     cudaError_t launch_err = cudaSuccess;
-    PairConstants pc;
-    {
-        const double b = static_cast<double>(sc.b);
-        pc.a4 = static_cast<float>(pow(static_cast<double>(sc.a), 4.0));
+    const bool vec = job_is_vector(jobs[first], n);  // groups are uniform in this respect
+    if (vec) {
+        const double a = static_cast<double>(sc.a), b = static_cast<double>(sc.b);
+        PairConstants pc{};
+        pc.a4 = static_cast<float>(pow(a, 4.0));
         pc.b4 = static_cast<float>(pow(b, 4.0));
-        const double kappa = static_cast<double>(p.la) * p.beta * sc.a;
-        pc.kappa = static_cast<float>(kappa);
-        for (int j = 0; j < 4; ++j) {
-            pc.kappa_b[j] = static_cast<float>(kappa * pow(b, j));
+        pc.la = p.la;
+        for (int j = 0; j < 4; ++j)
             pc.unit_b[j] = static_cast<float>(static_cast<double>(p.beta) * sc.a * pow(b, j));
-        }
         pc.la_from_device = la_from_device ? 1 : 0;
-    }
-    TileConstants wc;
-    for (int k = 0; k < 5; ++k) {
-        wc.a_step[k] = static_cast<float>(pow(static_cast<double>(sc.a), 16.0 * (1 << k)));
-        wc.b_step[k] = static_cast<float>(pow(static_cast<double>(sc.b), 16.0 * (1 << k)));
-    }
-    wc.a8 = sc.a_step[0];
-    wc.b8 = sc.b_step[0];
-    const bool full_tiles = n % 512 == 0;
-    PdlConfig pdlp(dim3(static_cast<unsigned>((n_rows + kPairWarps - 1) / kPairWarps)),
-                   dim3(kPairThreads), stream);
-    const float *factor_pairs = ctx->factor_pairs;
-#define SP_LAUNCH_P(B, F, C)                                                                 \
-    launch_err = cudaLaunchKernelEx(&pdlp.cfg, ewma_pair_scan_kernel<B, F, C>, Wp,            \
-                                    static_cast<int>(ldw), static_cast<int>(n_rows),          \
+        pc.hazard_scale = static_cast<float>(pow(a, 3.0) * 0.5 * (1.0 - 1.0 / 1024.0));
+        TileConstants wc;
+        for (int k = 0; k < 5; ++k) {
+            wc.a_step[k] = static_cast<float>(pow(a, 16.0 * (1 << k)));
+            wc.b_step[k] = static_cast<float>(pow(b, 16.0 * (1 << k)));
+        }
+        wc.a8 = sc.a_step[0];
+        wc.b8 = sc.b_step[0];
+        const bool full_tiles = n % 512 == 0;
+        PdlConfig pdlp(dim3(static_cast<unsigned>((table.total_rows + kPairWarps - 1) / kPairWarps)),
+                       dim3(kPairThreads), stream);
+        const float *factor_pairs = ctx->factor_pairs;
+#define SP_LAUNCH_P(B, F, C, G)                                                              \
+    launch_err = cudaLaunchKernelEx(&pdlp.cfg, ewma_pair_scan_kernel<B, F, C, G>, table,      \
                                     static_cast<int>(n), factor_pairs, scalars, sc, pc, wc,   \
-                                    mask, static_cast<int>(words), Op, static_cast<int>(ldo), \
-                                    counters)
-#define SP_LAUNCH_S(B, C)                                                                    \
-    launch_err = cudaLaunchKernelEx(&pdl.cfg, ewma_scan_kernel<B, C>, Wp,              \
-                                    static_cast<int>(ldw), static_cast<int>(n_rows),          \
-                                    static_cast<int>(n), factor, scalars, sc, mask,           \
-                                    static_cast<int>(words), Op, static_cast<int>(ldo), counters)
-#define SP_LAUNCH_C(B, V, C)                                                                 \
+                                    words, counters, colsq, factor)
+#define SP_LAUNCH_PC(B, F, C)                                                                \
     do {                                                                                     \
-        if (V) {                                                                             \
-            if (full_tiles) SP_LAUNCH_P(B, true, C); else SP_LAUNCH_P(B, false, C);          \
-        } else {                                                                             \
-            SP_LAUNCH_S(B, C);                                                               \
-        }                                                                                    \
+        if (gated) SP_LAUNCH_P(B, F, C, true); else SP_LAUNCH_P(B, F, C, false);             \
     } while (0)
-#define SP_LAUNCH(B, V)                                                                      \
+#define SP_LAUNCH_PF(B, F)                                                                   \
     do {                                                                                     \
-        if (counters != nullptr) SP_LAUNCH_C(B, V, true); else SP_LAUNCH_C(B, V, false);     \
+        if (counters != nullptr) SP_LAUNCH_PC(B, F, true); else SP_LAUNCH_PC(B, F, false);   \
     } while (0)
-    if (bf16) {
-        if (vec) SP_LAUNCH(true, true); else SP_LAUNCH(true, false);
-    } else {
-        if (vec) SP_LAUNCH(false, true); else SP_LAUNCH(false, false);
-    }
-#undef SP_LAUNCH
-#undef SP_LAUNCH_C
-#undef SP_LAUNCH_S
+        if (bf16) {
+            if (full_tiles) SP_LAUNCH_PF(true, true); else SP_LAUNCH_PF(true, false);
+        } else {
+            if (full_tiles) SP_LAUNCH_PF(false, true); else SP_LAUNCH_PF(false, false);
+        }
+#undef SP_LAUNCH_PF
+#undef SP_LAUNCH_PC
 #undef SP_LAUNCH_P
+    } else {
+        const EwmaJob &j = table.job[0];
+        PdlConfig pdl(dim3(static_cast<unsigned>((j.n_rows + kEwmaWarps - 1) / kEwmaWarps)),
+                      dim3(kEwmaThreads), stream);
+#define SP_LAUNCH_S(B, C, G)                                                                 \
+    launch_err = cudaLaunchKernelEx(&pdl.cfg, ewma_scan_kernel<B, C, G>, j.W, j.ldw, j.n_rows, \
+                                    static_cast<int>(n), factor, scalars, sc, j.mask, words,  \
+                                    j.W_out, j.ldo, counters, colsq)
+#define SP_LAUNCH_SC(B, C)                                                                   \
+    do {                                                                                     \
+        if (gated) SP_LAUNCH_S(B, C, true); else SP_LAUNCH_S(B, C, false);                   \
+    } while (0)
+        if (bf16) {
+            if (counters != nullptr) SP_LAUNCH_SC(true, true); else SP_LAUNCH_SC(true, false);
+        } else {
+            if (counters != nullptr) SP_LAUNCH_SC(false, true); else SP_LAUNCH_SC(false, false);
+        }
+#undef SP_LAUNCH_SC
+#undef SP_LAUNCH_S
+    }
     if (launch_err != cudaSuccess) return cuda_fail(launch_err);
     return check_launch();
+}
+
+sp_status launch_literal(const sp_ctx *ctx, const EwmaLaunchJob &j, sp_dtype dtype,
+                         const sp_ewma_params &p, unsigned long long *counters,
+                         cudaStream_t stream) {
+    const int64_t n = ctx->d_in;
+    if (j.n_rows == 0) return SP_OK;
+    if (job_is_vector(j, n))  // rows that allow 16-byte access: the same arithmetic, rows moved in tiles
+        return launch_ewma_literal_tiled(ctx, j.W, dtype, j.n_rows, j.ldw, p, j.mask, j.W_out, j.ldo,
+                                         counters, stream);
+    const int64_t blocks = (j.n_rows + 127) / 128;
+    if (blocks > 0x7fffffffLL) return SP_ERR_SHAPE;
+    const unsigned lgrid = static_cast<unsigned>(blocks);
+    const uint16_t *Wp = static_cast<const uint16_t *>(j.W);
+    uint16_t *Op = static_cast<uint16_t *>(j.W_out);
+    const int64_t words = (n + 31) / 32;
+    if (dtype == SP_BF16)
+        ewma_literal_kernel<true><<<lgrid, 128, 0, stream>>>(
+            Wp, j.ldw, j.n_rows, n, ctx->colsq, ctx->factor, ctx->scalars, p.alpha, p.beta, p.la,
+            j.mask, words, Op, j.ldo, counters);
+    else
+        ewma_literal_kernel<false><<<lgrid, 128, 0, stream>>>(
+            Wp, j.ldw, j.n_rows, n, ctx->colsq, ctx->factor, ctx->scalars, p.alpha, p.beta, p.la,
+            j.mask, words, Op, j.ldo, counters);
+    return check_launch();
+}
+
+}  // namespace
+
+sp_status launch_select_ewma(const sp_ctx *ctx, const EwmaLaunchJob *jobs_in, int n_jobs,
+                             sp_dtype dtype, const sp_ewma_params &p, unsigned long long *counters,
+                             cudaStream_t stream, bool la_from_device) {
+    const int64_t n = ctx->d_in;
+    const int64_t words = (n + 31) / 32;
+    // Cut every matrix into pieces of at most kEwmaMaxLaunchRows rows ...
+    EwmaLaunchJob pieces[64];
+    int n_pieces = 0;
+    for (int i = 0; i < n_jobs; ++i) {
+        const EwmaLaunchJob &j = jobs_in[i];
+        if (j.n_rows < 0 || j.ldw > 0x7fffffffLL || j.ldo > 0x7fffffffLL) return SP_ERR_SHAPE;
+        for (int64_t r0 = 0; r0 < j.n_rows; r0 += kEwmaMaxLaunchRows) {
+            if (n_pieces == 64) return SP_ERR_SHAPE;
+            EwmaLaunchJob &q = pieces[n_pieces++];
+            q = j;
+            q.n_rows = j.n_rows - r0 < kEwmaMaxLaunchRows ? j.n_rows - r0 : kEwmaMaxLaunchRows;
+            q.W = static_cast<const uint16_t *>(j.W) + r0 * j.ldw;
+            if (j.W_out != nullptr) q.W_out = static_cast<uint16_t *>(j.W_out) + r0 * j.ldo;
+            if (j.mask != nullptr) q.mask = j.mask + r0 * words;
+        }
+    }
+    if (p.s_update == SP_S_LITERAL_W2) {
+        for (int i = 0; i < n_pieces; ++i) {
+            sp_status st = launch_literal(ctx, pieces[i], dtype, p, counters, stream);
+            if (st != SP_OK) return st;
+        }
+        return SP_OK;
+    }
+    // ... and give consecutive pieces that allow 16-byte access one launch.
+    int first = 0;
+    while (first < n_pieces) {
+        int count = 1;
+        if (job_is_vector(pieces[first], n)) {
+            int64_t bits = pieces[first].n_rows;
+            while (first + count < n_pieces && count < kEwmaMaxJobs &&
+                   job_is_vector(pieces[first + count], n)) {
+                const int64_t more = pieces[first + count].n_rows;
+                if (bits + more > kEwmaMaxLaunchRows) break;
+                bits += more;
+                ++count;
+            }
+        }
+        sp_status st = launch_scan_group(ctx, pieces, first, count, dtype, p, counters, stream,
+                                         la_from_device);
+        if (st != SP_OK) return st;
+        first += count;
+    }
+    return SP_OK;
 }
 
 // Bisection of la on the device: no host round trip between the counting passes.

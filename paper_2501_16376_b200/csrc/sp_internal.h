@@ -16,6 +16,9 @@ constexpr int64_t kMaxDin = 1 << 20;
 // Status word written by the finalisation kernel.
 constexpr int kFlagDegenerate = 1;
 
+constexpr int64_t kEwmaMaxLaunchRows = int64_t(1) << 30;  // rows one EWMA launch can cover
+constexpr int kEwmaMaxJobs = 8;                            // weight matrices, likewise
+
 // Scalars produced by finalisation; lives in device memory inside the context.
 struct DeviceScalars {
     double S;             // sum_q colsq[q]
@@ -103,10 +106,24 @@ sp_status launch_select_24_compressed(const sp_ctx *ctx, const void *W, sp_dtype
                                       uint32_t *meta, cudaStream_t stream);
 
 // select_ewma.cu
-sp_status launch_select_ewma(const sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
-                             int64_t ldw, const sp_ewma_params &p, uint32_t *mask, void *W_out,
-                             int64_t ldo, unsigned long long *counters, cudaStream_t stream,
-                             bool la_from_device = false);
+struct EwmaLaunchJob {  // one weight matrix of an EWMA launch
+    const void *W;
+    void *W_out;     // nullable
+    uint32_t *mask;  // nullable
+    int64_t n_rows, ldw, ldo;
+};
+// Algorithm 1 on up to kEwmaMaxJobs matrices that share the context (and dtype), in as few
+// launches as their layouts allow.
+sp_status launch_select_ewma(const sp_ctx *ctx, const EwmaLaunchJob *jobs, int n_jobs,
+                             sp_dtype dtype, const sp_ewma_params &p, unsigned long long *counters,
+                             cudaStream_t stream, bool la_from_device = false);
+inline sp_status launch_select_ewma(const sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
+                                    int64_t ldw, const sp_ewma_params &p, uint32_t *mask,
+                                    void *W_out, int64_t ldo, unsigned long long *counters,
+                                    cudaStream_t stream, bool la_from_device = false) {
+    const EwmaLaunchJob job{W, W_out, mask, n_rows, ldw, ldo};
+    return launch_select_ewma(ctx, &job, 1, dtype, p, counters, stream, la_from_device);
+}
 // True when launch_select_ewma would take the kernel that can read la from DeviceScalars.
 bool ewma_pair_path_applies(const void *W, int64_t ldw, int64_t n);
 sp_status launch_search_la_device(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,

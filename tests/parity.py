@@ -12,6 +12,14 @@ SCORE_RTOL = 1e-5     # statistics and scores: relative tolerance
 BAND_RTOL = 1e-5      # a mask bit may differ only if the oracle score is this close to its threshold
 FLIP_FRACTION = 1e-6  # and at most this fraction of the entries may differ
 
+# Flip budget.  Two correct binary32 evaluations of the running threshold (the oracle's
+# sequential one, the kernels' scans) differ by a few 1e-7 relative, so an entry that sits
+# inside the band flips now and then: about 0.4e-6 of all entries.  A case with fewer than 1e6
+# entries cannot hold the fraction 1e-6 other than as "no flip at all", which no re-associated
+# evaluation can promise; such a case is allowed one in-band flip, and every flip is added to
+# this tally, whose total is held to FLIP_FRACTION by tests/test_gpu_z_flip_budget.py.
+FLIP_TALLY = {"flips": 0, "entries": 0, "cases": 0}
+
 
 def bits(t: torch.Tensor) -> np.ndarray:
     """uint16 bit patterns of a 16-bit float tensor (copied to the host)."""
@@ -72,8 +80,11 @@ def check_selection(gpu_mask: torch.Tensor, gpu_out: torch.Tensor, W: torch.Tens
         assert flips == 0, "mask differs in %d entries" % flips
     else:
         assert not (diff & ~allowed).any(), "mask differs outside the threshold band"
-        assert flips <= FLIP_FRACTION * diff.size, \
-            "%d flips in %d entries (limit %.3g)" % (flips, diff.size, FLIP_FRACTION * diff.size)
+        limit = max(1.0, FLIP_FRACTION * diff.size)
+        assert flips <= limit, "%d flips in %d entries (limit %.3g)" % (flips, diff.size, limit)
+        FLIP_TALLY["flips"] += flips
+        FLIP_TALLY["entries"] += int(diff.size)
+        FLIP_TALLY["cases"] += 1
     # mask words carry no bits past n
     words = mask_np(gpu_mask)
     if n % 32:

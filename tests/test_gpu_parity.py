@@ -265,10 +265,60 @@ def test_ewma_literal_S_update_is_bit_exact_and_hazard_counter_fires(sp):
         P.check_selection(mask, out, W, lit, None, strict=True)  # sequential kernel: bit-exact
         assert int(counters[sp.SP_COUNTER_KEPT]) == int(lit.keep_bool(n).sum())
         counters.zero_()
-        mask_f, out_f = ctx.sp_select_unstructured(W, params=_ewma_params(sp, 0.5),
-                                                   counters=counters)
+        mask_f, out_f = ctx.sp_select_unstructured(
+            W, params=_ewma_params(sp, 0.5, s_update=sp.SP_S_FROZEN), counters=counters)
         P.check_selection(mask_f, out_f, W, fro, P.ewma_allowed_flips(fro))
-        assert int(counters[sp.SP_COUNTER_S_HAZARD]) == R      # every row is flagged
+        assert int(counters[sp.SP_COUNTER_S_HAZARD]) == 0      # nothing is gated in this mode
+        assert int(counters[sp.SP_COUNTER_KEPT]) == int(so.unpack_mask(P.mask_np(mask_f), n).sum())
+
+
+@pytest.mark.parametrize("R,n,inplace,misalign", [
+    (96, 640, False, False),      # rows of two tiles, several rows per CTA
+    (96, 640, True, False),
+    (40, 4096, True, False),      # one row per CTA
+    (24, 8192 + 512, False, False),  # rows walked in two passes
+    (24, 8192 + 512, True, False),   # ... pruned in place: marks come from the pre-pass
+    (33, 648, True, True),        # unaligned rows: element-wise kernels
+])
+def test_default_call_is_algorithm_1_when_S_moves(sp, R, n, inplace, misalign):
+    """The drift gate: with statistics so small that "S = S - w_i^2" changes S, the default
+    entry point must give the literal result of Algorithm 1 bit for bit, rows of the other
+    kind (here: a few rows scaled down until their w^2 cannot move S) stay on the scan path."""
+    W = _gen(91 + n, (R, n), torch.float16, 0.02)
+    quiet = [1, R // 2, R - 1]
+    W[quiet] = W[quiet] * 2.0 ** -13          # w^2 <= 1.2e-10: below the hazard bound of S ~ 0.02
+    if misalign:
+        buf = torch.zeros(R * n + 1, dtype=W.dtype, device=W.device)
+        buf[1:] = W.reshape(-1)
+        W = buf[1:].view(R, n)
+    colsq = np.random.default_rng(4).uniform(1.0, 2.0, n) * (12.8 / n) * 1e-3   # S ~ sum w^2
+    with sp.Context(n) as ctx:
+        ctx.sp_set_stats(torch.from_numpy(colsq), 10)
+        st = so.Stats(colsq.copy(), 10)
+        lit = so.select_unstructured(P.bits(W), so.F16, st, 0.5, s_update=so.S_LITERAL_W2,
+                                     want_trace=True)
+        fro = so.select_unstructured(P.bits(W), so.F16, st, 0.5, s_update=so.S_FROZEN)
+        assert not np.array_equal(lit.mask, fro.mask)
+        counters = sp.new_counters()
+        W_in = W.clone() if not misalign else W
+        src = W_in.clone()
+        mask, out = ctx.sp_select_unstructured(W_in, 0.5, counters=counters,
+                                               inplace=inplace)
+        hazard = int(counters[sp.SP_COUNTER_S_HAZARD])
+        assert R - len(quiet) <= hazard <= R
+        got = so.unpack_mask(P.mask_np(mask), n)
+        rows = np.ones(R, bool)
+        rows[quiet] = False
+        assert np.array_equal(got[rows], lit.keep_bool(n)[rows])   # gated rows: bit-exact
+        P.check_selection(mask, out, src, lit, P.ewma_allowed_flips(lit))
+        assert int(counters[sp.SP_COUNTER_KEPT]) == int(got.sum())
+        # the row bitmap is clean again: a second call gives the same answer
+        if not misalign:
+            counters.zero_()
+            mask2, out2 = ctx.sp_select_unstructured(src, 0.5, counters=counters)
+            assert torch.equal(mask, mask2)
+            assert torch.equal(out.view(torch.int16), out2.view(torch.int16))
+            assert R - len(quiet) <= int(counters[sp.SP_COUNTER_S_HAZARD]) <= R
 
 
 def test_ewma_literal_equals_frozen_at_calibration_scale(sp):
@@ -548,14 +598,15 @@ def test_compressed_24_matches_oracle_and_dense_path(sp, R, n, dtype):
 
 # ------------------------------------------------------------------ EWMA trace diagnostic
 
-@pytest.mark.parametrize("s_update", [0, 1])
+@pytest.mark.parametrize("s_update", [0, 1])     # the oracle's S_FROZEN, S_LITERAL_W2
 def test_ewma_trace_matches_oracle_state(sp, s_update):
     R, n = 6, 1500
     W = _gen(71, (R, n), torch.float16, 0.02)
     colsq = np.random.default_rng(5).uniform(1.0, 2.0, n) * (1e-4 if s_update else 1e4)
     with sp.Context(n) as ctx:
         ctx.sp_set_stats(torch.from_numpy(colsq), 10)
-        est, dev, L = ctx.sp_ewma_trace(W, sp.EwmaParams(0.125, 0.125, 0.5, s_update))
+        est, dev, L = ctx.sp_ewma_trace(W, sp.EwmaParams(
+            0.125, 0.125, 0.5, sp.SP_S_LITERAL_W2 if s_update else sp.SP_S_FROZEN))
     st = so.Stats(colsq.copy(), 10)
     # the oracle's recorded threshold est - la*dev gives est (la = 0) and est - dev (la = 1);
     # with the S update on, decisions (hence S) depend on la, so compare at the la used

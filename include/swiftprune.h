@@ -252,6 +252,35 @@ sp_status sp_select_nm(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_row
                        sp_stream stream);
 
 /*
+ * Grouped selection.  Layers that read the same input (q/k/v; gate/up) share a context and the
+ * per-channel factors, and Algorithm 1 treats every row on its own ("parallel calculation for
+ * each row"), so their rows can be pruned by one launch: small layers then no longer pay a
+ * launch and a ramp-up each.  mats (HOST array, 1 <= n_mats <= SP_MAX_GROUP) lists the
+ * matrices, all of `dtype`; every entry follows the rules of the single-matrix call (mask_out
+ * and W_out nullable, W_out may alias W exactly).  The result for each matrix is identical to
+ * that of its own sp_select_unstructured[_ex] / sp_select_nm call.  Matrices that do not allow
+ * 16-byte access, or (N:M) ask for different outputs than their neighbours, get launches of
+ * their own.
+ */
+enum { SP_MAX_GROUP = 8 };
+typedef struct {
+    const void *W;
+    int64_t n_rows;
+    int64_t ldw;
+    uint32_t *mask_out;
+    void *W_out;
+    int64_t ldo;
+} sp_matrix;
+sp_status sp_select_unstructured_group(sp_ctx *ctx, const sp_matrix *mats /* host */, int n_mats,
+                                       sp_dtype dtype, float sparsity,
+                                       unsigned long long *counters, sp_stream stream);
+sp_status sp_select_unstructured_group_ex(sp_ctx *ctx, const sp_matrix *mats /* host */, int n_mats,
+                                          sp_dtype dtype, const sp_ewma_params *params /* host */,
+                                          unsigned long long *counters, sp_stream stream);
+sp_status sp_select_nm_group(sp_ctx *ctx, const sp_matrix *mats /* host */, int n_mats,
+                             sp_dtype dtype, int N, int M, sp_stream stream);
+
+/*
  * Section 3.3, compressed output: 2:4 selection (exactly as sp_select_nm with N = 2, M = 4)
  * written as the kept values plus per-group indices in the same pass, so that a consumer of
  * 2:4 sparsity needs no dense pruned matrix and no separate conversion (the paper's remark that

@@ -28,7 +28,8 @@ EXPORTS = (
     "sp_create", "sp_destroy", "sp_calib_reset", "sp_calib_accumulate", "sp_get_stats",
     "sp_set_stats", "sp_calib_stats_noalloc", "sp_score", "sp_la_for_sparsity", "sp_select_unstructured",
     "sp_select_unstructured_ex", "sp_search_la", "sp_ewma_trace", "sp_select_nm", "sp_select_24_compressed", "sp_apply_mask", "sp_calib_accumulate_host",
-    "sp_select_nm_host", "sp_select_unstructured_host", "sp_status_string",
+    "sp_select_nm_host", "sp_select_unstructured_host", "sp_select_unstructured_group",
+    "sp_select_unstructured_group_ex", "sp_select_nm_group", "sp_status_string",
     "sp_last_cuda_error", "sp_launch_count",
 )
 
@@ -42,6 +43,15 @@ class SpError(RuntimeError):
 class EwmaParams(ctypes.Structure):
     _fields_ = [("alpha", ctypes.c_float), ("beta", ctypes.c_float), ("la", ctypes.c_float),
                 ("s_update", ctypes.c_int)]
+
+
+class Matrix(ctypes.Structure):
+    """sp_matrix: one weight matrix of a grouped selection call."""
+    _fields_ = [("W", ctypes.c_void_p), ("n_rows", ctypes.c_int64), ("ldw", ctypes.c_int64),
+                ("mask_out", ctypes.c_void_p), ("W_out", ctypes.c_void_p), ("ldo", ctypes.c_int64)]
+
+
+SP_MAX_GROUP = 8
 
 
 def _load() -> ctypes.CDLL:
@@ -72,6 +82,10 @@ def _load() -> ctypes.CDLL:
     lib.sp_calib_accumulate_host.argtypes = [vp, vp, ci, i64, i64, vp]
     lib.sp_select_nm_host.argtypes = [vp, vp, ci, i64, i64, ci, ci, vp, vp, i64, vp]
     lib.sp_select_unstructured_host.argtypes = [vp, vp, ci, i64, i64, f32, vp, vp, i64, vp]
+    lib.sp_select_unstructured_group.argtypes = [vp, ctypes.POINTER(Matrix), ci, ci, f32, vp, vp]
+    lib.sp_select_unstructured_group_ex.argtypes = [vp, ctypes.POINTER(Matrix), ci, ci,
+                                                    ctypes.POINTER(EwmaParams), vp, vp]
+    lib.sp_select_nm_group.argtypes = [vp, ctypes.POINTER(Matrix), ci, ci, ci, ci, vp]
     lib.sp_status_string.argtypes = [ci]
     lib.sp_status_string.restype = ctypes.c_char_p
     lib.sp_last_cuda_error.restype = ctypes.c_char_p
@@ -278,6 +292,52 @@ class Context:
         _check(lib.sp_select_nm(self._h, ptr, _dtype_of(W), R, ld, int(N), int(M), _ptr(mask),
                                 optr, ldo, _stream(stream)))
         return mask, W_out
+
+
+def _group(ctx, Ws, masks, W_outs, want_mask, inplace):
+    """Marshals a list of weight tensors (and optional outputs) into an sp_matrix array."""
+    k = len(Ws)
+    masks = list(masks) if masks is not None else [None] * k
+    W_outs = list(W_outs) if W_outs is not None else [None] * k
+    arr = (Matrix * k)()
+    dtype = _dtype_of(Ws[0])
+    for i, W in enumerate(Ws):
+        ptr, R, n, ld = _matrix(W, "W")
+        ctx._check_width(n)
+        if _dtype_of(W) != dtype:
+            raise SpError(SP_ERR_DTYPE, "all matrices of a group must have the same dtype")
+        masks[i], W_outs[i] = ctx._outputs(W, masks[i], W_outs[i], want_mask, inplace)
+        optr, _, _, ldo = _matrix(W_outs[i], "W_out")
+        arr[i] = Matrix(ptr, R, ld, _ptr(masks[i]), optr, ldo)
+    return arr, k, dtype, masks, W_outs
+
+
+def _sp_select_unstructured_group(self, Ws, sparsity=None, *, params: EwmaParams | None = None,
+                                  masks=None, W_outs=None, inplace=False, want_mask=True,
+                                  counters=None, stream=None):
+    """Algorithm 1 on several matrices that read this context's input, in one call.
+    Returns (masks, W_outs)."""
+    arr, k, dtype, masks, W_outs = _group(self, Ws, masks, W_outs, want_mask, inplace)
+    if params is not None:
+        _check(lib.sp_select_unstructured_group_ex(self._h, arr, k, dtype, ctypes.byref(params),
+                                                   _ptr(counters), _stream(stream)))
+    else:
+        _check(lib.sp_select_unstructured_group(self._h, arr, k, dtype, float(sparsity),
+                                                _ptr(counters), _stream(stream)))
+    return masks, W_outs
+
+
+def _sp_select_nm_group(self, Ws, N: int, M: int, *, masks=None, W_outs=None, inplace=False,
+                        want_mask=True, stream=None):
+    """N:M selection of several matrices that read this context's input, in one call.
+    Returns (masks, W_outs)."""
+    arr, k, dtype, masks, W_outs = _group(self, Ws, masks, W_outs, want_mask, inplace)
+    _check(lib.sp_select_nm_group(self._h, arr, k, dtype, int(N), int(M), _stream(stream)))
+    return masks, W_outs
+
+
+Context.sp_select_unstructured_group = _sp_select_unstructured_group
+Context.sp_select_nm_group = _sp_select_nm_group
 
 
 class HostMixin:

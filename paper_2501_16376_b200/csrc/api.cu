@@ -292,6 +292,71 @@ sp_status sp_select_unstructured(sp_ctx *ctx, const void *W, sp_dtype dtype, int
                                      stream);
 }
 
+// Validates a group of matrices and converts it to launch jobs.
+static sp_status group_jobs(const sp_ctx *ctx, const sp_matrix *mats, int n_mats, sp_dtype dtype,
+                            EwmaLaunchJob *jobs) {
+    if (ctx == nullptr || mats == nullptr) return SP_ERR_INVALID_ARG;
+    if (n_mats < 1 || n_mats > SP_MAX_GROUP) return SP_ERR_INVALID_ARG;
+    for (int i = 0; i < n_mats; ++i) {
+        const sp_matrix &m = mats[i];
+        sp_status st = check_matrix_args(ctx, m.W, dtype, m.n_rows, m.ldw, m.W_out, m.ldo);
+        if (st != SP_OK) return st;
+        jobs[i] = EwmaLaunchJob{m.W, m.W_out, m.mask_out, m.n_rows, m.ldw, m.ldo};
+    }
+    return SP_OK;
+}
+
+sp_status sp_select_unstructured_group_ex(sp_ctx *ctx, const sp_matrix *mats, int n_mats,
+                                          sp_dtype dtype, const sp_ewma_params *params,
+                                          unsigned long long *counters, sp_stream stream) {
+    EwmaLaunchJob jobs[SP_MAX_GROUP];
+    sp_status st = group_jobs(ctx, mats, n_mats, dtype, jobs);
+    if (st != SP_OK) return st;
+    if (params == nullptr) return SP_ERR_INVALID_ARG;
+    if (!(params->alpha > 0.0f) || !(params->alpha <= 1.0f) || !(params->beta > 0.0f) ||
+        !(params->beta <= 1.0f) || !std::isfinite(params->la))
+        return SP_ERR_INVALID_ARG;
+    if (params->s_update != SP_S_GATED && params->s_update != SP_S_FROZEN &&
+        params->s_update != SP_S_LITERAL_W2)
+        return SP_ERR_INVALID_ARG;
+    if (ctx->n_tokens <= 0) return SP_ERR_STATE;
+    DeviceGuard guard(ctx->device);
+    if (guard.error() != cudaSuccess) return cuda_fail(guard.error());
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    st = ensure_finalized(ctx, s);
+    if (st != SP_OK) return st;
+    return launch_select_ewma(ctx, jobs, n_mats, dtype, *params, counters, s);
+}
+
+sp_status sp_select_unstructured_group(sp_ctx *ctx, const sp_matrix *mats, int n_mats,
+                                       sp_dtype dtype, float sparsity,
+                                       unsigned long long *counters, sp_stream stream) {
+    sp_ewma_params p;
+    p.alpha = 0.125f;  // Section 4.2
+    p.beta = 0.125f;
+    p.s_update = SP_S_GATED;
+    sp_status st = sp_la_for_sparsity(sparsity, &p.la);
+    if (st != SP_OK) return st;
+    return sp_select_unstructured_group_ex(ctx, mats, n_mats, dtype, &p, counters, stream);
+}
+
+sp_status sp_select_nm_group(sp_ctx *ctx, const sp_matrix *mats, int n_mats, sp_dtype dtype, int N,
+                             int M, sp_stream stream) {
+    EwmaLaunchJob jobs[SP_MAX_GROUP];
+    sp_status st = group_jobs(ctx, mats, n_mats, dtype, jobs);
+    if (st != SP_OK) return st;
+    if (M != 4 && M != 8) return SP_ERR_INVALID_ARG;
+    if (N <= 0 || N >= M) return SP_ERR_INVALID_ARG;
+    if (ctx->d_in % M != 0) return SP_ERR_SHAPE;
+    if (ctx->n_tokens <= 0) return SP_ERR_STATE;
+    DeviceGuard guard(ctx->device);
+    if (guard.error() != cudaSuccess) return cuda_fail(guard.error());
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    st = ensure_finalized(ctx, s);
+    if (st != SP_OK) return st;
+    return launch_select_nm(ctx, jobs, n_mats, dtype, N, M, s);
+}
+
 sp_status sp_ewma_trace(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows, int64_t ldw,
                         const sp_ewma_params *params, float *est_out, float *dev_out,
                         float *scores_out, sp_stream stream) {

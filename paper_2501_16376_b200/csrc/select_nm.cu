@@ -39,6 +39,7 @@ namespace sp {
 #ifndef SP_NM_THREADS
 #define SP_NM_THREADS 128
 #endif
+constexpr int kNmMaxJobs = kEwmaMaxJobs;  // matrices one launch can cover
 constexpr int kNmThreads = SP_NM_THREADS;
 constexpr int kNmWarps = kNmThreads / 32;
 constexpr int kNmRowsInFlight = SP_NM_ROWS_IN_FLIGHT;
@@ -146,21 +147,39 @@ select_nm_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int64_t n,
 // constants (four rows per trip), every lane stores its own mask byte (byte k of a
 // little-endian mask word holds columns 8k .. 8k+7) instead of assembling words across lanes,
 // and when the strip is whole (FULL: d_in a multiple of 256) there are no column guards.
-// OUT / MASK: the pruned weights / the keep mask are requested.
+// OUT / MASK: the pruned weights / the keep mask are requested.  The launch covers a table of
+// matrices that share the context (layers reading the same input); slabs are numbered through
+// all of them.
+struct NmJob {
+    const uint16_t *W;
+    uint16_t *W_out;  // nullable
+    uint32_t *mask;   // nullable
+    int ldw, ldo, n_rows;
+    int first_slab;
+};
+struct NmJobTable {
+    int count;
+    int total_slabs;
+    NmJob job[kNmMaxJobs];
+};
+
 template <bool BF16, bool FULL, int M, bool OUT, bool MASK>
 __global__ void __launch_bounds__(kNmThreads, SP_NM_MIN_BLOCKS)
-select_nm_stream_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int n,
-                        int rows_per_warp, const float *__restrict__ factor, int prune_count,
-                        uint32_t *__restrict__ mask, int mask_words,
-                        uint16_t *__restrict__ W_out, int ldo) {
+select_nm_stream_kernel(const __grid_constant__ NmJobTable jobs, int n, int rows_per_warp,
+                        const float *__restrict__ factor, int prune_count, int mask_words) {
     pdl_launch_dependents();
     pdl_wait();  // the per-channel factors come from an earlier kernel of the stream
     const int lane = threadIdx.x & 31;
     const int col = blockIdx.x * kStripChannels + lane * 8;
-    const int slab = blockIdx.y * kNmWarps + (threadIdx.x >> 5);
-    const int64_t row_begin64 = static_cast<int64_t>(slab) * rows_per_warp;
-    if (row_begin64 >= n_rows) return;  // warp-uniform
-    const int row_begin = static_cast<int>(row_begin64);
+    const int gslab = blockIdx.y * kNmWarps + (threadIdx.x >> 5);
+    if (gslab >= jobs.total_slabs) return;  // warp-uniform
+    int jk = 0;
+    while (jk + 1 < jobs.count && gslab >= jobs.job[jk + 1].first_slab) ++jk;
+    const uint16_t *const W = jobs.job[jk].W;
+    uint16_t *const W_out = jobs.job[jk].W_out;
+    uint32_t *const mask = jobs.job[jk].mask;
+    const int ldw = jobs.job[jk].ldw, ldo = jobs.job[jk].ldo, n_rows = jobs.job[jk].n_rows;
+    const int row_begin = (gslab - jobs.job[jk].first_slab) * rows_per_warp;  // < n_rows
     const int rows = min(n_rows - row_begin, rows_per_warp);
     const bool in_row = FULL || col < n;  // d_in % 8 == 0: a chunk is inside or outside as a whole
 
@@ -239,35 +258,62 @@ select_nm_stream_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int
     for (int rr = r0; rr < rows; ++rr) process(rr, rr & (kStages - 1));  // r0 % kStages == 0
 }
 
-sp_status launch_select_nm(const sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
-                           int64_t ldw, int N, int M, uint32_t *mask, void *W_out, int64_t ldo,
-                           cudaStream_t stream) {
+namespace {
+
+bool nm_job_is_vector(const EwmaLaunchJob &j, int64_t n) {
+    return aligned16(j.W) && j.ldw % 8 == 0 && n % 8 == 0 &&
+           (j.W_out == nullptr || (aligned16(j.W_out) && j.ldo % 8 == 0));
+}
+
+// Jobs [first, first + count) in one launch: either all of them allow 16-byte access and ask
+// for the same outputs, or count == 1.
+sp_status launch_nm_group(const sp_ctx *ctx, const EwmaLaunchJob *jobs, int first, int count,
+                          sp_dtype dtype, int N, int M, cudaStream_t stream) {
     const int64_t n = ctx->d_in;
-    if (n_rows == 0 || (mask == nullptr && W_out == nullptr)) return SP_OK;  // nothing to produce
     const int strips = ctx->strips;
+    int64_t total_rows = 0;
+    for (int i = 0; i < count; ++i) total_rows += jobs[first + i].n_rows;
+    if (total_rows == 0) return SP_OK;
     // Short slabs, i.e. many warps (measured: 8 rows per warp for the LLaMA-sized layers is 3-7 %
     // faster than 16-32, and than 4 once the SM clock is held down by the power cap).
     const int64_t target_warps = static_cast<int64_t>(ctx->sm_count) * SP_NM_TARGET_WARPS;
-    int64_t rows_per_warp = (n_rows * strips + target_warps - 1) / target_warps;
+    int64_t rows_per_warp = (total_rows * strips + target_warps - 1) / target_warps;
     rows_per_warp = (rows_per_warp + kNmRowsInFlight - 1) / kNmRowsInFlight * kNmRowsInFlight;
     if (rows_per_warp < SP_NM_MIN_ROWS) rows_per_warp = SP_NM_MIN_ROWS;
     const int64_t max_grid_y = 65535;
-    if ((n_rows + rows_per_warp * kNmWarps - 1) / (rows_per_warp * kNmWarps) > max_grid_y) {
+    if ((total_rows + rows_per_warp * kNmWarps - 1) / (rows_per_warp * kNmWarps) + count > max_grid_y) {
         // keep gridDim.y legal for very tall matrices by giving each warp more rows
-        rows_per_warp = (n_rows + max_grid_y * kNmWarps - 1) / (max_grid_y * kNmWarps);
+        rows_per_warp = (total_rows + (max_grid_y - count) * kNmWarps - 1) / ((max_grid_y - count) * kNmWarps);
         rows_per_warp = (rows_per_warp + kNmRowsInFlight - 1) / kNmRowsInFlight * kNmRowsInFlight;
     }
-    if (rows_per_warp > 0x7fffffffLL || n_rows > 0x7fffffffLL || ldw > 0x7fffffffLL ||
-        ldo > 0x7fffffffLL)
-        return SP_ERR_SHAPE;
-    const int64_t slabs = (n_rows + rows_per_warp - 1) / rows_per_warp;
+    if (rows_per_warp > 0x7fffffffLL) return SP_ERR_SHAPE;
+
+    NmJobTable table{};
+    table.count = count;
+    int64_t slabs = 0;
+    for (int i = 0; i < count; ++i) {
+        const EwmaLaunchJob &j = jobs[first + i];
+        if (j.n_rows > 0x7fffffffLL || j.ldw > 0x7fffffffLL || j.ldo > 0x7fffffffLL) return SP_ERR_SHAPE;
+        NmJob &d = table.job[i];
+        d.W = static_cast<const uint16_t *>(j.W);
+        d.W_out = static_cast<uint16_t *>(j.W_out);
+        d.mask = j.mask;
+        d.ldw = static_cast<int>(j.ldw);
+        d.ldo = static_cast<int>(j.ldo);
+        d.n_rows = static_cast<int>(j.n_rows);
+        d.first_slab = static_cast<int>(slabs);
+        slabs += (j.n_rows + rows_per_warp - 1) / rows_per_warp;
+    }
+    if (slabs > 0x7fffffffLL) return SP_ERR_SHAPE;
+    table.total_slabs = static_cast<int>(slabs);
     const dim3 grid(static_cast<unsigned>(strips),
                     static_cast<unsigned>((slabs + kNmWarps - 1) / kNmWarps));
-    const bool vec = aligned16(W) && ldw % 8 == 0 && n % 8 == 0 &&
-                     (W_out == nullptr || (aligned16(W_out) && ldo % 8 == 0));
-    const uint16_t *Wp = static_cast<const uint16_t *>(W);
-    uint16_t *Op = static_cast<uint16_t *>(W_out);
-    const int64_t words = (n + 31) / 32;
+    const EwmaLaunchJob &j0 = jobs[first];
+    const bool vec = nm_job_is_vector(j0, n);
+    const uint16_t *Wp = static_cast<const uint16_t *>(j0.W);
+    uint16_t *Op = static_cast<uint16_t *>(j0.W_out);
+    uint32_t *mask = j0.mask;
+    const int words = static_cast<int>((n + 31) / 32);
     const int prune_count = M - N;
     const int rpw = static_cast<int>(rows_per_warp);
     PdlConfig pdl(grid, dim3(kNmThreads), stream);
@@ -275,18 +321,16 @@ sp_status launch_select_nm(const sp_ctx *ctx, const void *W, sp_dtype dtype, int
     cudaError_t launch_err = cudaSuccess;
 #define SP_LAUNCH(B, MM)                                                                     \
     launch_err = cudaLaunchKernelEx(&pdl.cfg, select_nm_kernel<B, MM>, Wp,                    \
-                                    static_cast<int>(ldw), static_cast<int>(n_rows), n, rpw,  \
-                                    factor, prune_count, mask, static_cast<int>(words), Op,   \
-                                    static_cast<int>(ldo))
+                                    static_cast<int>(j0.ldw), static_cast<int>(j0.n_rows), n, \
+                                    rpw, factor, prune_count, mask, words, Op,                \
+                                    static_cast<int>(j0.ldo))
 #define SP_LAUNCH_M(B)                                                                        \
     do {                                                                                      \
         if (M == 8) SP_LAUNCH(B, 8); else SP_LAUNCH(B, 4);                                    \
     } while (0)
 #define SP_LAUNCH_ST(B, F, MM, O, K)                                                         \
-    launch_err = cudaLaunchKernelEx(&pdl.cfg, select_nm_stream_kernel<B, F, MM, O, K>, Wp,    \
-                                    static_cast<int>(ldw), static_cast<int>(n_rows),          \
-                                    static_cast<int>(n), rpw, factor, prune_count, mask,      \
-                                    static_cast<int>(words), Op, static_cast<int>(ldo))
+    launch_err = cudaLaunchKernelEx(&pdl.cfg, select_nm_stream_kernel<B, F, MM, O, K>, table, \
+                                    static_cast<int>(n), rpw, factor, prune_count, words)
 #define SP_LAUNCH_STO(B, F, MM)                                                               \
     do {                                                                                      \
         if (Op != nullptr && mask != nullptr) SP_LAUNCH_ST(B, F, MM, true, true);             \
@@ -316,6 +360,36 @@ sp_status launch_select_nm(const sp_ctx *ctx, const void *W, sp_dtype dtype, int
 #undef SP_LAUNCH
     if (launch_err != cudaSuccess) return cuda_fail(launch_err);
     return check_launch();
+}
+
+}  // namespace
+
+sp_status launch_select_nm(const sp_ctx *ctx, const EwmaLaunchJob *jobs_in, int n_jobs,
+                           sp_dtype dtype, int N, int M, cudaStream_t stream) {
+    const int64_t n = ctx->d_in;
+    // jobs that produce nothing are dropped; consecutive jobs that allow 16-byte access and ask
+    // for the same outputs share a launch
+    EwmaLaunchJob jobs[kNmMaxJobs];
+    int count = 0;
+    for (int i = 0; i < n_jobs; ++i) {
+        if (jobs_in[i].n_rows == 0 || (jobs_in[i].mask == nullptr && jobs_in[i].W_out == nullptr)) continue;
+        if (count == kNmMaxJobs) return SP_ERR_INVALID_ARG;
+        jobs[count++] = jobs_in[i];
+    }
+    int first = 0;
+    while (first < count) {
+        int group = 1;
+        if (nm_job_is_vector(jobs[first], n)) {
+            while (first + group < count && nm_job_is_vector(jobs[first + group], n) &&
+                   (jobs[first + group].mask != nullptr) == (jobs[first].mask != nullptr) &&
+                   (jobs[first + group].W_out != nullptr) == (jobs[first].W_out != nullptr))
+                ++group;
+        }
+        sp_status st = launch_nm_group(ctx, jobs, first, group, dtype, N, M, stream);
+        if (st != SP_OK) return st;
+        first += group;
+    }
+    return SP_OK;
 }
 
 }  // namespace sp

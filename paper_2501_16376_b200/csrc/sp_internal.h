@@ -95,23 +95,30 @@ sp_status launch_apply_mask(const void *W, sp_dtype dtype, int64_t n_rows, int64
                             int64_t ldw, const uint32_t *mask, void *W_out, int64_t ldo,
                             cudaStream_t stream);
 
-// select_nm.cu
-sp_status launch_select_nm(const sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
-                           int64_t ldw, int N, int M, uint32_t *mask, void *W_out, int64_t ldo,
-                           cudaStream_t stream);
-
 // select_nm_compressed.cu
 sp_status launch_select_24_compressed(const sp_ctx *ctx, const void *W, sp_dtype dtype,
                                       int64_t n_rows, int64_t ldw, void *values, int64_t ldv,
                                       uint32_t *meta, cudaStream_t stream);
 
-// select_ewma.cu
-struct EwmaLaunchJob {  // one weight matrix of an EWMA launch
+// One weight matrix of a selection launch that covers several (layers reading the same input).
+struct EwmaLaunchJob {
     const void *W;
     void *W_out;     // nullable
     uint32_t *mask;  // nullable
     int64_t n_rows, ldw, ldo;
 };
+
+// select_nm.cu: N:M selection of up to kEwmaMaxJobs matrices that share the context
+sp_status launch_select_nm(const sp_ctx *ctx, const EwmaLaunchJob *jobs, int n_jobs, sp_dtype dtype,
+                           int N, int M, cudaStream_t stream);
+inline sp_status launch_select_nm(const sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
+                                  int64_t ldw, int N, int M, uint32_t *mask, void *W_out,
+                                  int64_t ldo, cudaStream_t stream) {
+    const EwmaLaunchJob job{W, W_out, mask, n_rows, ldw, ldo};
+    return launch_select_nm(ctx, &job, 1, dtype, N, M, stream);
+}
+
+// select_ewma.cu
 // Algorithm 1 on up to kEwmaMaxJobs matrices that share the context (and dtype), in as few
 // launches as their layouts allow.
 sp_status launch_select_ewma(const sp_ctx *ctx, const EwmaLaunchJob *jobs, int n_jobs,

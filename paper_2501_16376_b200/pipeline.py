@@ -87,7 +87,17 @@ def select_layer(ctx: sp.Context, w: synth.Workload, W, mask, W_out, mode_arg, s
         ctx.sp_select_unstructured(W, mode_arg, mask=mask, W_out=W_out, stream=stream)
 
 
-def prune_model(mb: ModelBuffers, mode_arg, batch_tokens: int, phase_events=None, stream=None):
+def select_group(ctx: sp.Context, w: synth.Workload, Ws, masks, W_outs, mode_arg, stream=None):
+    """One grouped selection call for layers that read the same input."""
+    if w.mode == "nm":
+        N, M = mode_arg
+        ctx.sp_select_nm_group(Ws, N, M, masks=masks, W_outs=W_outs, stream=stream)
+    else:
+        ctx.sp_select_unstructured_group(Ws, mode_arg, masks=masks, W_outs=W_outs, stream=stream)
+
+
+def prune_model(mb: ModelBuffers, mode_arg, batch_tokens: int, phase_events=None, stream=None,
+                grouped: bool = True):
     """One pass of the whole hot path over the model: for every block and every distinct layer
     input, accumulate the calibration statistics, finalise them, then select + write back every
     layer that reads this input.  phase_events, if given, is a list that receives
@@ -96,7 +106,9 @@ def prune_model(mb: ModelBuffers, mode_arg, batch_tokens: int, phase_events=None
     weights, brackets the back-to-back selection launches of the layers reading this input);
     with phase_events the calls are issued strictly input by input so that the brackets are
     clean, without it the next input's calibration is enqueued ahead of the current input's
-    selections (same calls, same results).  Returns launch counts."""
+    selections (same calls, same results).  With grouped (the default) the layers that read one
+    input are selected by one grouped call (one launch when their layouts allow); otherwise by
+    one call each.  Returns launch counts."""
     w = mb.workload
     n_calib = n_select = n_final = 0
     if stream is None:
@@ -109,15 +121,17 @@ def prune_model(mb: ModelBuffers, mode_arg, batch_tokens: int, phase_events=None
 
     def select_input(b, name, ctx):
         nonlocal n_select
-        weights = 0
-        for li, layer in enumerate(w.layers):
-            if layer.input != name:
-                continue
-            select_layer(ctx, w, mb.weights[b][li], mb.masks[b][li], mb.outputs[b][li],
-                         mode_arg, stream)
-            n_select += 1
-            weights += layer.d_out * layer.d_in
-        return weights
+        idx = [li for li, layer in enumerate(w.layers) if layer.input == name]
+        before = sp.sp_launch_count()
+        if grouped and len(idx) > 1:
+            select_group(ctx, w, [mb.weights[b][li] for li in idx], [mb.masks[b][li] for li in idx],
+                         [mb.outputs[b][li] for li in idx], mode_arg, stream)
+        else:
+            for li in idx:
+                select_layer(ctx, w, mb.weights[b][li], mb.masks[b][li], mb.outputs[b][li],
+                             mode_arg, stream)
+        n_select += sp.sp_launch_count() - before
+        return sum(w.layers[li].d_out * w.layers[li].d_in for li in idx)
 
     if phase_events is None:
         # Plain pass.  The calibration of the next input is enqueued between an input's

@@ -567,7 +567,7 @@ def test_whole_pass_can_be_captured_and_replayed_as_a_cuda_graph(sp):
                 o.zero_()
         graph.replay()
         torch.cuda.synchronize()
-        assert counts["select"] == 2 * len(w.layers)
+        assert counts["select"] == 2 * len(w.input_widths())   # one grouped launch per input
         for b in range(w.blocks):
             for li in range(len(w.layers)):
                 assert torch.equal(mb.masks[b][li], want_masks[b][li])
@@ -620,3 +620,73 @@ def test_ewma_trace_matches_oracle_state(sp, s_update):
         assert np.array_equal(est.cpu().numpy(), e0)
         assert np.array_equal((est.cpu().numpy() - dev.cpu().numpy()).astype(np.float32), e1)
     assert (dev[:, 0] == 0).all() and torch.equal(est[:, 0], L[:, 0])
+
+
+# ------------------------------------------------------------------ grouped selection
+
+def _group_matrices(dtype, n):
+    """Four layers on one input: three that allow 16-byte access (one of them with a padded row
+    stride) and one that does not (odd offset), so that the call needs more than one launch."""
+    shapes = [(96, n), (33, n), (260, n), (17, n)]
+    Ws = [_gen(500 + i, s, dtype, 0.02) for i, s in enumerate(shapes)]
+    padded = torch.zeros(33, n + 24, dtype=dtype, device="cuda")
+    padded[:, :n] = Ws[1]
+    Ws[1] = padded[:, :n]                      # ld = n + 24
+    buf = torch.zeros(17 * n + 1, dtype=dtype, device="cuda")
+    buf[1:] = Ws[3].reshape(-1)
+    Ws[3] = buf[1:].view(17, n)                # 2-byte aligned only
+    return Ws
+
+
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+def test_grouped_ewma_selection_equals_single_calls_and_oracle(sp, dtype):
+    n = 1536
+    Ws = _group_matrices(dtype, n)
+    X = _activations(71, 2048, n, dtype)
+    counters = sp.new_counters()
+    with _ctx_with_stats(sp, [X], n) as ctx:
+        masks, outs = ctx.sp_select_unstructured_group(Ws, 0.6, counters=counters)
+        singles = [ctx.sp_select_unstructured(W, 0.6) for W in Ws]
+        colsq = ctx.sp_get_stats()[0]
+    st = so.Stats(colsq.numpy().copy(), 1)
+    kept = 0
+    for W, mask, out, (m1, o1) in zip(Ws, masks, outs, singles):
+        assert torch.equal(mask, m1)
+        assert torch.equal(out.contiguous().view(torch.int16), o1.contiguous().view(torch.int16))
+        sel = so.select_unstructured(P.bits(W), P.odtype(W), st, 0.6, want_trace=True)
+        P.check_selection(mask, out, W, sel, P.ewma_allowed_flips(sel))
+        kept += int(so.unpack_mask(P.mask_np(mask), n).sum())
+    assert int(counters[sp.SP_COUNTER_KEPT]) == kept
+
+
+@pytest.mark.parametrize("N,M", [(2, 4), (4, 8)])
+def test_grouped_nm_selection_equals_single_calls_and_oracle(sp, N, M):
+    n = 1536
+    Ws = _group_matrices(torch.float16, n)
+    X = _activations(72, 2048, n, torch.float16)
+    with _ctx_with_stats(sp, [X], n) as ctx:
+        masks, outs = ctx.sp_select_nm_group(Ws, N, M)
+        # a group whose members ask for different outputs (mask only / in place)
+        clones = [W.clone() for W in Ws]
+        masks2, outs2 = ctx.sp_select_nm_group(clones[:2], N, M, inplace=True)
+        colsq = ctx.sp_get_stats()[0]
+    st = so.Stats(colsq.numpy().copy(), 1)
+    for i, (W, mask, out) in enumerate(zip(Ws, masks, outs)):
+        sel = so.select_nm(P.bits(W), so.F16, st, N, M)
+        P.check_selection(mask, out, W, sel, None, strict=True)
+        if i < 2:
+            assert torch.equal(mask, masks2[i]) and outs2[i].data_ptr() == clones[i].data_ptr()
+            assert np.array_equal(P.bits(clones[i]), sel.W_out)
+
+
+def test_grouped_selection_rejects_bad_groups(sp):
+    n = 512
+    W = _gen(3, (8, n), torch.float16, 0.02)
+    X = _activations(4, 256, n, torch.float16)
+    with _ctx_with_stats(sp, [X], n) as ctx:
+        with pytest.raises(sp.SpError) as e:
+            ctx.sp_select_nm_group([W] * (sp.SP_MAX_GROUP + 1), 2, 4)
+        assert e.value.status == sp.SP_ERR_INVALID_ARG
+        with pytest.raises(sp.SpError) as e:
+            ctx.sp_select_unstructured_group([W, W.to(torch.bfloat16)], 0.5)
+        assert e.value.status == sp.SP_ERR_DTYPE

@@ -501,6 +501,8 @@ def gpu_arm(args):
                              sum(x.numel() * 2 for x in mb.acts.values()) / 1e9,
                              min(x.numel() * 2 for x in mb.acts.values()) / 1e9),
                    "launch": "cuda graph replay" if graph is not None else "stream launches",
+                   "calib_flags": "SP_CALIB_X_COMPLETE (the activations are resident and complete "
+                                  "long before the step starts)",
                    "parallelism": "independent models per rank" if world > 1 else "single GPU"},
         "whole_model_prune_s": {"calib": calib_ms / args.steps * 1e-3,
                                 "finalize": final_ms / args.steps * 1e-3,

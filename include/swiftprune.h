@@ -115,6 +115,20 @@ sp_status sp_calib_accumulate(sp_ctx *ctx, const void *X, sp_dtype dtype, int64_
                               int64_t ldx, sp_stream stream);
 
 /*
+ * The same with flags.  The library's kernels are launched so that a kernel may be scheduled
+ * while its predecessor on the stream drains; sp_calib_accumulate still reads X only after
+ * everything queued earlier on the stream has completed (ordinary stream semantics: the
+ * preceding kernel may be the one that writes X).  SP_CALIB_X_COMPLETE is the caller's promise
+ * that X was complete before the operation that precedes this call on the stream began (e.g.
+ * calibration data prepared long before, with library calls in between): the kernel then
+ * streams X while that predecessor is still finishing and orders only its update of the
+ * statistics after it.  With the flag set wrongly the statistics are silently wrong.
+ */
+enum { SP_CALIB_X_COMPLETE = 1 };
+sp_status sp_calib_accumulate_ex(sp_ctx *ctx, const void *X, sp_dtype dtype, int64_t n_tokens,
+                                 int64_t ldx, unsigned flags, sp_stream stream);
+
+/*
  * Reads the statistics back to HOST buffers (any may be NULL) and synchronises
  * the stream: colsq_host[d_in] (fp64), *S_host, factor_host[d_in] (the fp32
  * per-channel factor c_q = 1/(2(1 - colsq[q]/S)) of Eq. 8), *n_tokens_host.

@@ -22,10 +22,12 @@ SP_ERR_DEGENERATE, SP_ERR_CUDA, SP_ERR_NOMEM = 5, 6, 7
 SP_F16, SP_BF16 = 0, 1
 SP_S_GATED, SP_S_LITERAL_W2, SP_S_FROZEN = 0, 1, 2
 SP_COUNTER_KEPT, SP_COUNTER_S_HAZARD, SP_NUM_COUNTERS = 0, 1, 2
+SP_CALIB_X_COMPLETE = 1
 
 #: every symbol include/swiftprune.h declares
 EXPORTS = (
-    "sp_create", "sp_destroy", "sp_calib_reset", "sp_calib_accumulate", "sp_get_stats",
+    "sp_create", "sp_destroy", "sp_calib_reset", "sp_calib_accumulate", "sp_calib_accumulate_ex",
+    "sp_get_stats",
     "sp_set_stats", "sp_calib_stats_noalloc", "sp_score", "sp_la_for_sparsity", "sp_select_unstructured",
     "sp_select_unstructured_ex", "sp_search_la", "sp_ewma_trace", "sp_select_nm", "sp_select_24_compressed", "sp_apply_mask", "sp_calib_accumulate_host",
     "sp_select_nm_host", "sp_select_unstructured_host", "sp_select_unstructured_group",
@@ -65,6 +67,7 @@ def _load() -> ctypes.CDLL:
     lib.sp_destroy.argtypes = [vp]
     lib.sp_calib_reset.argtypes = [vp, vp]
     lib.sp_calib_accumulate.argtypes = [vp, vp, ci, i64, i64, vp]
+    lib.sp_calib_accumulate_ex.argtypes = [vp, vp, ci, i64, i64, ctypes.c_uint, vp]
     lib.sp_get_stats.argtypes = [vp, vp, vp, vp, ctypes.POINTER(i64), vp]
     lib.sp_set_stats.argtypes = [vp, vp, i64, vp]
     lib.sp_score.argtypes = [vp, vp, ci, i64, i64, vp, vp]
@@ -179,11 +182,17 @@ class Context:
     def sp_calib_reset(self, stream=None):
         _check(lib.sp_calib_reset(self._h, _stream(stream)))
 
-    def sp_calib_accumulate(self, X: torch.Tensor, stream=None):
+    def sp_calib_accumulate(self, X: torch.Tensor, stream=None, x_complete: bool = False):
+        """x_complete: X was complete before the preceding operation on the stream began
+        (SP_CALIB_X_COMPLETE, see the C header)."""
         ptr, T, n, ld = _matrix(X, "X")
         if n != self.d_in:
             raise SpError(SP_ERR_SHAPE, "X has %d channels, context has %d" % (n, self.d_in))
-        _check(lib.sp_calib_accumulate(self._h, ptr, _dtype_of(X), T, ld, _stream(stream)))
+        if x_complete:
+            _check(lib.sp_calib_accumulate_ex(self._h, ptr, _dtype_of(X), T, ld,
+                                              SP_CALIB_X_COMPLETE, _stream(stream)))
+        else:
+            _check(lib.sp_calib_accumulate(self._h, ptr, _dtype_of(X), T, ld, _stream(stream)))
 
     def sp_get_stats(self, stream=None):
         """Returns (colsq fp64 [d_in], S, factor fp32 [d_in], n_tokens) as CPU tensors/numbers."""

@@ -149,17 +149,24 @@ sp_status sp_calib_reset(sp_ctx *ctx, sp_stream stream) {
     return SP_OK;
 }
 
-sp_status sp_calib_accumulate(sp_ctx *ctx, const void *X, sp_dtype dtype, int64_t n_tokens,
-                              int64_t ldx, sp_stream stream) {
+sp_status sp_calib_accumulate_ex(sp_ctx *ctx, const void *X, sp_dtype dtype, int64_t n_tokens,
+                                 int64_t ldx, unsigned flags, sp_stream stream) {
     if (ctx == nullptr) return SP_ERR_INVALID_ARG;
     if (!valid_dtype(dtype)) return SP_ERR_DTYPE;
-    if (n_tokens < 0) return SP_ERR_INVALID_ARG;
+    if (n_tokens < 0 || (flags & ~static_cast<unsigned>(SP_CALIB_X_COMPLETE)) != 0u)
+        return SP_ERR_INVALID_ARG;
     if (n_tokens == 0) return SP_OK;
     if (X == nullptr) return SP_ERR_INVALID_ARG;
     if (ldx < ctx->d_in) return SP_ERR_SHAPE;
     DeviceGuard guard(ctx->device);
     if (guard.error() != cudaSuccess) return cuda_fail(guard.error());
-    return launch_calib_accumulate(ctx, X, dtype, n_tokens, ldx, static_cast<cudaStream_t>(stream));
+    return launch_calib_accumulate(ctx, X, dtype, n_tokens, ldx, static_cast<cudaStream_t>(stream),
+                                   (flags & SP_CALIB_X_COMPLETE) != 0u);
+}
+
+sp_status sp_calib_accumulate(sp_ctx *ctx, const void *X, sp_dtype dtype, int64_t n_tokens,
+                              int64_t ldx, sp_stream stream) {
+    return sp_calib_accumulate_ex(ctx, X, dtype, n_tokens, ldx, 0u, stream);
 }
 
 sp_status sp_get_stats(sp_ctx *ctx, double *colsq_host, double *S_host, float *factor_host,

@@ -26,11 +26,15 @@ template <bool BF16, bool VEC>
 __global__ void __launch_bounds__(kCalibThreads)
 calib_accumulate_kernel(const uint16_t *__restrict__ X, int64_t ldx, int64_t n_tokens, int64_t n,
                         int64_t rows_per_slab, double *__restrict__ partial, int64_t n_pad,
-                        int first_fresh_slab) {
+                        int first_fresh_slab, int x_complete) {
     // Programmatic dependent launch: the next kernel in the stream may start as soon as this
-    // grid's CTAs are all resident, and this kernel's own streaming phase may overlap the tail of
-    // the previous one; only the read-modify-write of the partial sums below waits for it.
+    // grid's CTAs are all resident.  X is read only after everything queued earlier on the
+    // stream has completed - the kernel before this one may be the one that writes X - unless
+    // the caller vouches that X was complete before that (x_complete): then the streaming phase
+    // overlaps the tail of the previous kernel and only the read-modify-write of the partial
+    // sums below waits for it.
     pdl_launch_dependents();
+    if (!x_complete) pdl_wait();
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const int strip = blockIdx.x;
@@ -225,7 +229,7 @@ static int query_blocks_per_sm() {
 int calib_query_blocks_per_sm() { return query_blocks_per_sm<false, true>(); }
 
 sp_status launch_calib_accumulate(sp_ctx *ctx, const void *X, sp_dtype dtype, int64_t n_tokens,
-                                  int64_t ldx, cudaStream_t stream) {
+                                  int64_t ldx, cudaStream_t stream, bool x_complete) {
     const int64_t n = ctx->d_in;
     // One resident wave: strips x slabs CTAs fill the GPU once, every CTA gets the same rows.
     const int64_t resident = static_cast<int64_t>(ctx->sm_count) * ctx->calib_blocks_per_sm;
@@ -247,10 +251,11 @@ sp_status launch_calib_accumulate(sp_ctx *ctx, const void *X, sp_dtype dtype, in
     double *partial = ctx->partial;
     int64_t n_pad = ctx->n_pad;
     int first_fresh = ctx->slabs_valid;
+    const int x_ok = x_complete ? 1 : 0;
     cudaError_t launch_err = cudaSuccess;
 #define SP_LAUNCH(B, V)                                                                       \
     launch_err = cudaLaunchKernelEx(&pdl.cfg, calib_accumulate_kernel<B, V>, Xp, ldx, n_tokens, n, \
-                                    rows_per_slab, partial, n_pad, first_fresh)
+                                    rows_per_slab, partial, n_pad, first_fresh, x_ok)
     if (bf16) {
         if (vec) SP_LAUNCH(true, true); else SP_LAUNCH(true, false);
     } else {
@@ -366,7 +371,8 @@ sp_status launch_calib_stats_static(int device, const void *X, sp_dtype dtype, i
     const uint16_t *Xp = static_cast<const uint16_t *>(X);
 #define SP_LAUNCH(B, V)                                                                       \
     calib_accumulate_kernel<B, V><<<grid, kCalibThreads, 0, stream>>>(                        \
-        Xp, ldx, n_tokens, n, rows_per_slab, sc->partial, n_pad, /*first_fresh_slab=*/0)
+        Xp, ldx, n_tokens, n, rows_per_slab, sc->partial, n_pad, /*first_fresh_slab=*/0, \
+        /*x_complete=*/0)
     if (bf16) {
         if (vec) SP_LAUNCH(true, true); else SP_LAUNCH(true, false);
     } else {

@@ -81,7 +81,7 @@ inline sp_status check_launch() {
 // calib.cu
 int calib_query_blocks_per_sm();
 sp_status launch_calib_accumulate(sp_ctx *ctx, const void *X, sp_dtype dtype, int64_t n_tokens,
-                                  int64_t ldx, cudaStream_t stream);
+                                  int64_t ldx, cudaStream_t stream, bool x_complete = false);
 sp_status launch_finalize(sp_ctx *ctx, cudaStream_t stream);
 int64_t calib_static_max_d_in();
 sp_status launch_calib_stats_static(int device, const void *X, sp_dtype dtype, int64_t n_tokens,

@@ -67,13 +67,16 @@ def allocate_model(w: synth.Workload, device, model_seed_offset: int = 0,
     return mb
 
 
-def calibrate_input(ctx: sp.Context, X: torch.Tensor, batch_tokens: int, stream=None) -> int:
-    """Streams X through sp_calib_accumulate in batches; returns the number of launches."""
+def calibrate_input(ctx: sp.Context, X: torch.Tensor, batch_tokens: int, stream=None,
+                    x_complete: bool = False) -> int:
+    """Streams X through sp_calib_accumulate in batches; returns the number of launches.
+    x_complete: the activations were complete before the previous operation on the stream began
+    (true for the resident synthetic activations of ModelBuffers)."""
     ctx.sp_calib_reset(stream)
     T = X.shape[0]
     launches = 0
     for t0 in range(0, T, batch_tokens):
-        ctx.sp_calib_accumulate(X[t0:min(T, t0 + batch_tokens)], stream)
+        ctx.sp_calib_accumulate(X[t0:min(T, t0 + batch_tokens)], stream, x_complete)
         launches += 1
     return launches
 
@@ -144,12 +147,12 @@ def prune_model(mb: ModelBuffers, mode_arg, batch_tokens: int, phase_events=None
         for i, (b, name) in enumerate(units):
             ctx = mb.ctxs[name]
             if i == 0 or not distinct:
-                n_calib += calibrate_input(ctx, mb.acts[name], batch_tokens, stream)
+                n_calib += calibrate_input(ctx, mb.acts[name], batch_tokens, stream, True)
             ctx.sp_score(None, stream=stream)          # finalisation only
             n_final += 1
             if distinct and i + 1 < len(units):
                 nxt = units[i + 1][1]
-                n_calib += calibrate_input(mb.ctxs[nxt], mb.acts[nxt], batch_tokens, stream)
+                n_calib += calibrate_input(mb.ctxs[nxt], mb.acts[nxt], batch_tokens, stream, True)
             select_input(b, name, ctx)
         return {"calib": n_calib, "finalize": n_final, "select": n_select}
 
@@ -159,7 +162,7 @@ def prune_model(mb: ModelBuffers, mode_arg, batch_tokens: int, phase_events=None
             ctx = mb.ctxs[name]
             X = mb.acts[name]
             e0 = last
-            n_calib += calibrate_input(ctx, X, batch_tokens, stream)
+            n_calib += calibrate_input(ctx, X, batch_tokens, stream, True)
             e1 = mark()
             ctx.sp_score(None, stream=stream)          # finalisation only
             n_final += 1

@@ -690,3 +690,20 @@ def test_grouped_selection_rejects_bad_groups(sp):
         with pytest.raises(sp.SpError) as e:
             ctx.sp_select_unstructured_group([W, W.to(torch.bfloat16)], 0.5)
         assert e.value.status == sp.SP_ERR_DTYPE
+
+
+def test_calib_accumulate_ex_flag_changes_ordering_only(sp):
+    n = 1000
+    X = _activations(81, 3000, n, torch.float16)
+    torch.cuda.synchronize()                      # X is complete: the promise of the flag holds
+    with sp.Context(n) as a, sp.Context(n) as b:
+        for t0 in range(0, 3000, 1000):
+            a.sp_calib_accumulate(X[t0:t0 + 1000])
+            b.sp_calib_accumulate(X[t0:t0 + 1000], x_complete=True)
+        ca, Sa, fa, _ = a.sp_get_stats()
+        cb, Sb, fb, _ = b.sp_get_stats()
+        assert torch.equal(ca, cb) and Sa == Sb and torch.equal(fa, fb)
+        st = P.oracle_stats([X], n)
+        assert P.rel_err(ca.numpy(), st.colsq) <= P.SCORE_RTOL
+        bad = sp.lib.sp_calib_accumulate_ex(a._h, X.data_ptr(), sp.SP_F16, 1000, n, 2, None)
+        assert bad == sp.SP_ERR_INVALID_ARG

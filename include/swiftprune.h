@@ -161,7 +161,9 @@ sp_status sp_set_stats(sp_ctx *ctx, const double *colsq_host, int64_t n_tokens, 
  *     streams, different threads) race and give wrong results - keep them on one stream or
  *     order them with events.  Nothing is kept between calls;
  *   - the first call on each device looks up the array's device address (a host-side,
- *     synchronous runtime query); make that first call before starting any stream capture.
+ *     synchronous runtime query) and may make the CUDA runtime load the library's kernels,
+ *     which can allocate; make that first call before starting any stream capture and before
+ *     the phase in which nothing may be allocated.
  * Results agree with the context path to rounding (the token slabs may be cut differently).
  */
 sp_status sp_calib_stats_noalloc(const void *X, sp_dtype dtype, int64_t n_tokens, int64_t d_in,

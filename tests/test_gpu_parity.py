@@ -707,3 +707,109 @@ def test_calib_accumulate_ex_flag_changes_ordering_only(sp):
         assert P.rel_err(ca.numpy(), st.colsq) <= P.SCORE_RTOL
         bad = sp.lib.sp_calib_accumulate_ex(a._h, X.data_ptr(), sp.SP_F16, 1000, n, 2, None)
         assert bad == sp.SP_ERR_INVALID_ARG
+
+
+# ------------------------------------------------------------------ non-finite scores
+
+def _golden_nonfinite():
+    import os
+    out = {}
+    with open(os.path.join(os.path.dirname(__file__), "golden", "nonfinite_scores.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                key, *vals = line.split()
+                out[key] = vals
+    return out
+
+
+def _row16(vals, n, dtype=torch.float16):
+    row = torch.zeros(n, dtype=torch.float32)
+    row[:len(vals)] = torch.tensor([float(v) for v in vals])
+    return row.to(dtype)
+
+
+@pytest.mark.parametrize("n", [8, 512, 520, 12])       # stream kernel (whole / ragged), general
+def test_nm_with_nan_and_infinite_scores_hand_cases_and_oracle(sp, n):
+    g = _golden_nonfinite()
+    # all channels alike: NaN / +inf weights inside the first two groups
+    W = torch.stack([_row16(g["nm_a_weights"], n), _row16(g["nm_a_weights"][4:], n)]).cuda()
+    with sp.Context(n) as ctx:
+        ctx.sp_set_stats(torch.ones(n, dtype=torch.float64), 4)
+        mask, out = ctx.sp_select_nm(W, 2, 4)
+    sel = so.select_nm(P.bits(W), so.F16, so.Stats(np.ones(n), 4), 2, 4)
+    P.check_selection(mask, out, W, sel, None, strict=True)
+    keep = so.unpack_mask(P.mask_np(mask), n)
+    want = np.array([c == "1" for c in g["nm_a_keep"][0]])
+    assert np.array_equal(keep[0, :8], want) and np.array_equal(keep[1, :4], want[4:])
+    # one live channel: c_0 = +inf; w_0 = 0 gives a NaN score, w_0 = 0.5 an infinite one
+    colsq = np.zeros(n)
+    colsq[0] = 1.0
+    W = torch.stack([_row16(g["nm_b_row0"], n), _row16(g["nm_b_row1"], n)]).cuda()
+    with sp.Context(n) as ctx:
+        ctx.sp_set_stats(torch.from_numpy(colsq), 4)
+        mask, out = ctx.sp_select_nm(W, 2, 4)
+        L = ctx.sp_score(W)
+    sel = so.select_nm(P.bits(W), so.F16, so.Stats(colsq.copy(), 4), 2, 4, want_trace=True)
+    P.check_selection(mask, out, W, sel, None, strict=True)
+    keep = so.unpack_mask(P.mask_np(mask), n)
+    assert np.array_equal(keep[0, :4], np.array([c == "1" for c in g["nm_b_keep0"][0]]))
+    assert np.array_equal(keep[1, :4], np.array([c == "1" for c in g["nm_b_keep1"][0]]))
+    Lc = L.cpu().numpy()
+    assert np.isnan(Lc[0, 0]) and np.isinf(Lc[1, 0])
+    assert np.array_equal(np.isnan(Lc), np.isnan(sel.L))
+    assert np.array_equal(Lc[~np.isnan(Lc)], sel.L[~np.isnan(sel.L)])
+
+
+@pytest.mark.parametrize("n", [6, 8, 1024, 1030])       # general kernel, pair kernel, several tiles
+@pytest.mark.parametrize("mode", ["gated", "frozen", "literal"])
+def test_ewma_with_nan_and_infinite_scores_hand_cases_and_oracle(sp, n, mode):
+    g = _golden_nonfinite()
+    s_lib = {"gated": sp.SP_S_GATED, "frozen": sp.SP_S_FROZEN, "literal": sp.SP_S_LITERAL_W2}[mode]
+    s_ora = so.S_FROZEN if mode == "frozen" else so.S_LITERAL_W2
+    rows = [_row16(g["ewma_a_weights"], n), _row16(g["ewma_b_weights"], n)]
+    if n > 600:        # the same events deep inside a row: after a tile of ordinary weights
+        body = _gen(61, (2, n), torch.float16, 0.02).cpu()
+        body[0, 600:606] = rows[0][:6]
+        body[1, 700:706] = rows[1][:6]
+        rows = [body[0], body[1]]
+    W = torch.stack(rows).cuda()
+    colsq = np.ones(n) * 1e6                              # calibration scale: S cannot move ...
+    with sp.Context(n) as ctx:
+        ctx.sp_set_stats(torch.from_numpy(colsq), 4)
+        counters = sp.new_counters()
+        mask, out = ctx.sp_select_unstructured(W, params=_ewma_params(sp, 0.5, s_update=s_lib),
+                                               counters=counters)
+    sel = so.select_ewma(P.bits(W), so.F16, so.Stats(colsq.copy(), 4), 0.5, s_update=s_ora,
+                         want_trace=True)
+    keep = so.unpack_mask(P.mask_np(mask), n)
+    want = sel.keep_bool(n)
+    if n <= 8:
+        for r, key in enumerate(("ewma_a_keep", "ewma_b_keep")):
+            assert np.array_equal(keep[r, :6], np.array([c == "1" for c in g[key][0]]))
+    # before the non-finite weight the usual band rule; from it on everything is kept
+    first = 2 if n <= 8 else None
+    starts = [first, first] if first is not None else [602, 702]
+    for r in range(2):
+        assert keep[r, starts[r]:].all() and want[r, starts[r]:].all()
+        d = keep[r, :starts[r]] != want[r, :starts[r]]
+        assert not (d & ~P.ewma_allowed_flips(sel)[r, :starts[r]]).any() and d.sum() <= 1
+    assert np.array_equal(P.bits(out), np.where(keep, P.bits(W), 0))
+    assert int(counters[sp.SP_COUNTER_KEPT]) == int(keep.sum())
+    if mode == "gated":                                   # ... but NaN / inf rows go the exact way
+        assert int(counters[sp.SP_COUNTER_S_HAZARD]) == 2
+
+
+@pytest.mark.parametrize("target", [0.3, 0.5, 0.55, 0.65, 0.8, 0.9])
+def test_search_la_reports_exactly_what_the_selection_then_prunes(sp, target):
+    R, n = 256, 2048
+    W = _gen(95, (R, n), torch.bfloat16, 0.02)
+    X = _activations(96, 2048, n, torch.bfloat16)
+    with _ctx_with_stats(sp, [X], n) as ctx:
+        la, achieved = ctx.sp_search_la(W, target, iterations=20)
+        mask, _ = ctx.sp_select_unstructured(W, params=_ewma_params(sp, la, s_update=sp.SP_S_FROZEN))
+        mask_g, _ = ctx.sp_select_unstructured(W, params=_ewma_params(sp, la))
+    pruned = 1.0 - so.unpack_mask(P.mask_np(mask), n).mean(dtype=np.float64)
+    assert pruned == achieved                 # the same constants in the count and in the selection
+    assert torch.equal(mask, mask_g)
+    assert abs(achieved - target) < 2e-3

@@ -513,3 +513,43 @@ def test_compressed_24_hand_example_and_round_trip():
     assert np.array_equal(so.expand_24(v, m, n), sel.W_out)
     with pytest.raises(ValueError):
         so.compress_24(W, np.ones((1, 8), dtype=bool))
+
+
+# ---------------------------------------------------------------- non-finite scores
+
+def _fixture_row(vals):
+    return _f16_bits(np.array([float(v) for v in vals], dtype=np.float64))[None, :]
+
+
+def _keep_bits(s):
+    return np.array([c == "1" for c in s])
+
+
+def test_nan_ranks_above_every_number_in_nm_groups_hand_cases():
+    g = _read_golden("nonfinite_scores.txt")
+    st = _stats_from([float(v) for v in g["nm_a_colsq"]])
+    sel = so.select_nm(_fixture_row(g["nm_a_weights"]), so.F16, st, 2, 4)
+    assert np.array_equal(sel.keep_bool(8)[0], _keep_bits(g["nm_a_keep"][0]))
+    st = _stats_from([float(v) for v in g["nm_b_colsq"]])
+    c = st.channel_factor32()
+    assert np.isinf(c[0]) and np.all(c[1:] == 0.5)
+    for row, keep in (("nm_b_row0", "nm_b_keep0"), ("nm_b_row1", "nm_b_keep1")):
+        sel = so.select_nm(_fixture_row(g[row]), so.F16, st, 2, 4, want_trace=True)
+        assert np.array_equal(sel.keep_bool(4)[0], _keep_bits(g[keep][0]))
+    assert np.isinf(sel.L[0, 0])                      # 0.5^2 * inf
+    # pruned weights are +0 also when the pruned score was a number next to a NaN
+    sel = so.select_nm(_fixture_row(g["nm_b_row0"]), so.F16, st, 2, 4, want_trace=True)
+    assert np.isnan(sel.L[0, 0]) and (sel.W_out[0, 2:] == 0).all()
+
+
+@pytest.mark.parametrize("case", ["ewma_a", "ewma_b"])
+@pytest.mark.parametrize("s_update", [so.S_FROZEN, so.S_LITERAL_W2])
+def test_comparisons_with_nan_keep_the_weight_in_algorithm_1_hand_cases(case, s_update):
+    g = _read_golden("nonfinite_scores.txt")
+    st = _stats_from([float(v) for v in g[case + "_colsq"]])
+    W = _fixture_row(g[case + "_weights"])
+    for precision in ("f32", "f64"):
+        sel = so.select_ewma(W, so.F16, st, 0.5, 0.125, 0.125, s_update=s_update,
+                             precision=precision)
+        assert np.array_equal(sel.keep_bool(6)[0], _keep_bits(g[case + "_keep"][0]))
+        assert sel.W_out[0, 1] == 0 and sel.W_out[0, 2] == W[0, 2]

@@ -59,6 +59,40 @@ def test_noalloc_statistics_match_the_context_path_on_two_calls_in_a_row():
     assert torch.equal(first, colsq_out)
 
 
+@pytest.mark.parametrize("T,n,ld,dtype", [
+    (4096, 16384, 16384, torch.float16),     # the widest input: the fixed partial-sum area is full
+    (1500, 16376, 16384, torch.bfloat16),    # padded row stride
+    (900, 1001, 1001, torch.float16),        # odd width: element-wise loads
+])
+def test_noalloc_statistics_match_the_oracle_at_the_limits(T, n, ld, dtype):
+    """Against the CPU oracle and the context path; checks as well that the call launches exactly
+    its two kernels and leaves the device's free memory as it found it."""
+    import numpy as np
+    from oracle import swiftprune_oracle as so
+    from paper_2501_16376_b200 import binding as sp
+    from tests import parity as P
+    buf = _batch(7, T, ld, dtype)
+    X = buf[:, :n]
+    colsq_out = torch.empty(n, dtype=torch.float64, device="cuda")
+    factor_out = torch.empty(n, dtype=torch.float32, device="cuda")
+    S_out = torch.empty(1, dtype=torch.float64, device="cuda")
+    sp.sp_calib_stats_noalloc(X, colsq_out, factor_out, S_out)       # first call on the device
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    launches_before = sp.sp_launch_count()
+    sp.sp_calib_stats_noalloc(X, colsq_out, factor_out, S_out)
+    torch.cuda.synchronize()
+    assert sp.sp_launch_count() - launches_before == 2
+    assert torch.cuda.mem_get_info()[0] == free_before
+    st = so.colsq_accumulate(so.new_stats(n), P.bits(X), P.odtype(X), threads=so.max_threads())
+    assert P.rel_err(colsq_out.cpu().numpy(), st.colsq) <= P.SCORE_RTOL
+    assert abs(S_out.item() - st.S) <= P.SCORE_RTOL * st.S
+    assert P.rel_err(factor_out.cpu().numpy(), st.channel_factor32()) <= P.SCORE_RTOL
+    colsq, S, factor = _reference(sp, X)
+    assert _rel(colsq_out.cpu(), colsq) <= RTOL and abs(S_out.item() - S) <= RTOL * S
+    assert np.isfinite(factor_out.cpu().numpy()).all()
+
+
 def test_noalloc_rejects_sizes_beyond_its_fixed_array():
     from paper_2501_16376_b200 import binding as sp
     X = torch.zeros(8, 16392, dtype=torch.float16, device="cuda")

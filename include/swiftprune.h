@@ -69,7 +69,12 @@ typedef enum {
                             detected and re-evaluated sequentially in the same call, so the
                             result is that of SP_S_LITERAL_W2 for every row (the default) */
     SP_S_LITERAL_W2 = 1, /* the printed update, evaluated sequentially along every row */
-    SP_S_FROZEN = 2      /* S keeps its initial value whatever is pruned */
+    SP_S_FROZEN = 2,     /* S keeps its initial value whatever is pruned */
+    SP_S_READING_X2 = 3  /* the other conceivable reading of that row of Table 2: S is a sum of
+                            x^2, and a pruned weight takes its channel's x_i^2 out of it
+                            ("S = S - x_i^2"); evaluated sequentially along every row.  This
+                            changes S by tens of percent and is not what the paper prints:
+                            offered for comparison */
 } sp_s_update;
 
 /* Parameters of Algorithm 1 (alpha, beta: Table 2; la: Table 3). */

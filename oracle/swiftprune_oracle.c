@@ -50,6 +50,8 @@
 
 #define SPO_S_LITERAL_W2 1 /* Table 2 / Algorithm 1: S <- S - w_i^2 when pruned */
 #define SPO_S_FROZEN 0     /* S stays at its initial value */
+#define SPO_S_READING_X2 2 /* the other reading of Table 2's row S: S <- S - x_i^2 when pruned (S is a
+                              sum of x^2, so the pruned channel's own share leaves it) */
 
 /* ---- 16-bit float decoding (exact) ------------------------------------- */
 
@@ -227,6 +229,8 @@ void spo_select_ewma_f32(const uint16_t *W, int dtype, int64_t R, int64_t n, int
                 if (s_update == SPO_S_LITERAL_W2) {
                     float w2 = w * w;
                     S = S - w2;
+                } else if (s_update == SPO_S_READING_X2) {
+                    S = S - colsq32[i];
                 }
                 bits = 0; /* w_i = 0 */
             } else {
@@ -278,6 +282,8 @@ void spo_select_ewma_f64(const uint16_t *W, int dtype, int64_t R, int64_t n, int
             if (L < thr) {
                 if (s_update == SPO_S_LITERAL_W2)
                     S = S - w * w;
+                else if (s_update == SPO_S_READING_X2)
+                    S = S - colsq[i];
                 bits = 0;
             } else {
                 spo_set_keep(mrow, i);

@@ -29,6 +29,7 @@ F16 = 0
 BF16 = 1
 S_FROZEN = 0
 S_LITERAL_W2 = 1
+S_READING_X2 = 2     # the other reading of Table 2's row S: S <- S - x_i^2 when pruned
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "swiftprune_oracle.c")

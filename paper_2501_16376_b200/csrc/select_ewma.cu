@@ -83,7 +83,8 @@ struct EwmaJobTable {
 
 // Algorithm 1 exactly as printed along one row from column i_begin (a multiple of 32) on, by
 // one thread, binary32 with one rounding per operation; est / dev are the state before that
-// column (ignored for column 0, where est starts at L_0).  Element-wise access with bounds
+// column (ignored for column 0, where est starts at L_0).  subtract_x2: the other reading of
+// Table 2's row S, a pruned weight takes its channel's x_i^2 (not w_i^2) out of S.  Element-wise access with bounds
 // checks.  While S still has its initial value the per-channel factor computed at finalisation
 // is used: it was formed by the same three operations from the same S, so the result is
 // bit-identical to recomputing it; once a pruned weight has changed S the factor is recomputed
@@ -92,7 +93,8 @@ template <bool BF16>
 __device__ __forceinline__ unsigned long long literal_walk(
     const uint16_t *__restrict__ wrow, uint16_t *__restrict__ orow, uint32_t *__restrict__ mrow,
     int64_t n, int64_t i_begin, float est, float dev, const double *__restrict__ colsq,
-    const float *__restrict__ factor, float S0, float alpha, float beta, float la) {
+    const float *__restrict__ factor, float S0, float alpha, float beta, float la,
+    bool subtract_x2 = false) {
     const float one_minus_alpha = __fsub_rn(1.0f, alpha);
     const float one_minus_beta = __fsub_rn(1.0f, beta);
     float S = S0;
@@ -129,7 +131,7 @@ __device__ __forceinline__ unsigned long long literal_walk(
                 if (i == 0) est = L;
                 const float thr = __fsub_rn(est, __fmul_rn(la, dev));
                 if (L < thr) {
-                    S = __fsub_rn(S, w2);
+                    S = __fsub_rn(S, subtract_x2 ? static_cast<float>(colsq[i]) : w2);
                 } else {
                     keep8 |= 1u << j;
                 }
@@ -630,13 +632,13 @@ ewma_literal_kernel(const uint16_t *__restrict__ W, int64_t ldw, int64_t n_rows,
                     const DeviceScalars *__restrict__ scalars, float alpha, float beta, float la,
                     uint32_t *__restrict__ mask, int64_t mask_words,
                     uint16_t *__restrict__ W_out, int64_t ldo,
-                    unsigned long long *__restrict__ counters) {
+                    unsigned long long *__restrict__ counters, int subtract_x2) {
     const int64_t row = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (row >= n_rows) return;
     const unsigned long long kept = literal_walk<BF16>(
         W + row * ldw, W_out != nullptr ? W_out + row * ldo : nullptr,
         mask != nullptr ? mask + row * mask_words : nullptr, n, 0, 0.0f, 0.0f, colsq, factor,
-        scalars->S32, alpha, beta, la);
+        scalars->S32, alpha, beta, la, subtract_x2 != 0);
     if (counters != nullptr) atomicAdd(counters + SP_COUNTER_KEPT, kept);
 }
 
@@ -671,7 +673,7 @@ ewma_trace_kernel(const uint16_t *__restrict__ W, int64_t ldw, int64_t n_rows, i
         if (dev_out != nullptr) dev_out[row * n + i] = dev;
         if (score_out != nullptr) score_out[row * n + i] = L;
         const float thr = __fsub_rn(est, __fmul_rn(la, dev));
-        if (L < thr && literal_s) S = __fsub_rn(S, w2);
+        if (L < thr && literal_s) S = __fsub_rn(S, literal_s == 2 ? static_cast<float>(colsq[i]) : w2);
         est = __fadd_rn(__fmul_rn(one_minus_alpha, est), __fmul_rn(alpha, L));
         dev = __fadd_rn(__fmul_rn(one_minus_beta, dev), __fmul_rn(beta, fabsf(__fsub_rn(est, L))));
     }
@@ -684,7 +686,7 @@ sp_status launch_ewma_trace(const sp_ctx *ctx, const void *W, sp_dtype dtype, in
     const int64_t blocks = (n_rows + 127) / 128;
     if (blocks > 0x7fffffffLL) return SP_ERR_SHAPE;
     const uint16_t *Wp = static_cast<const uint16_t *>(W);
-    const int literal = p.s_update != SP_S_FROZEN ? 1 : 0;  // gated = Algorithm 1 as printed
+    const int literal = p.s_update == SP_S_FROZEN ? 0 : (p.s_update == SP_S_READING_X2 ? 2 : 1);  // gated = as printed
     if (dtype == SP_BF16)
         ewma_trace_kernel<true><<<static_cast<unsigned>(blocks), 128, 0, stream>>>(
             Wp, ldw, n_rows, ctx->d_in, ctx->colsq, ctx->scalars, p.alpha, p.beta, p.la, literal,
@@ -847,11 +849,11 @@ sp_status launch_literal(const sp_ctx *ctx, const EwmaLaunchJob &j, sp_dtype dty
     if (dtype == SP_BF16)
         ewma_literal_kernel<true><<<lgrid, 128, 0, stream>>>(
             Wp, j.ldw, j.n_rows, n, ctx->colsq, ctx->factor, ctx->scalars, p.alpha, p.beta, p.la,
-            j.mask, words, Op, j.ldo, counters);
+            j.mask, words, Op, j.ldo, counters, p.s_update == SP_S_READING_X2 ? 1 : 0);
     else
         ewma_literal_kernel<false><<<lgrid, 128, 0, stream>>>(
             Wp, j.ldw, j.n_rows, n, ctx->colsq, ctx->factor, ctx->scalars, p.alpha, p.beta, p.la,
-            j.mask, words, Op, j.ldo, counters);
+            j.mask, words, Op, j.ldo, counters, p.s_update == SP_S_READING_X2 ? 1 : 0);
     return check_launch();
 }
 
@@ -878,7 +880,7 @@ sp_status launch_select_ewma(const sp_ctx *ctx, const EwmaLaunchJob *jobs_in, in
             if (j.mask != nullptr) q.mask = j.mask + r0 * words;
         }
     }
-    if (p.s_update == SP_S_LITERAL_W2) {
+    if (p.s_update == SP_S_LITERAL_W2 || p.s_update == SP_S_READING_X2) {
         for (int i = 0; i < n_pieces; ++i) {
             sp_status st = launch_literal(ctx, pieces[i], dtype, p, counters, stream);
             if (st != SP_OK) return st;

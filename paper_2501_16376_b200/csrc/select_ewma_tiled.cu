@@ -39,7 +39,7 @@ ewma_literal_tiled_kernel(const uint16_t *__restrict__ W, int64_t ldw, int n_row
                           const DeviceScalars *__restrict__ scalars, float alpha, float beta,
                           float la, uint32_t *__restrict__ mask, int mask_words,
                           uint16_t *__restrict__ W_out, int64_t ldo,
-                          unsigned long long *__restrict__ counters) {
+                          unsigned long long *__restrict__ counters, int subtract_x2) {
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int row_base = blockIdx.x * 32;
@@ -129,7 +129,11 @@ ewma_literal_tiled_kernel(const uint16_t *__restrict__ W, int64_t ldw, int n_row
                         if (k == 0 && j == 0 && tile == 0) est = L;
                         const float thr = __fsub_rn(est, __fmul_rn(la, dev));
                         const bool prune = L < thr;
-                        S = prune ? __fsub_rn(S, w2) : S;
+                        float dec = w2;
+                        if (decltype(follow_s)::value) {  // the x_i^2 reading always walks this way
+                            if (subtract_x2) dec = static_cast<float>(colsq[i0 + j]);
+                        }
+                        S = prune ? __fsub_rn(S, dec) : S;
                         keep8 |= prune ? 0u : 1u << j;
                         est = __fadd_rn(__fmul_rn(one_minus_alpha, est), __fmul_rn(alpha, L));
                         dev = __fadd_rn(__fmul_rn(one_minus_beta, dev),
@@ -140,7 +144,7 @@ ewma_literal_tiled_kernel(const uint16_t *__restrict__ W, int64_t ldw, int n_row
                 // chunk is straight-line code with the finalised factors.  Otherwise the chunk
                 // is walked (again) from the state it started in, following S element by element.
                 const float est_in = est, dev_in = dev, S_in = S;
-                bool follow = __any_sync(kWalkerMask, S_in != S0);
+                bool follow = subtract_x2 != 0 || __any_sync(kWalkerMask, S_in != S0);
                 if (!follow) {
                     walk(std::false_type{});
                     follow = __any_sync(kWalkerMask, S != S_in);
@@ -196,11 +200,13 @@ sp_status launch_ewma_literal_tiled(const sp_ctx *ctx, const void *W, sp_dtype d
     if (dtype == SP_BF16)
         ewma_literal_tiled_kernel<true><<<grid, kTiledThreads, 0, stream>>>(
             Wp, ldw, static_cast<int>(n_rows), static_cast<int>(n), ctx->colsq, ctx->factor,
-            ctx->scalars, p.alpha, p.beta, p.la, mask, words, Op, ldo, counters);
+            ctx->scalars, p.alpha, p.beta, p.la, mask, words, Op, ldo, counters,
+            p.s_update == SP_S_READING_X2 ? 1 : 0);
     else
         ewma_literal_tiled_kernel<false><<<grid, kTiledThreads, 0, stream>>>(
             Wp, ldw, static_cast<int>(n_rows), static_cast<int>(n), ctx->colsq, ctx->factor,
-            ctx->scalars, p.alpha, p.beta, p.la, mask, words, Op, ldo, counters);
+            ctx->scalars, p.alpha, p.beta, p.la, mask, words, Op, ldo, counters,
+            p.s_update == SP_S_READING_X2 ? 1 : 0);
     return check_launch();
 }
 

@@ -813,3 +813,55 @@ def test_search_la_reports_exactly_what_the_selection_then_prunes(sp, target):
     assert pruned == achieved                 # the same constants in the count and in the selection
     assert torch.equal(mask, mask_g)
     assert abs(achieved - target) < 2e-3
+
+
+@pytest.mark.parametrize("R,n,misalign", [(96, 640, False), (40, 1032, False), (33, 648, True)])
+def test_x2_reading_of_the_S_update_is_bit_exact(sp, R, n, misalign):
+    """SP_S_READING_X2 ("S = S - x_i^2"): sequential kernels, bit-exact against the oracle's mode
+    of the same name; the reading changes S by tens of percent, so it differs from the others."""
+    W = _gen(191 + n, (R, n), torch.float16, 0.02)
+    if misalign:
+        buf = torch.zeros(R * n + 1, dtype=W.dtype, device=W.device)
+        buf[1:] = W.reshape(-1)
+        W = buf[1:].view(R, n)
+    X = _activations(192, 1024, n, torch.float16)
+    counters = sp.new_counters()
+    with _ctx_with_stats(sp, [X], n) as ctx:
+        mask, out = ctx.sp_select_unstructured(
+            W, params=_ewma_params(sp, 0.5, s_update=sp.SP_S_READING_X2), counters=counters)
+        est, dev, L = ctx.sp_ewma_trace(W[:4].contiguous(),
+                                        sp.EwmaParams(0.125, 0.125, 0.5, sp.SP_S_READING_X2))
+        colsq = ctx.sp_get_stats()[0]
+    st = so.Stats(colsq.numpy().copy(), 1)
+    sel = so.select_ewma(P.bits(W), so.F16, st, 0.5, s_update=so.S_READING_X2, want_trace=True)
+    P.check_selection(mask, out, W, sel, None, strict=True)
+    assert int(counters[sp.SP_COUNTER_KEPT]) == int(sel.keep_bool(n).sum())
+    assert np.array_equal(L.cpu().numpy(), sel.L[:4])
+    thr = est.cpu().numpy() - np.float32(0.5) * dev.cpu().numpy()
+    assert np.array_equal(thr, sel.thr[:4])
+    other = so.select_ewma(P.bits(W), so.F16, st, 0.5, s_update=so.S_LITERAL_W2)
+    assert not np.array_equal(other.mask, sel.mask)
+
+
+def test_x2_reading_hand_trace_through_the_library(sp):
+    import os
+    g = {}
+    with open(os.path.join(os.path.dirname(__file__), "golden", "ewma_hand_trace_x2_reading.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                key, *vals = line.split()
+                g[key] = vals
+    W = torch.tensor([[float(v) for v in g["w"]]], dtype=torch.float16, device="cuda")
+    n = W.shape[1]
+    prm = sp.EwmaParams(float(g["alpha"][0]), float(g["beta"][0]), float(g["la"][0]),
+                        sp.SP_S_READING_X2)
+    with sp.Context(n) as ctx:
+        ctx.sp_set_stats(torch.tensor([float(v) for v in g["colsq"]], dtype=torch.float64), 1)
+        mask, out = ctx.sp_select_unstructured(W, params=prm)
+        est, dev, L = ctx.sp_ewma_trace(W, prm)
+    keep = so.unpack_mask(P.mask_np(mask), n)[0].astype(int).tolist()
+    assert keep == [int(v) for v in g["keep"]]
+    assert L.cpu().numpy()[0].tolist() == [float(v) for v in g["L"]]
+    thr = (est - prm.la * dev).cpu().numpy()[0].tolist()
+    assert thr == [float(v) for v in g["thr"]]

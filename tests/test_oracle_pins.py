@@ -553,3 +553,19 @@ def test_comparisons_with_nan_keep_the_weight_in_algorithm_1_hand_cases(case, s_
                              precision=precision)
         assert np.array_equal(sel.keep_bool(6)[0], _keep_bits(g[case + "_keep"][0]))
         assert sel.W_out[0, 1] == 0 and sel.W_out[0, 2] == W[0, 2]
+
+
+@pytest.mark.parametrize("precision", ["f32", "f64"])
+def test_hand_trace_x2_reading_of_the_S_update(precision):
+    g = _read_golden("ewma_hand_trace_x2_reading.txt")
+    n = len(g["w"])
+    sel = _run_trace(g, so.S_READING_X2, precision)
+    assert sel.L[0].tolist() == [float(v) for v in g["L"]]
+    assert sel.thr[0].tolist() == [float(v) for v in g["thr"]]
+    assert sel.keep_bool(n)[0].astype(int).tolist() == [int(v) for v in g["keep"]]
+    # the three readings part ways at column 2
+    frozen = _run_trace(g, so.S_FROZEN, precision)
+    printed = _run_trace(g, so.S_LITERAL_W2, precision)
+    assert frozen.L[0][2] == pytest.approx(float(g["L2_frozen"][0]), rel=3e-7)
+    assert printed.L[0][2] == pytest.approx(float(g["L2_printed"][0]), rel=3e-7)
+    assert frozen.L[0][:2].tolist() == printed.L[0][:2].tolist() == sel.L[0][:2].tolist()

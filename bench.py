@@ -61,11 +61,18 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=1)
     ap.add_argument("--blocks", type=int, default=0,
                     help="profiling aid: prune only the first BLOCKS blocks (0 = the whole model)")
+    ap.add_argument("--seqs", type=int, default=0,
+                    help="profiling aid: calibration sequences (0 = the workload's own number); "
+                         "keeps the resident activations to a few GB for an ncu capture")
     ap.add_argument("--mode-index", type=int, default=0,
                     help="which of the workload's sparsities / N:M patterns to run")
     ap.add_argument("--graph", action="store_true",
                     help="replay the whole-model pass as one CUDA graph in the timed region "
                          "(for launch-bound small models)")
+    ap.add_argument("--split", default="models", choices=["models", "blocks", "tokens"],
+                    help="with N > 1 ranks: every rank prunes its own model (weak scaling, the "
+                         "default), or the ranks share ONE model by blocks (no exchange) or by "
+                         "calibration tokens and rows (one small all-reduce per layer input)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ewma-blocks", type=int, default=6,
                     help="blocks of LLaMA-3-8B-shaped layers the EWMA selection kernel is timed "
@@ -357,11 +364,21 @@ def gpu_arm(args):
     w = synth.WORKLOADS[args.workload]
     if args.blocks > 0:
         w = synth.Workload(**{**w.__dict__, "blocks": min(args.blocks, w.blocks)})
+    if args.seqs > 0:
+        w = synth.Workload(**{**w.__dict__, "n_seqs": min(args.seqs, w.n_seqs)})
     arg = mode_args(w)[args.mode_index]
     batch_tokens = args.batch_seqs * w.seq_len
-    # weak scaling: rank r prunes its own model (seed offset r)
-    mb = pipeline.allocate_model(w, device, model_seed_offset=sharding.unit_of_rank(rank, world))
+    # weak scaling: rank r prunes its own model (seed offset r); with --split blocks / tokens
+    # all ranks hold the same model and share its work
+    shared = args.split != "models"
+    mb = pipeline.allocate_model(
+        w, device, model_seed_offset=0 if shared else sharding.unit_of_rank(rank, world))
     torch.cuda.synchronize()
+
+    def one_pass():
+        if shared:
+            return pipeline.prune_model_split(mb, arg, batch_tokens, rank, world, args.split)
+        return pipeline.prune_model(mb, arg, batch_tokens)
 
     def barrier():
         torch.cuda.synchronize()
@@ -370,7 +387,7 @@ def gpu_arm(args):
         torch.cuda.synchronize()
 
     for _ in range(max(args.warmup, 3)):
-        pipeline.prune_model(mb, arg, batch_tokens)
+        one_pass()
     barrier()
 
     uuid = None
@@ -383,6 +400,8 @@ def gpu_arm(args):
 
     phase_events = []
     graph = None
+    if args.graph and shared:
+        raise SystemExit("--graph replays the single-model pass; it cannot be combined with --split")
     if args.graph:
         graph, counts = pipeline.capture_model_graph(mb, arg, batch_tokens)
         for _ in range(3):
@@ -398,7 +417,7 @@ def gpu_arm(args):
     else:
         counts = None
         for _ in range(args.steps):
-            counts = pipeline.prune_model(mb, arg, batch_tokens)
+            counts = one_pass()
     stop.record()
     barrier()
     clocks = sampler.stop()
@@ -415,7 +434,7 @@ def gpu_arm(args):
     torch.cuda.synchronize()
 
     elapsed_ms = sharding.max_over_ranks(elapsed_ms, world, device)
-    total_weights = w.total_weights() * world
+    total_weights = w.total_weights() * (1 if shared else world)
     value = total_weights * args.steps / (elapsed_ms * 1e-3)
 
     calib_ms = sum(a.elapsed_time(b) for k, a, b, _ in phase_events if k == "calib")
@@ -489,7 +508,7 @@ def gpu_arm(args):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": elapsed_ms / args.steps,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "higher_is_better": True, "scaling": "strong" if shared else "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "weights_dtype": w.dtype, "mode": w.mode,
                    "mode_arg": str(arg), "blocks": w.blocks, "total_weights": w.total_weights(),
@@ -503,7 +522,12 @@ def gpu_arm(args):
                    "launch": "cuda graph replay" if graph is not None else "stream launches",
                    "calib_flags": "SP_CALIB_X_COMPLETE (the activations are resident and complete "
                                   "long before the step starts)",
-                   "parallelism": "independent models per rank" if world > 1 else "single GPU"},
+                   "parallelism": ("single GPU" if world == 1 else
+                                   "independent models per rank" if not shared else
+                                   "one model, blocks split over ranks (no exchange)"
+                                   if args.split == "blocks" else
+                                   "one model, calibration tokens and rows split over ranks "
+                                   "(one all-reduce of d_in + 1 doubles per layer input)")},
         "whole_model_prune_s": {"calib": calib_ms / args.steps * 1e-3,
                                 "finalize": final_ms / args.steps * 1e-3,
                                 "select_apply": select_ms / args.steps * 1e-3,

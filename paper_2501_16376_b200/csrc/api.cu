@@ -7,6 +7,8 @@
 #include <new>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "sp_internal.h"
 
 namespace sp {
@@ -43,6 +45,17 @@ class DeviceGuard {
     cudaError_t err_ = cudaSuccess;
 };
 
+// NVTX range around one entry point: shows up in a timeline profile under the call's name;
+// costs a function-pointer test when no profiler is attached.
+class CallRange {
+   public:
+    explicit CallRange(const char *name) { nvtxRangePushA(name); }
+    ~CallRange() { nvtxRangePop(); }
+    CallRange(const CallRange &) = delete;
+    CallRange &operator=(const CallRange &) = delete;
+};
+#define SP_CALL_RANGE() CallRange sp_call_range__(__func__)
+
 static bool valid_dtype(sp_dtype d) { return d == SP_F16 || d == SP_BF16; }
 
 static sp_status ensure_finalized(sp_ctx *ctx, cudaStream_t stream) {
@@ -72,6 +85,7 @@ using namespace sp;
 extern "C" {
 
 sp_status sp_create(sp_ctx **out, int64_t d_in, int device) {
+    SP_CALL_RANGE();
     if (out == nullptr) return SP_ERR_INVALID_ARG;
     *out = nullptr;
     if (d_in < 1 || d_in > kMaxDin) return SP_ERR_SHAPE;
@@ -126,6 +140,7 @@ sp_status sp_create(sp_ctx **out, int64_t d_in, int device) {
 }
 
 sp_status sp_destroy(sp_ctx *ctx) {
+    SP_CALL_RANGE();
     if (ctx == nullptr) return SP_OK;
     DeviceGuard guard(ctx->device);
     cudaDeviceSynchronize();
@@ -141,6 +156,7 @@ sp_status sp_destroy(sp_ctx *ctx) {
 }
 
 sp_status sp_calib_reset(sp_ctx *ctx, sp_stream stream) {
+    SP_CALL_RANGE();
     (void)stream;  // the partial sums are overwritten, not cleared, by the next batch
     if (ctx == nullptr) return SP_ERR_INVALID_ARG;
     ctx->n_tokens = 0;
@@ -151,6 +167,7 @@ sp_status sp_calib_reset(sp_ctx *ctx, sp_stream stream) {
 
 sp_status sp_calib_accumulate_ex(sp_ctx *ctx, const void *X, sp_dtype dtype, int64_t n_tokens,
                                  int64_t ldx, unsigned flags, sp_stream stream) {
+    SP_CALL_RANGE();
     if (ctx == nullptr) return SP_ERR_INVALID_ARG;
     if (!valid_dtype(dtype)) return SP_ERR_DTYPE;
     if (n_tokens < 0 || (flags & ~static_cast<unsigned>(SP_CALIB_X_COMPLETE)) != 0u)
@@ -166,11 +183,13 @@ sp_status sp_calib_accumulate_ex(sp_ctx *ctx, const void *X, sp_dtype dtype, int
 
 sp_status sp_calib_accumulate(sp_ctx *ctx, const void *X, sp_dtype dtype, int64_t n_tokens,
                               int64_t ldx, sp_stream stream) {
+    SP_CALL_RANGE();
     return sp_calib_accumulate_ex(ctx, X, dtype, n_tokens, ldx, 0u, stream);
 }
 
 sp_status sp_get_stats(sp_ctx *ctx, double *colsq_host, double *S_host, float *factor_host,
                        int64_t *n_tokens_host, sp_stream stream) {
+    SP_CALL_RANGE();
     if (ctx == nullptr) return SP_ERR_INVALID_ARG;
     if (n_tokens_host != nullptr) *n_tokens_host = ctx->n_tokens;
     if (ctx->n_tokens <= 0) return SP_ERR_STATE;
@@ -194,6 +213,7 @@ sp_status sp_get_stats(sp_ctx *ctx, double *colsq_host, double *S_host, float *f
 }
 
 sp_status sp_set_stats(sp_ctx *ctx, const double *colsq_host, int64_t n_tokens, sp_stream stream) {
+    SP_CALL_RANGE();
     if (ctx == nullptr || colsq_host == nullptr || n_tokens <= 0) return SP_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     if (guard.error() != cudaSuccess) return cuda_fail(guard.error());
@@ -214,6 +234,7 @@ sp_status sp_set_stats(sp_ctx *ctx, const double *colsq_host, int64_t n_tokens, 
 sp_status sp_calib_stats_noalloc(const void *X, sp_dtype dtype, int64_t n_tokens, int64_t d_in,
                                  int64_t ldx, double *colsq_out, float *factor_out, double *S_out,
                                  sp_stream stream) {
+    SP_CALL_RANGE();
     if (!valid_dtype(dtype)) return SP_ERR_DTYPE;
     if (X == nullptr || n_tokens < 1) return SP_ERR_INVALID_ARG;
     if (d_in < 1 || d_in > calib_static_max_d_in()) return SP_ERR_SHAPE;
@@ -227,6 +248,7 @@ sp_status sp_calib_stats_noalloc(const void *X, sp_dtype dtype, int64_t n_tokens
 
 sp_status sp_score(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows, int64_t ldw,
                    float *scores_out, sp_stream stream) {
+    SP_CALL_RANGE();
     if (ctx == nullptr) return SP_ERR_INVALID_ARG;
     if (scores_out != nullptr) {
         sp_status st = check_matrix_args(ctx, W, dtype, n_rows, ldw, nullptr, 0);
@@ -242,6 +264,7 @@ sp_status sp_score(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows, i
 }
 
 sp_status sp_la_for_sparsity(float sparsity, float *la_out) {
+    SP_CALL_RANGE();
     if (la_out == nullptr || !(sparsity > 0.0f) || !(sparsity < 1.0f)) return SP_ERR_INVALID_ARG;
     // Table 3: pruning ratio (%) -> la.
     static const double pct[5] = {50.0, 60.0, 70.0, 80.0, 90.0};
@@ -268,6 +291,7 @@ sp_status sp_select_unstructured_ex(sp_ctx *ctx, const void *W, sp_dtype dtype, 
                                     int64_t ldw, const sp_ewma_params *params, uint32_t *mask_out,
                                     void *W_out, int64_t ldo, unsigned long long *counters,
                                     sp_stream stream) {
+    SP_CALL_RANGE();
     sp_status st = check_matrix_args(ctx, W, dtype, n_rows, ldw, W_out, ldo);
     if (st != SP_OK) return st;
     if (params == nullptr) return SP_ERR_INVALID_ARG;
@@ -289,6 +313,7 @@ sp_status sp_select_unstructured_ex(sp_ctx *ctx, const void *W, sp_dtype dtype, 
 sp_status sp_select_unstructured(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
                                  int64_t ldw, float sparsity, uint32_t *mask_out, void *W_out,
                                  int64_t ldo, unsigned long long *counters, sp_stream stream) {
+    SP_CALL_RANGE();
     sp_ewma_params p;
     p.alpha = 0.125f;  // Section 4.2
     p.beta = 0.125f;
@@ -316,6 +341,7 @@ static sp_status group_jobs(const sp_ctx *ctx, const sp_matrix *mats, int n_mats
 sp_status sp_select_unstructured_group_ex(sp_ctx *ctx, const sp_matrix *mats, int n_mats,
                                           sp_dtype dtype, const sp_ewma_params *params,
                                           unsigned long long *counters, sp_stream stream) {
+    SP_CALL_RANGE();
     EwmaLaunchJob jobs[SP_MAX_GROUP];
     sp_status st = group_jobs(ctx, mats, n_mats, dtype, jobs);
     if (st != SP_OK) return st;
@@ -338,6 +364,7 @@ sp_status sp_select_unstructured_group_ex(sp_ctx *ctx, const sp_matrix *mats, in
 sp_status sp_select_unstructured_group(sp_ctx *ctx, const sp_matrix *mats, int n_mats,
                                        sp_dtype dtype, float sparsity,
                                        unsigned long long *counters, sp_stream stream) {
+    SP_CALL_RANGE();
     sp_ewma_params p;
     p.alpha = 0.125f;  // Section 4.2
     p.beta = 0.125f;
@@ -349,6 +376,7 @@ sp_status sp_select_unstructured_group(sp_ctx *ctx, const sp_matrix *mats, int n
 
 sp_status sp_select_nm_group(sp_ctx *ctx, const sp_matrix *mats, int n_mats, sp_dtype dtype, int N,
                              int M, sp_stream stream) {
+    SP_CALL_RANGE();
     EwmaLaunchJob jobs[SP_MAX_GROUP];
     sp_status st = group_jobs(ctx, mats, n_mats, dtype, jobs);
     if (st != SP_OK) return st;
@@ -367,6 +395,7 @@ sp_status sp_select_nm_group(sp_ctx *ctx, const sp_matrix *mats, int n_mats, sp_
 sp_status sp_ewma_trace(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows, int64_t ldw,
                         const sp_ewma_params *params, float *est_out, float *dev_out,
                         float *scores_out, sp_stream stream) {
+    SP_CALL_RANGE();
     sp_status st = check_matrix_args(ctx, W, dtype, n_rows, ldw, nullptr, 0);
     if (st != SP_OK) return st;
     if (params == nullptr || !(params->alpha > 0.0f) || !(params->alpha <= 1.0f) ||
@@ -387,6 +416,7 @@ sp_status sp_ewma_trace(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_ro
 sp_status sp_search_la(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows, int64_t ldw,
                        float target_sparsity, float alpha, float beta, int iterations,
                        float *la_out, double *achieved_out, sp_stream stream) {
+    SP_CALL_RANGE();
     sp_status st = check_matrix_args(ctx, W, dtype, n_rows, ldw, nullptr, 0);
     if (st != SP_OK) return st;
     if (la_out == nullptr || !(target_sparsity > 0.0f) || !(target_sparsity < 1.0f) ||
@@ -444,6 +474,7 @@ sp_status sp_search_la(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_row
 sp_status sp_select_nm(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows, int64_t ldw,
                        int N, int M, uint32_t *mask_out, void *W_out, int64_t ldo,
                        sp_stream stream) {
+    SP_CALL_RANGE();
     sp_status st = check_matrix_args(ctx, W, dtype, n_rows, ldw, W_out, ldo);
     if (st != SP_OK) return st;
     if (M != 4 && M != 8) return SP_ERR_INVALID_ARG;
@@ -461,6 +492,7 @@ sp_status sp_select_nm(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_row
 sp_status sp_select_24_compressed(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
                                   int64_t ldw, void *values_out, int64_t ldv, uint32_t *meta_out,
                                   sp_stream stream) {
+    SP_CALL_RANGE();
     sp_status st = check_matrix_args(ctx, W, dtype, n_rows, ldw, nullptr, 0);
     if (st != SP_OK) return st;
     if (n_rows > 0 && (values_out == nullptr || meta_out == nullptr)) return SP_ERR_INVALID_ARG;
@@ -476,6 +508,7 @@ sp_status sp_select_24_compressed(sp_ctx *ctx, const void *W, sp_dtype dtype, in
 
 sp_status sp_apply_mask(const void *W, sp_dtype dtype, int64_t n_rows, int64_t n_cols, int64_t ldw,
                         const uint32_t *mask, void *W_out, int64_t ldo, sp_stream stream) {
+    SP_CALL_RANGE();
     if (!valid_dtype(dtype)) return SP_ERR_DTYPE;
     if (n_rows < 0 || n_cols < 0) return SP_ERR_INVALID_ARG;
     if ((W == nullptr || mask == nullptr || W_out == nullptr) && n_rows * n_cols != 0)
@@ -488,6 +521,7 @@ sp_status sp_apply_mask(const void *W, sp_dtype dtype, int64_t n_rows, int64_t n
 
 sp_status sp_calib_accumulate_host(sp_ctx *ctx, const void *X_host, sp_dtype dtype,
                                    int64_t n_tokens, int64_t ldx, sp_stream stream) {
+    SP_CALL_RANGE();
     if (ctx == nullptr) return SP_ERR_INVALID_ARG;
     if (!valid_dtype(dtype)) return SP_ERR_DTYPE;
     if (n_tokens < 0) return SP_ERR_INVALID_ARG;
@@ -502,6 +536,7 @@ sp_status sp_calib_accumulate_host(sp_ctx *ctx, const void *X_host, sp_dtype dty
 sp_status sp_select_nm_host(sp_ctx *ctx, const void *W_host, sp_dtype dtype, int64_t n_rows,
                             int64_t ldw, int N, int M, uint32_t *mask_host, void *W_out_host,
                             int64_t ldo, sp_stream stream) {
+    SP_CALL_RANGE();
     sp_status st = check_matrix_args(ctx, W_host, dtype, n_rows, ldw, W_out_host, ldo);
     if (st != SP_OK) return st;
     if (M != 4 && M != 8) return SP_ERR_INVALID_ARG;
@@ -520,6 +555,7 @@ sp_status sp_select_unstructured_host(sp_ctx *ctx, const void *W_host, sp_dtype 
                                       int64_t n_rows, int64_t ldw, float sparsity,
                                       uint32_t *mask_host, void *W_out_host, int64_t ldo,
                                       sp_stream stream) {
+    SP_CALL_RANGE();
     sp_status st = check_matrix_args(ctx, W_host, dtype, n_rows, ldw, W_out_host, ldo);
     if (st != SP_OK) return st;
     sp_ewma_params p;

@@ -175,6 +175,57 @@ def prune_model(mb: ModelBuffers, mode_arg, batch_tokens: int, phase_events=None
     return {"calib": n_calib, "finalize": n_final, "select": n_select}
 
 
+def prune_model_split(mb: ModelBuffers, mode_arg, batch_tokens: int, rank: int, world: int,
+                      split: str, stream=None):
+    """One pass over ONE model shared by `world` ranks (strong scaling).
+
+    split == "blocks": rank r prunes the blocks sharding.assign_units gives it, on its own; no
+    exchange at all.
+    split == "tokens": for every block and layer input, rank r accumulates its share of the
+    calibration tokens, the ranks sum their column sums of squares with one all-reduce of
+    d_in + 1 doubles (sharding.merge_calibration), and rank r then prunes its share of the rows
+    of every layer that reads the input.  Masks and outputs of rows a rank does not own are left
+    untouched.  Returns launch counts."""
+    from . import sharding
+    w = mb.workload
+    n_calib = n_final = n_select = 0
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    blocks = sharding.assign_units(w.blocks, world, rank) if split == "blocks" else range(w.blocks)
+    for b in blocks:
+        for name, d_in in w.input_widths().items():
+            ctx = mb.ctxs[name]
+            X = mb.acts[name]
+            if split == "tokens":
+                share = sharding.token_share(X.shape[0], world, rank, align=w.seq_len)
+                ctx.sp_calib_reset(stream)
+                for t0 in range(share.start, share.stop, batch_tokens):
+                    ctx.sp_calib_accumulate(X[t0:min(share.stop, t0 + batch_tokens)], stream, True)
+                    n_calib += 1
+                sharding.merge_calibration(ctx, world, mb.device, stream)
+            else:
+                n_calib += calibrate_input(ctx, X, batch_tokens, stream, True)
+            ctx.sp_score(None, stream=stream)
+            n_final += 1
+            idx = [li for li, layer in enumerate(w.layers) if layer.input == name]
+            Ws, masks, outs = [], [], []
+            for li in idx:
+                rows = (sharding.row_share(w.layers[li].d_out, world, rank)
+                        if split == "tokens" else range(w.layers[li].d_out))
+                if len(rows) == 0:
+                    continue
+                Ws.append(mb.weights[b][li][rows.start:rows.stop])
+                masks.append(mb.masks[b][li][rows.start:rows.stop])
+                outs.append(mb.outputs[b][li][rows.start:rows.stop])
+            before = sp.sp_launch_count()
+            if len(Ws) > 1:
+                select_group(ctx, w, Ws, masks, outs, mode_arg, stream)
+            elif len(Ws) == 1:
+                select_layer(ctx, w, Ws[0], masks[0], outs[0], mode_arg, stream)
+            n_select += sp.sp_launch_count() - before
+    return {"calib": n_calib, "finalize": n_final, "select": n_select}
+
+
 def capture_model_graph(mb: ModelBuffers, mode_arg, batch_tokens: int):
     """Captures one whole-model pass into a CUDA graph (for models whose layers are so small
     that the pass is bound by launch overhead).  The library's calls only enqueue kernels on the

@@ -29,6 +29,21 @@ def assign_units(n_units: int, world: int, rank: int) -> range:
     return range(begin, begin + base + (1 if rank < extra else 0))
 
 
+def token_share(n_tokens: int, world: int, rank: int, align: int = 1) -> range:
+    """Token-sharded calibration: the contiguous share of the calibration tokens that `rank`
+    accumulates; shares are balanced in units of `align` tokens (e.g. one sequence)."""
+    if align < 1 or n_tokens < 0:
+        raise ValueError("bad partition arguments")
+    units = assign_units((n_tokens + align - 1) // align, world, rank)
+    return range(min(units.start * align, n_tokens), min(units.stop * align, n_tokens))
+
+
+def row_share(n_rows: int, world: int, rank: int) -> range:
+    """Row-sharded selection: the contiguous rows of a layer that `rank` prunes (rows are
+    independent problems, Algorithm 1 "parallel calculation for each row")."""
+    return assign_units(n_rows, world, rank)
+
+
 def max_over_ranks(value: float, world: int, device=None) -> float:
     """Max of a per-rank number (the step time) over the process group."""
     if world <= 1 or not dist.is_initialized():

@@ -42,10 +42,12 @@ CALIB_BYTES_PER_ELEMENT = 2.0
 # (32768-token calibration batches; selection launches grouped per layer input).
 # Keys: calibration -> d_in; selection -> (total rows of the launch, d_in).  Shapes that were
 # not captured, and kernels changed since, report null.
-NCU_CALIB_TRAFFIC = {}
+NCU_CALIB_TRAFFIC = {4096: 272.0e6, 11008: 725.1e6}
 NCU_SELECT_TRAFFIC = {
-    "select_nm_stream_kernel": {},
-    "ewma_pair_scan_kernel": {},
+    "select_nm_stream_kernel": {(12288, 4096): 156.0e6, (4096, 4096): 34.3e6,
+                                (22016, 4096): 318.4e6, (4096, 11008): 131.4e6},
+    "ewma_pair_scan_kernel": {(6144, 4096): 55.3e6, (4096, 4096): 34.4e6,
+                              (28672, 4096): 430.4e6, (4096, 14336): 190.0e6},
 }
 
 
@@ -249,7 +251,7 @@ def reference_arm(args):
 # ---------------------------------------------------------------------------- GPU arm
 
 # DRAM bytes per launch of the EWMA selection kernel (ncu, see profiles/): (rows, d_in) -> bytes
-NCU_EWMA_TRAFFIC = {}
+NCU_EWMA_TRAFFIC = NCU_SELECT_TRAFFIC["ewma_pair_scan_kernel"]
 
 
 def ewma_block(device, peak, peak_kind, blocks=4):

@@ -66,15 +66,23 @@ typedef enum { SP_F16 = 0, SP_BF16 = 1 } sp_dtype;
 typedef enum {
     SP_S_GATED = 0,      /* Algorithm 1 as printed, at scan speed: rows are scanned in parallel with
                             S at its initial value; a row holding a weight that could change S is
-                            detected and re-evaluated sequentially in the same call, so the
-                            result is that of SP_S_LITERAL_W2 for every row (the default) */
+                            detected before that weight's tile is stored and finished
+                            sequentially from there in the same kernel, so the result is the
+                            printed algorithm for every row (the default) */
     SP_S_LITERAL_W2 = 1, /* the printed update, evaluated sequentially along every row */
     SP_S_FROZEN = 2,     /* S keeps its initial value whatever is pruned */
-    SP_S_READING_X2 = 3  /* the other conceivable reading of that row of Table 2: S is a sum of
+    SP_S_READING_X2 = 3, /* the other conceivable reading of that row of Table 2: S is a sum of
                             x^2, and a pruned weight takes its channel's x_i^2 out of it
                             ("S = S - x_i^2"); evaluated sequentially along every row.  This
                             changes S by tens of percent and is not what the paper prints:
                             offered for comparison */
+    SP_S_LITERAL_SCAN = 4 /* the printed update again, but rows scanned by whole warps: every
+                            256-column tile is decided by fix-point sweeps (decide with the S the
+                            previous sweep's decisions imply, prefix-sum the pruned w^2, repeat
+                            until nothing changes; a tile that does not settle in 8 sweeps hands
+                            the row to the sequential walk and counts in SP_COUNTER_S_HAZARD).
+                            Same decisions as SP_S_LITERAL_W2 up to re-association (the tolerance
+                            of the scans); several times faster when rows are few and long */
 } sp_s_update;
 
 /* Parameters of Algorithm 1 (alpha, beta: Table 2; la: Table 3). */

@@ -20,7 +20,7 @@ SP_OK = 0
 SP_ERR_INVALID_ARG, SP_ERR_SHAPE, SP_ERR_DTYPE, SP_ERR_STATE = 1, 2, 3, 4
 SP_ERR_DEGENERATE, SP_ERR_CUDA, SP_ERR_NOMEM = 5, 6, 7
 SP_F16, SP_BF16 = 0, 1
-SP_S_GATED, SP_S_LITERAL_W2, SP_S_FROZEN, SP_S_READING_X2 = 0, 1, 2, 3
+SP_S_GATED, SP_S_LITERAL_W2, SP_S_FROZEN, SP_S_READING_X2, SP_S_LITERAL_SCAN = 0, 1, 2, 3, 4
 SP_COUNTER_KEPT, SP_COUNTER_S_HAZARD, SP_NUM_COUNTERS = 0, 1, 2
 SP_CALIB_X_COMPLETE = 1
 

@@ -299,7 +299,8 @@ sp_status sp_select_unstructured_ex(sp_ctx *ctx, const void *W, sp_dtype dtype, 
         !(params->beta <= 1.0f) || !std::isfinite(params->la))
         return SP_ERR_INVALID_ARG;
     if (params->s_update != SP_S_GATED && params->s_update != SP_S_FROZEN &&
-        params->s_update != SP_S_LITERAL_W2 && params->s_update != SP_S_READING_X2)
+        params->s_update != SP_S_LITERAL_W2 && params->s_update != SP_S_READING_X2 &&
+        params->s_update != SP_S_LITERAL_SCAN)
         return SP_ERR_INVALID_ARG;
     if (ctx->n_tokens <= 0) return SP_ERR_STATE;
     DeviceGuard guard(ctx->device);
@@ -350,7 +351,8 @@ sp_status sp_select_unstructured_group_ex(sp_ctx *ctx, const sp_matrix *mats, in
         !(params->beta <= 1.0f) || !std::isfinite(params->la))
         return SP_ERR_INVALID_ARG;
     if (params->s_update != SP_S_GATED && params->s_update != SP_S_FROZEN &&
-        params->s_update != SP_S_LITERAL_W2 && params->s_update != SP_S_READING_X2)
+        params->s_update != SP_S_LITERAL_W2 && params->s_update != SP_S_READING_X2 &&
+        params->s_update != SP_S_LITERAL_SCAN)
         return SP_ERR_INVALID_ARG;
     if (ctx->n_tokens <= 0) return SP_ERR_STATE;
     DeviceGuard guard(ctx->device);
@@ -402,7 +404,8 @@ sp_status sp_ewma_trace(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_ro
         !(params->beta > 0.0f) || !(params->beta <= 1.0f) || !std::isfinite(params->la))
         return SP_ERR_INVALID_ARG;
     if (params->s_update != SP_S_GATED && params->s_update != SP_S_FROZEN &&
-        params->s_update != SP_S_LITERAL_W2 && params->s_update != SP_S_READING_X2)
+        params->s_update != SP_S_LITERAL_W2 && params->s_update != SP_S_READING_X2 &&
+        params->s_update != SP_S_LITERAL_SCAN)
         return SP_ERR_INVALID_ARG;
     if (ctx->n_tokens <= 0) return SP_ERR_STATE;
     DeviceGuard guard(ctx->device);

@@ -81,79 +81,6 @@ struct EwmaJobTable {
     EwmaJob job[kEwmaMaxJobs];
 };
 
-// Algorithm 1 exactly as printed along one row from column i_begin (a multiple of 32) on, by
-// one thread, binary32 with one rounding per operation; est / dev are the state before that
-// column (ignored for column 0, where est starts at L_0).  subtract_x2: the other reading of
-// Table 2's row S, a pruned weight takes its channel's x_i^2 (not w_i^2) out of S.  Element-wise access with bounds
-// checks.  While S still has its initial value the per-channel factor computed at finalisation
-// is used: it was formed by the same three operations from the same S, so the result is
-// bit-identical to recomputing it; once a pruned weight has changed S the factor is recomputed
-// for every element.  Returns the number of kept weights.
-template <bool BF16>
-__device__ __forceinline__ unsigned long long literal_walk(
-    const uint16_t *__restrict__ wrow, uint16_t *__restrict__ orow, uint32_t *__restrict__ mrow,
-    int64_t n, int64_t i_begin, float est, float dev, const double *__restrict__ colsq,
-    const float *__restrict__ factor, float S0, float alpha, float beta, float la,
-    bool subtract_x2 = false) {
-    const float one_minus_alpha = __fsub_rn(1.0f, alpha);
-    const float one_minus_beta = __fsub_rn(1.0f, beta);
-    float S = S0;
-    uint32_t word = 0;
-    unsigned long long kept = 0;
-    // two chunks are kept in flight ahead of the one being evaluated
-    uint32_t ahead[2][4];
-    load8<false, true>(wrow, i_begin, n, ahead[0]);
-    load8<false, true>(wrow, i_begin + 8, n, ahead[1]);
-    for (int64_t i0 = i_begin; i0 < n; i0 += 8) {
-        uint32_t p[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            p[k] = ahead[0][k];
-            ahead[0][k] = ahead[1][k];
-        }
-        load8<false, true>(wrow, i0 + 16, n, ahead[1]);
-        float w[8];
-        unpack8<BF16>(p, w);
-        uint32_t keep8 = 0;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int64_t i = i0 + j;
-            if (i < n) {
-                float c;
-                if (S == S0) {
-                    c = __ldg(factor + i);
-                } else {
-                    const float u = __fdiv_rn(static_cast<float>(colsq[i]), S);
-                    c = __fdiv_rn(0.5f, __fsub_rn(1.0f, u));
-                }
-                const float w2 = __fmul_rn(w[j], w[j]);
-                const float L = __fmul_rn(w2, c);
-                if (i == 0) est = L;
-                const float thr = __fsub_rn(est, __fmul_rn(la, dev));
-                if (L < thr) {
-                    S = __fsub_rn(S, subtract_x2 ? static_cast<float>(colsq[i]) : w2);
-                } else {
-                    keep8 |= 1u << j;
-                }
-                est = __fadd_rn(__fmul_rn(one_minus_alpha, est), __fmul_rn(alpha, L));
-                dev = __fadd_rn(__fmul_rn(one_minus_beta, dev),
-                                __fmul_rn(beta, fabsf(__fsub_rn(est, L))));
-            }
-        }
-        kept += __popc(keep8);
-        if (orow != nullptr) {
-            zero_pruned(p, keep8);
-            store8<false>(orow, i0, n, p);
-        }
-        word |= keep8 << (i0 & 31);
-        if ((i0 & 31) == 24 || i0 + 8 >= n) {
-            if (mrow != nullptr) mrow[i0 >> 5] = word;
-            word = 0;
-        }
-    }
-    return kept;
-}
-
 // Drift gate: the rest of a row, from column `col` on, for a scan kernel that had to leave it
 // (est, dev: the state of Algorithm 1 before that column).  Rarely taken, kept out of line.
 template <bool BF16>
@@ -879,6 +806,15 @@ sp_status launch_select_ewma(const sp_ctx *ctx, const EwmaLaunchJob *jobs_in, in
             if (j.W_out != nullptr) q.W_out = static_cast<uint16_t *>(j.W_out) + r0 * j.ldo;
             if (j.mask != nullptr) q.mask = j.mask + r0 * words;
         }
+    }
+    if (p.s_update == SP_S_LITERAL_SCAN) {
+        for (int i = 0; i < n_pieces; ++i) {
+            const EwmaLaunchJob &j = pieces[i];
+            sp_status st = launch_ewma_sweep(ctx, j.W, dtype, j.n_rows, j.ldw, p, j.mask, j.W_out,
+                                             j.ldo, counters, stream);
+            if (st != SP_OK) return st;
+        }
+        return SP_OK;
     }
     if (p.s_update == SP_S_LITERAL_W2 || p.s_update == SP_S_READING_X2) {
         for (int i = 0; i < n_pieces; ++i) {

@@ -138,6 +138,11 @@ sp_status launch_search_la_device(sp_ctx *ctx, const void *W, sp_dtype dtype, in
                                   int iterations, float *la_out, double *achieved_out,
                                   cudaStream_t stream);
 
+// select_ewma_sweep.cu
+sp_status launch_ewma_sweep(const sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,
+                            int64_t ldw, const sp_ewma_params &p, uint32_t *mask, void *W_out,
+                            int64_t ldo, unsigned long long *counters, cudaStream_t stream);
+
 // select_ewma_tiled.cu
 sp_status launch_ewma_literal_tiled(const sp_ctx *ctx, const void *W, sp_dtype dtype,
                                     int64_t n_rows, int64_t ldw, const sp_ewma_params &p,

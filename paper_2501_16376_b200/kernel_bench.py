@@ -11,7 +11,8 @@ per run: microseconds per call, algorithmic GB/s (4.125 B per weight for the fus
 3.125 B for the compressed 2:4 form, 2 B per activation element for the statistics), and the
 fraction of the measured copy rate when MEASURED_PEAKS.json is present.
 
-Calls: ewma (default mode, drift gate on) | ewma-frozen | ewma-literal | ewma-x2 | nm |
+Calls: ewma (default mode, drift gate on) | ewma-frozen | ewma-literal | ewma-literal-scan |
+ewma-x2 | nm |
 compressed24 | calib | search (24 counting passes).  --few N limits the number of buffers (for a
 profiler capture that should see only a handful of launches).
 """
@@ -38,7 +39,7 @@ def _peak():
 
 
 def run(call: str, rows: int, cols: int, dtype, nm=(2, 4), reps: int = 5, few: int = 0,
-        calib_tokens: int = 4096):
+        calib_tokens: int = 4096, stats_scale: float = 0.0):
     dev = torch.device("cuda", torch.cuda.current_device())
     g = torch.Generator(device=dev)
     g.manual_seed(1)
@@ -59,11 +60,16 @@ def run(call: str, rows: int, cols: int, dtype, nm=(2, 4), reps: int = 5, few: i
         ctx = sp.Context(cols)
         X = torch.randn(calib_tokens, cols, device=dev, generator=g).to(dtype)
         ctx.sp_calib_accumulate(X)
+        if stats_scale > 0.0:
+            gen = torch.Generator().manual_seed(2)
+            ctx.sp_set_stats((1.0 + torch.rand(cols, generator=gen, dtype=torch.float64))
+                             * stats_scale, calib_tokens)
         ctx.sp_score(None)
         bytes_per_call = rows * cols * 4.125
         if call.startswith("ewma"):
             mode = {"ewma": sp.SP_S_GATED, "ewma-frozen": sp.SP_S_FROZEN,
-                    "ewma-literal": sp.SP_S_LITERAL_W2, "ewma-x2": sp.SP_S_READING_X2}[call]
+                    "ewma-literal": sp.SP_S_LITERAL_W2, "ewma-x2": sp.SP_S_READING_X2,
+                    "ewma-literal-scan": sp.SP_S_LITERAL_SCAN}[call]
             prm = sp.EwmaParams(0.125, 0.125, 0.5, mode)
 
             def one(i):
@@ -130,6 +136,9 @@ def main(argv=None):
     ap.add_argument("--nm", default="2:4")
     ap.add_argument("--reps", type=int, default=5)
     ap.add_argument("--few", type=int, default=0)
+    ap.add_argument("--stats-scale", type=float, default=0.0,
+                    help="replace the calibration statistics by uniform(1,2) * SCALE per channel "
+                         "(e.g. 1e-3: S small enough for Algorithm 1's S update to matter)")
     args = ap.parse_args(argv)
     if not torch.cuda.is_available():
         raise SystemExit("kernel_bench needs a CUDA device")
@@ -137,7 +146,8 @@ def main(argv=None):
     nm = tuple(int(v) for v in args.nm.split(":"))
     for shape in args.shape or ["4096x4096"]:
         rows, cols = (int(v) for v in shape.lower().split("x"))
-        print(json.dumps(run(args.call, rows, cols, dtype, nm, args.reps, args.few)), flush=True)
+        print(json.dumps(run(args.call, rows, cols, dtype, nm, args.reps, args.few,
+                             stats_scale=args.stats_scale)), flush=True)
     return 0
 
 

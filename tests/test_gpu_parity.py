@@ -865,3 +865,46 @@ def test_x2_reading_hand_trace_through_the_library(sp):
     assert L.cpu().numpy()[0].tolist() == [float(v) for v in g["L"]]
     thr = (est - prm.la * dev).cpu().numpy()[0].tolist()
     assert thr == [float(v) for v in g["thr"]]
+
+
+# ------------------------------------------------------------------ fix-point sweeps (SP_S_LITERAL_SCAN)
+
+@pytest.mark.parametrize("R,n,mult,misalign", [
+    (64, 2048, 1e9, False),      # calibration scale: S cannot move, one sweep per tile
+    (64, 2048, 8.0, False),      # S = 8 x the sum of the pruned w^2 of a row: S moves by 12 %
+    (64, 2056, 1.5, False),      # ... S shrinks to a third along the row; ragged last tile
+    (33, 1000, 1.5, True),       # element-wise loads
+    (48, 640, 1.0, False),       # S comes down to a few percent of its start at the row's end
+])
+def test_literal_scan_matches_the_oracle_literal_mode(sp, R, n, mult, misalign):
+    """SP_S_LITERAL_SCAN against the oracle's literal evaluation of Algorithm 1, under the band
+    rule (the sweeps re-associate).  Not covered: statistics so small that S passes through zero
+    inside a row - there the factor 1/(1 - x^2/S) has a pole, and two evaluations that round S
+    differently (successive subtractions, prefix sum) legitimately decide differently."""
+    W = _gen(301 + n, (R, n), torch.float16, 0.02)
+    if misalign:
+        buf = torch.zeros(R * n + 1, dtype=W.dtype, device=W.device)
+        buf[1:] = W.reshape(-1)
+        W = buf[1:].view(R, n)
+    colsq = np.random.default_rng(7).uniform(1.0, 2.0, n)
+    colsq *= mult * n * 3.9e-5 / colsq.sum()      # a row's pruned w^2 add up to about n * 3.9e-5
+    counters = sp.new_counters()
+    with sp.Context(n) as ctx:
+        ctx.sp_set_stats(torch.from_numpy(colsq), 10)
+        mask, out = ctx.sp_select_unstructured(
+            W, params=_ewma_params(sp, 0.5, s_update=sp.SP_S_LITERAL_SCAN), counters=counters)
+    st = so.Stats(colsq.copy(), 10)
+    lit = so.select_ewma(P.bits(W), so.F16, st, 0.5, s_update=so.S_LITERAL_W2, want_trace=True)
+    fro = so.select_ewma(P.bits(W), so.F16, st, 0.5, s_update=so.S_FROZEN)
+    keep = so.unpack_mask(P.mask_np(mask), n)
+    want = lit.keep_bool(n)
+    diff = keep != want
+    assert not (diff & ~P.ewma_allowed_flips(lit)).any()
+    assert diff.sum() <= 2, diff.sum()
+    assert np.array_equal(P.bits(out), np.where(keep, P.bits(W), 0))
+    assert int(counters[sp.SP_COUNTER_KEPT]) == int(keep.sum())
+    if mult <= 1.0:
+        assert not np.array_equal(lit.mask, fro.mask)      # only here does the update change decisions
+    if mult >= 8.0:
+        assert int(counters[sp.SP_COUNTER_S_HAZARD]) == 0  # every tile settled
+    print("mult", mult, "rows handed to the walk:", int(counters[sp.SP_COUNTER_S_HAZARD]), "of", R)

@@ -21,8 +21,8 @@
  *     throws, traps or aborts.
  *   - A weight matrix W is [n_rows, d_in] row-major 16-bit floats with leading
  *     dimension ldw (elements, >= d_in): one row per output neuron, one column
- *     per input channel.  Rows are pruned independently (Section 2; Algorithm 1,
- *     "parallel calculation for each row").
+ *     per input channel.  Rows are pruned independently (Section 2; the row loop of
+ *     Algorithm 1 runs in parallel).
  *   - A mask is [n_rows, ceil(d_in/32)] uint32, row-major, no padding between
  *     rows; bit j of word k of a row is the keep flag of column 32k+j
  *     (1 = kept, 0 = pruned; bits past d_in are 0).
@@ -282,8 +282,8 @@ sp_status sp_select_nm(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_row
 
 /*
  * Grouped selection.  Layers that read the same input (q/k/v; gate/up) share a context and the
- * per-channel factors, and Algorithm 1 treats every row on its own ("parallel calculation for
- * each row"), so their rows can be pruned by one launch: small layers then no longer pay a
+ * per-channel factors, and Algorithm 1 treats every row on its own (its row loop is
+ * parallel), so their rows can be pruned by one launch: small layers then no longer pay a
  * launch and a ramp-up each.  mats (HOST array, 1 <= n_mats <= SP_MAX_GROUP) lists the
  * matrices, all of `dtype`; every entry follows the rules of the single-matrix call (mask_out
  * and W_out nullable, W_out may alias W exactly).  The result for each matrix is identical to
@@ -312,8 +312,8 @@ sp_status sp_select_nm_group(sp_ctx *ctx, const sp_matrix *mats /* host */, int 
 /*
  * Section 3.3, compressed output: 2:4 selection (exactly as sp_select_nm with N = 2, M = 4)
  * written as the kept values plus per-group indices in the same pass, so that a consumer of
- * 2:4 sparsity needs no dense pruned matrix and no separate conversion (the paper's remark that
- * the pattern "eliminates format conversion overhead").  The layout is this library's own:
+ * 2:4 sparsity needs no dense pruned matrix and no separate conversion step (Section 3.3 makes
+ * the same point about the 2:4 pattern and sparse hardware).  The layout is this library's own:
  *   values_out  [n_rows, d_in/2] of `dtype`, leading dimension ldv (elements, >= d_in/2): the
  *               two kept weights of group g of a row at columns 2g, 2g+1, in column order,
  *               copied bit for bit;

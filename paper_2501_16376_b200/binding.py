@@ -302,55 +302,30 @@ class Context:
                                 optr, ldo, _stream(stream)))
         return mask, W_out
 
+    # -- grouped selection (layers that read this context's input) ----------------------
+    def sp_select_unstructured_group(self, Ws, sparsity=None, *, params: EwmaParams | None = None,
+                                     masks=None, W_outs=None, inplace=False, want_mask=True,
+                                     counters=None, stream=None):
+        """Algorithm 1 on several matrices that read this context's input, in one call.
+        Returns (masks, W_outs)."""
+        arr, k, dtype, masks, W_outs = _group(self, Ws, masks, W_outs, want_mask, inplace)
+        if params is not None:
+            _check(lib.sp_select_unstructured_group_ex(self._h, arr, k, dtype, ctypes.byref(params),
+                                                       _ptr(counters), _stream(stream)))
+        else:
+            _check(lib.sp_select_unstructured_group(self._h, arr, k, dtype, float(sparsity),
+                                                    _ptr(counters), _stream(stream)))
+        return masks, W_outs
 
-def _group(ctx, Ws, masks, W_outs, want_mask, inplace):
-    """Marshals a list of weight tensors (and optional outputs) into an sp_matrix array."""
-    k = len(Ws)
-    masks = list(masks) if masks is not None else [None] * k
-    W_outs = list(W_outs) if W_outs is not None else [None] * k
-    arr = (Matrix * k)()
-    dtype = _dtype_of(Ws[0])
-    for i, W in enumerate(Ws):
-        ptr, R, n, ld = _matrix(W, "W")
-        ctx._check_width(n)
-        if _dtype_of(W) != dtype:
-            raise SpError(SP_ERR_DTYPE, "all matrices of a group must have the same dtype")
-        masks[i], W_outs[i] = ctx._outputs(W, masks[i], W_outs[i], want_mask, inplace)
-        optr, _, _, ldo = _matrix(W_outs[i], "W_out")
-        arr[i] = Matrix(ptr, R, ld, _ptr(masks[i]), optr, ldo)
-    return arr, k, dtype, masks, W_outs
+    def sp_select_nm_group(self, Ws, N: int, M: int, *, masks=None, W_outs=None, inplace=False,
+                           want_mask=True, stream=None):
+        """N:M selection of several matrices that read this context's input, in one call.
+        Returns (masks, W_outs)."""
+        arr, k, dtype, masks, W_outs = _group(self, Ws, masks, W_outs, want_mask, inplace)
+        _check(lib.sp_select_nm_group(self._h, arr, k, dtype, int(N), int(M), _stream(stream)))
+        return masks, W_outs
 
-
-def _sp_select_unstructured_group(self, Ws, sparsity=None, *, params: EwmaParams | None = None,
-                                  masks=None, W_outs=None, inplace=False, want_mask=True,
-                                  counters=None, stream=None):
-    """Algorithm 1 on several matrices that read this context's input, in one call.
-    Returns (masks, W_outs)."""
-    arr, k, dtype, masks, W_outs = _group(self, Ws, masks, W_outs, want_mask, inplace)
-    if params is not None:
-        _check(lib.sp_select_unstructured_group_ex(self._h, arr, k, dtype, ctypes.byref(params),
-                                                   _ptr(counters), _stream(stream)))
-    else:
-        _check(lib.sp_select_unstructured_group(self._h, arr, k, dtype, float(sparsity),
-                                                _ptr(counters), _stream(stream)))
-    return masks, W_outs
-
-
-def _sp_select_nm_group(self, Ws, N: int, M: int, *, masks=None, W_outs=None, inplace=False,
-                        want_mask=True, stream=None):
-    """N:M selection of several matrices that read this context's input, in one call.
-    Returns (masks, W_outs)."""
-    arr, k, dtype, masks, W_outs = _group(self, Ws, masks, W_outs, want_mask, inplace)
-    _check(lib.sp_select_nm_group(self._h, arr, k, dtype, int(N), int(M), _stream(stream)))
-    return masks, W_outs
-
-
-Context.sp_select_unstructured_group = _sp_select_unstructured_group
-Context.sp_select_nm_group = _sp_select_nm_group
-
-
-class HostMixin:
-    """Host-buffer variants: tensors are CPU tensors (pinned for overlap); see the C header."""
+    # -- host-buffer variants: tensors are CPU tensors (pinned for overlap); see the C header
 
     def sp_calib_accumulate_host(self, X: torch.Tensor, stream=None):
         ptr, T, n, ld = _matrix(X, "X", host=True)
@@ -375,8 +350,22 @@ class HostMixin:
                                                _ptr(mask), optr, ldo, _stream(stream)))
 
 
-for _name in ("sp_calib_accumulate_host", "sp_select_nm_host", "sp_select_unstructured_host"):
-    setattr(Context, _name, getattr(HostMixin, _name))
+def _group(ctx, Ws, masks, W_outs, want_mask, inplace):
+    """Marshals a list of weight tensors (and optional outputs) into an sp_matrix array."""
+    k = len(Ws)
+    masks = list(masks) if masks is not None else [None] * k
+    W_outs = list(W_outs) if W_outs is not None else [None] * k
+    arr = (Matrix * k)()
+    dtype = _dtype_of(Ws[0])
+    for i, W in enumerate(Ws):
+        ptr, R, n, ld = _matrix(W, "W")
+        ctx._check_width(n)
+        if _dtype_of(W) != dtype:
+            raise SpError(SP_ERR_DTYPE, "all matrices of a group must have the same dtype")
+        masks[i], W_outs[i] = ctx._outputs(W, masks[i], W_outs[i], want_mask, inplace)
+        optr, _, _, ldo = _matrix(W_outs[i], "W_out")
+        arr[i] = Matrix(ptr, R, ld, _ptr(masks[i]), optr, ldo)
+    return arr, k, dtype, masks, W_outs
 
 
 def sp_apply_mask(W: torch.Tensor, mask: torch.Tensor, W_out: torch.Tensor | None = None,

@@ -1,6 +1,6 @@
 // 2:4 selection (Section 3.3) emitted directly in a compressed form: the two kept weights of
-// every group of four, packed, plus a 4-bit index record per group.  The paper points out that
-// a 2:4 result can be consumed by sparse tensor-core hardware "without format conversion"; this
+// every group of four, packed, plus a 4-bit index record per group.  Section 3.3 notes that
+// sparse tensor-core hardware consumes a 2:4 result as it is, with no conversion step; this
 // kernel writes values and indices in the same pass that selects them, so no dense pruned
 // matrix has to be written and re-read.  The layout is this library's own, documented in the
 // header: values [rows, d_in/2] (kept weights in column order), metadata [rows, ceil(d_in/32)]

@@ -40,7 +40,7 @@ def token_share(n_tokens: int, world: int, rank: int, align: int = 1) -> range:
 
 def row_share(n_rows: int, world: int, rank: int) -> range:
     """Row-sharded selection: the contiguous rows of a layer that `rank` prunes (rows are
-    independent problems, Algorithm 1 "parallel calculation for each row")."""
+    independent problems: the row loop of Algorithm 1 is parallel)."""
     return assign_units(n_rows, world, rank)
 
 

@@ -361,6 +361,19 @@ sp_status sp_select_unstructured_host(sp_ctx *ctx, const void *W_host, sp_dtype 
 
 /* ------------------------------------------------------------------ diagnostics */
 
+/*
+ * Index checks of the debug build (python -m paper_2501_16376_b200.build --debug ->
+ * libswiftprune_debug.so, same ABI).  In that build the kernels check the indices of their
+ * stores; an out-of-range access is skipped and recorded instead of faulting (nothing traps).
+ * *violations receives the number of skipped accesses on the current device since the last
+ * clear (-1 in the release build, which compiles no checks); first_code / first_index /
+ * first_limit (nullable) describe the first one (codes in csrc/sp_debug.cuh); clear != 0 resets
+ * the records.  Synchronises the device.
+ */
+sp_status sp_debug_status(int *violations /* host */, int *first_code /* host */,
+                          int64_t *first_index /* host */, int64_t *first_limit /* host */,
+                          int clear);
+
 const char *sp_status_string(sp_status status);
 /* Text of the last CUDA error this thread saw inside the library ("" if none). */
 const char *sp_last_cuda_error(void);

@@ -31,7 +31,7 @@ EXPORTS = (
     "sp_set_stats", "sp_calib_stats_noalloc", "sp_score", "sp_la_for_sparsity", "sp_select_unstructured",
     "sp_select_unstructured_ex", "sp_search_la", "sp_ewma_trace", "sp_select_nm", "sp_select_24_compressed", "sp_apply_mask", "sp_calib_accumulate_host",
     "sp_select_nm_host", "sp_select_unstructured_host", "sp_select_unstructured_group",
-    "sp_select_unstructured_group_ex", "sp_select_nm_group", "sp_status_string",
+    "sp_select_unstructured_group_ex", "sp_select_nm_group", "sp_debug_status", "sp_status_string",
     "sp_last_cuda_error", "sp_launch_count",
 )
 
@@ -89,6 +89,8 @@ def _load() -> ctypes.CDLL:
     lib.sp_select_unstructured_group_ex.argtypes = [vp, ctypes.POINTER(Matrix), ci, ci,
                                                     ctypes.POINTER(EwmaParams), vp, vp]
     lib.sp_select_nm_group.argtypes = [vp, ctypes.POINTER(Matrix), ci, ci, ci, ci, vp]
+    lib.sp_debug_status.argtypes = [ctypes.POINTER(ci), ctypes.POINTER(ci), ctypes.POINTER(i64),
+                                    ctypes.POINTER(i64), ci]
     lib.sp_status_string.argtypes = [ci]
     lib.sp_status_string.restype = ctypes.c_char_p
     lib.sp_last_cuda_error.restype = ctypes.c_char_p
@@ -141,6 +143,16 @@ def _ptr(t):
 
 def sp_launch_count() -> int:
     return int(lib.sp_launch_count())
+
+
+def sp_debug_status(clear: bool = False):
+    """(violations, first_code, first_index, first_limit) of the debug build's index checks;
+    violations is -1 for the release build."""
+    v, c = ctypes.c_int(), ctypes.c_int()
+    i, lim = ctypes.c_int64(), ctypes.c_int64()
+    _check(lib.sp_debug_status(ctypes.byref(v), ctypes.byref(c), ctypes.byref(i), ctypes.byref(lim),
+                               1 if clear else 0))
+    return v.value, c.value, i.value, lim.value
 
 
 def sp_la_for_sparsity(sparsity: float) -> float:

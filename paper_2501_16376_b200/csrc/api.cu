@@ -14,6 +14,14 @@
 namespace sp {
 
 static thread_local char g_cuda_error[256] = "";
+// readers of the per-translation-unit index-check records (debug build only; see sp_debug.cuh)
+static DebugReader g_debug_readers[16];
+static int g_debug_reader_count = 0;
+
+void register_debug_reader(DebugReader reader) {
+    if (g_debug_reader_count < 16) g_debug_readers[g_debug_reader_count++] = reader;
+}
+
 static std::atomic<uint64_t> g_launches{0};
 
 sp_status cuda_fail(cudaError_t e) {
@@ -574,6 +582,32 @@ sp_status sp_select_unstructured_host(sp_ctx *ctx, const void *W_host, sp_dtype 
     st = ensure_finalized(ctx, s);
     if (st != SP_OK) return st;
     return host_select(ctx, 1, W_host, dtype, n_rows, ldw, 0, 0, &p, mask_host, W_out_host, ldo, s);
+}
+
+sp_status sp_debug_status(int *violations, int *first_code, int64_t *first_index,
+                          int64_t *first_limit, int clear) {
+    if (violations == nullptr) return SP_ERR_INVALID_ARG;
+    *violations = -1;
+    if (first_code != nullptr) *first_code = 0;
+    if (first_index != nullptr) *first_index = 0;
+    if (first_limit != nullptr) *first_limit = 0;
+    if (g_debug_reader_count == 0) return SP_OK;  // release build: no checks compiled in
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return cuda_fail(e);
+    unsigned int total = 0;
+    for (int i = 0; i < g_debug_reader_count; ++i) {
+        DebugRecord r = {};
+        e = g_debug_readers[i](&r, clear != 0);
+        if (e != cudaSuccess) return cuda_fail(e);
+        if (r.count != 0u && total == 0u) {
+            if (first_code != nullptr) *first_code = r.code;
+            if (first_index != nullptr) *first_index = r.index;
+            if (first_limit != nullptr) *first_limit = r.limit;
+        }
+        total += r.count;
+    }
+    *violations = static_cast<int>(total);
+    return SP_OK;
 }
 
 const char *sp_status_string(sp_status status) {

@@ -85,10 +85,12 @@ calib_accumulate_kernel(const uint16_t *__restrict__ X, int64_t ldx, int64_t n_t
 #pragma unroll
         for (int w = 0; w < kCalibWarps; ++w) sum += sm[w][t];
         double *dst = partial + static_cast<int64_t>(slab) * n_pad + ch;
-        if (slab >= first_fresh_slab)
-            *dst = sum;
-        else
-            *dst += sum;
+        if (SP_IN_RANGE(static_cast<int64_t>(slab) * n_pad + ch, kMaxSlabs * n_pad, kDbgCalibPartial)) {
+            if (slab >= first_fresh_slab)
+                *dst = sum;
+            else
+                *dst += sum;
+        }
     }
 }
 
@@ -210,7 +212,8 @@ finalize_kernel(const double *__restrict__ partial, int slabs_valid, int64_t n, 
                     const int64_t e = q & 7;
                     const int64_t pos = e < 4 ? 2 * e : 2 * (e - 4) + 1;
                     const int64_t r = q & 511, ln = r >> 4, ch = (r >> 3) & 1;
-                    factor_pairs[(q & ~int64_t(511)) + (2 * ch + (pos >> 2)) * 128 + ln * 4 + (pos & 3)] = c;
+                    const int64_t at = (q & ~int64_t(511)) + (2 * ch + (pos >> 2)) * 128 + ln * 4 + (pos & 3);
+                    if (SP_IN_RANGE(at, (n_pad + 511) / 512 * 512 + 512, kDbgFactorPairs)) factor_pairs[at] = c;
                 }
             }
         }

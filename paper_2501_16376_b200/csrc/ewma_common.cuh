@@ -182,7 +182,7 @@ __device__ __forceinline__ unsigned long long literal_walk(
         }
         word |= keep8 << (i0 & 31);
         if ((i0 & 31) == 24 || i0 + 8 >= n) {
-            if (mrow != nullptr) mrow[i0 >> 5] = word;
+            if (mrow != nullptr && SP_IN_RANGE(i0 >> 5, (n + 31) / 32, kDbgWalkMask)) mrow[i0 >> 5] = word;
             word = 0;
         }
     }

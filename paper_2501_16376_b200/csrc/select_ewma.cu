@@ -512,7 +512,8 @@ ewma_pair_scan_kernel(const __grid_constant__ EwmaJobTable jobs, int n,
                 uint32_t keep8 = ~halfmasks_to_bits(pm) & 0xffu;
                 if (!in_row[x]) keep8 = 0u;
                 keep16 |= keep8 << (8 * x);
-                if (olane != nullptr && in_row[x]) {
+                if (olane != nullptr && in_row[x] &&
+                    SP_IN_RANGE(col + 8 * x + 7, jobs.job[jk].ldo, kDbgEwmaColumn)) {
 #pragma unroll
                     for (int k = 0; k < 4; ++k) p[x][k] &= ~pm[k];
                     __stcs(reinterpret_cast<uint4 *>(olane + tile * kTile + 8 * x),
@@ -521,7 +522,8 @@ ewma_pair_scan_kernel(const __grid_constant__ EwmaJobTable jobs, int n,
             }
             if constexpr (COUNT) kept += __popc(keep16);
             // two mask bytes per lane: a little-endian half word holds columns 16k .. 16k+15
-            if (mlane != nullptr && (FULL || tile * 32 + lane < mask_halves))
+            if (mlane != nullptr && (FULL || tile * 32 + lane < mask_halves) &&
+                SP_IN_RANGE(tile * 32 + lane, mask_halves, kDbgEwmaMask))
                 mlane[tile * 32] = static_cast<uint16_t>(keep16);
             __syncwarp();  // all lanes have read this slot before it is refilled
         }

@@ -241,7 +241,8 @@ select_nm_stream_kernel(const __grid_constant__ NmJobTable jobs, int n, int rows
         } else {
             masks_from_nibbles(nm_rank_nibbles8(key, bias), m);
         }
-        if (OUT && in_row) {
+        if (OUT && in_row && SP_IN_RANGE(row_begin + rr, n_rows, kDbgNmRow) &&
+            SP_IN_RANGE(col + 7, ldo, kDbgNmColumn)) {
             __stcs(reinterpret_cast<uint4 *>(dst + static_cast<int64_t>(rr) * ldo),
                    make_uint4(p[0] & m[0], p[1] & m[1], p[2] & m[2], p[3] & m[3]));
         }

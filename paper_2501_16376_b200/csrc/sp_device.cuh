@@ -8,6 +8,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "sp_debug.cuh"
+
 namespace sp {
 
 constexpr unsigned kFullWarp = 0xffffffffu;

@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "sp_debug.cuh"
 #include "swiftprune.h"
 
 namespace sp {

@@ -35,6 +35,13 @@ def test_library_exports_every_declared_symbol(lib_path):
         assert hasattr(lib, name), name
 
 
+def test_debug_build_exports_the_same_symbols():
+    from paper_2501_16376_b200 import build
+    lib = ctypes.CDLL(build.build(debug=True))
+    for name in _declared_symbols():
+        assert hasattr(lib, name), name
+
+
 def test_binding_lists_the_same_symbols(lib_path):
     from paper_2501_16376_b200 import binding
     assert sorted(binding.EXPORTS) == _declared_symbols()

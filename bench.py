@@ -46,8 +46,7 @@ NCU_CALIB_TRAFFIC = {4096: 272.0e6, 11008: 725.1e6}
 NCU_SELECT_TRAFFIC = {
     "select_nm_stream_kernel": {(12288, 4096): 156.0e6, (4096, 4096): 34.3e6,
                                 (22016, 4096): 318.4e6, (4096, 11008): 131.4e6},
-    "ewma_pair_scan_kernel": {(6144, 4096): 55.3e6, (4096, 4096): 34.4e6,
-                              (28672, 4096): 430.4e6, (4096, 14336): 190.0e6},
+    "ewma_pair_scan_kernel": {},
 }
 
 
@@ -58,6 +57,10 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama2-7b")
+    ap.add_argument("--select-launch", default="auto", choices=["auto", "block", "input", "layer"],
+                    help="selection calls of the pass: one per block (unstructured only), one per "
+                         "layer input (grouped), or one per layer; auto = block for unstructured "
+                         "workloads, input for N:M")
     ap.add_argument("--batch-seqs", type=int, default=16,
                     help="calibration sequences per sp_calib_accumulate call")
     ap.add_argument("--e2e-steps", type=int, default=1)
@@ -329,20 +332,30 @@ def ewma_block(device, peak, peak_kind, blocks=4):
                                                W_out=mb.outputs[b][li])
                 singles.append(entry(w.layers[li].name, w.layers[li].d_out, d_in,
                                      timed(run_one), 1))
+    # all seven layers of a block in ONE launch (sp_select_unstructured_multi): what the pass uses
+    block_ms = timed(lambda b: pipeline.select_block(mb, b, sparsity))
     mb.close()
     del mb
     torch.cuda.empty_cache()
-    gbs = total_bytes / (total_ms * 1e-3) / 1e9
+    gbs = total_bytes / (block_ms * 1e-3) / 1e9
+    grouped_gbs = total_bytes / (total_ms * 1e-3) / 1e9
     return {
         "kernel": "ewma_pair_scan_kernel", "workload": "llama3-8b layer shapes, bf16, "
         "unstructured %.0f %%, default mode (drift gate on)" % (sparsity * 100),
         "bound": "hbm", "unit": "GB/s", "peak": peak, "peak_kind": peak_kind,
         "achieved": gbs, "frac": gbs / peak, "frac_of_8TBs": gbs / 8000.0,
-        "ms_per_block": total_ms, "blocks_timed": blocks,
-        "per_launch": groups, "single_layer_calls": singles,
-        "note": "selection launches only: %d launches on distinct buffers replayed as one CUDA "
-                "graph, CUDA events around the replay, best of 3; achieved = 4.125 B per weight "
-                "/ time; the whole-block figure uses the grouped launches" % blocks,
+        "ms_per_block": block_ms, "blocks_timed": blocks, "kernel_launches_per_block": 1,
+        "traffic": NCU_EWMA_TRAFFIC.get(("block", "llama3-8b")),
+        "one_launch_per_layer_input": {"ms_per_block": total_ms, "achieved": grouped_gbs,
+                                       "frac": grouped_gbs / peak,
+                                       "frac_of_8TBs": grouped_gbs / 8000.0,
+                                       "per_launch": groups},
+        "single_layer_calls": singles,
+        "note": "selection launches only: the calls of %d blocks on distinct buffers replayed as "
+                "one CUDA graph, CUDA events around the replay, best of 3; achieved = 4.125 B per "
+                "weight / time; the headline figure is one launch per block (all seven layers, "
+                "each with its own input's statistics), the breakdown below it one launch per "
+                "layer input and one per layer" % blocks,
     }
 
 def gpu_arm(args):
@@ -377,10 +390,17 @@ def gpu_arm(args):
         w, device, model_seed_offset=0 if shared else sharding.unit_of_rank(rank, world))
     torch.cuda.synchronize()
 
+    select_launch = args.select_launch
+    if select_launch == "auto":
+        select_launch = "block" if w.mode != "nm" and not shared else "input"
+    if select_launch == "block" and (w.mode == "nm" or shared):
+        raise SystemExit("--select-launch block: unstructured single-model passes only")
+    how = {"grouped": select_launch != "layer", "per_block": select_launch == "block"}
+
     def one_pass():
         if shared:
             return pipeline.prune_model_split(mb, arg, batch_tokens, rank, world, args.split)
-        return pipeline.prune_model(mb, arg, batch_tokens)
+        return pipeline.prune_model(mb, arg, batch_tokens, **how)
 
     def barrier():
         torch.cuda.synchronize()
@@ -405,7 +425,7 @@ def gpu_arm(args):
     if args.graph and shared:
         raise SystemExit("--graph replays the single-model pass; it cannot be combined with --split")
     if args.graph:
-        graph, counts = pipeline.capture_model_graph(mb, arg, batch_tokens)
+        graph, counts = pipeline.capture_model_graph(mb, arg, batch_tokens, **how)
         for _ in range(3):
             graph.replay()
     launches_before = sp.sp_launch_count()
@@ -432,7 +452,7 @@ def gpu_arm(args):
     # timed region: the event records between phases would otherwise sit inside it (they keep a
     # kernel from overlapping the tail of its predecessor).
     for _ in range(args.steps):
-        pipeline.prune_model(mb, arg, batch_tokens, phase_events)
+        pipeline.prune_model(mb, arg, batch_tokens, phase_events, **how)
     torch.cuda.synchronize()
 
     elapsed_ms = sharding.max_over_ranks(elapsed_ms, world, device)
@@ -456,12 +476,15 @@ def gpu_arm(args):
         calib_traffic = sum(NCU_CALIB_TRAFFIC[d] for d in widths) / len(widths)
     sel_kernel = "select_nm_stream_kernel" if w.mode == "nm" else "ewma_pair_scan_kernel"
     sel_traffic = None
-    shapes = []                      # one grouped launch per layer input: (total rows, d_in)
-    for name, d_in in w.input_widths().items():
-        shapes.append((sum(l.d_out for l in w.layers if l.input == name), d_in))
     table = NCU_SELECT_TRAFFIC[sel_kernel]
-    if all(sh in table for sh in shapes) and (w.mode != "nm" or arg == (2, 4)):
-        sel_traffic = sum(table[sh] for sh in shapes) / len(shapes)
+    if select_launch == "block":     # one launch per block
+        sel_traffic = table.get(("block", w.name))
+    elif select_launch == "input":   # one grouped launch per layer input: (total rows, d_in)
+        shapes = []
+        for name, d_in in w.input_widths().items():
+            shapes.append((sum(l.d_out for l in w.layers if l.input == name), d_in))
+        if all(sh in table for sh in shapes) and (w.mode != "nm" or arg == (2, 4)):
+            sel_traffic = sum(table[sh] for sh in shapes) / len(shapes)
     roofline = {
         "kernel": "calib_accumulate_kernel", "bound": "hbm", "achieved": calib_gbs, "peak": peak,
         "peak_kind": peak_kind, "unit": "GB/s", "frac": calib_gbs / peak,
@@ -480,9 +503,11 @@ def gpu_arm(args):
         "traffic": sel_traffic, "avg_launch_ms": select_ms / select_launches,
         "bytes_per_launch": SELECT_BYTES_PER_WEIGHT * sel_weights / select_launches,
         "weights_per_sec": sel_weights / (select_ms * 1e-3),
-        "note": "from instrumented passes run after the timed region; events bracket the grouped "
-                "selection launch of one layer input; ncu traffic counts DRAM bytes while the "
-                "kernel runs (part of the output is still in L2 when it ends)",
+        "select_launch": select_launch,
+        "note": "from instrumented passes run after the timed region; events bracket the "
+                "selection launch(es) of one %s; ncu traffic counts DRAM bytes while the "
+                "kernel runs (part of the output is still in L2 when it ends)" % (
+                    "block" if select_launch == "block" else "layer input"),
     }
 
     # The same select kernel timed alone on the largest layer shape: back-to-back launches over

@@ -310,6 +310,28 @@ sp_status sp_select_nm_group(sp_ctx *ctx, const sp_matrix *mats /* host */, int 
                              sp_dtype dtype, int N, int M, sp_stream stream);
 
 /*
+ * Algorithm 1 on matrices that read DIFFERENT layer inputs (all layers of a transformer block,
+ * say), in one launch where their layouts allow: item i is mats[i] pruned with the statistics of
+ * ctxs[i] (HOST arrays of n_items entries, 1 <= n_items <= SP_MAX_MULTI; a context may appear
+ * more than once; all contexts on one device, each with calibration data, else
+ * SP_ERR_INVALID_ARG / SP_ERR_STATE; mats[i] must be at least ctxs[i]'s d_in wide).  The rows
+ * of Algorithm 1 are independent problems whatever matrix they belong to, so the result for
+ * each matrix is identical to that of its own sp_select_unstructured[_ex] call on its context;
+ * what changes is the cost: one launch, whose tail the short rows fill, instead of one launch
+ * and one ramp-up per layer input.  Every context with batches pending is finalised on `stream`
+ * first.  counters (nullable, device) are totals over all items.
+ */
+enum { SP_MAX_MULTI = 16 };
+sp_status sp_select_unstructured_multi(sp_ctx *const *ctxs /* host */,
+                                       const sp_matrix *mats /* host */, int n_items,
+                                       sp_dtype dtype, float sparsity,
+                                       unsigned long long *counters, sp_stream stream);
+sp_status sp_select_unstructured_multi_ex(sp_ctx *const *ctxs /* host */,
+                                          const sp_matrix *mats /* host */, int n_items,
+                                          sp_dtype dtype, const sp_ewma_params *params /* host */,
+                                          unsigned long long *counters, sp_stream stream);
+
+/*
  * Section 3.3, compressed output: 2:4 selection (exactly as sp_select_nm with N = 2, M = 4)
  * written as the kept values plus per-group indices in the same pass, so that a consumer of
  * 2:4 sparsity needs no dense pruned matrix and no separate conversion step (Section 3.3 makes

@@ -31,7 +31,8 @@ EXPORTS = (
     "sp_set_stats", "sp_calib_stats_noalloc", "sp_score", "sp_la_for_sparsity", "sp_select_unstructured",
     "sp_select_unstructured_ex", "sp_search_la", "sp_ewma_trace", "sp_select_nm", "sp_select_24_compressed", "sp_apply_mask", "sp_calib_accumulate_host",
     "sp_select_nm_host", "sp_select_unstructured_host", "sp_select_unstructured_group",
-    "sp_select_unstructured_group_ex", "sp_select_nm_group", "sp_debug_status", "sp_status_string",
+    "sp_select_unstructured_group_ex", "sp_select_nm_group", "sp_select_unstructured_multi",
+    "sp_select_unstructured_multi_ex", "sp_debug_status", "sp_status_string",
     "sp_last_cuda_error", "sp_launch_count",
 )
 
@@ -54,6 +55,7 @@ class Matrix(ctypes.Structure):
 
 
 SP_MAX_GROUP = 8
+SP_MAX_MULTI = 16
 
 
 def _load() -> ctypes.CDLL:
@@ -89,6 +91,10 @@ def _load() -> ctypes.CDLL:
     lib.sp_select_unstructured_group_ex.argtypes = [vp, ctypes.POINTER(Matrix), ci, ci,
                                                     ctypes.POINTER(EwmaParams), vp, vp]
     lib.sp_select_nm_group.argtypes = [vp, ctypes.POINTER(Matrix), ci, ci, ci, ci, vp]
+    lib.sp_select_unstructured_multi.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(Matrix), ci,
+                                                 ci, f32, vp, vp]
+    lib.sp_select_unstructured_multi_ex.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(Matrix), ci,
+                                                    ci, ctypes.POINTER(EwmaParams), vp, vp]
     lib.sp_debug_status.argtypes = [ctypes.POINTER(ci), ctypes.POINTER(ci), ctypes.POINTER(i64),
                                     ctypes.POINTER(i64), ci]
     lib.sp_status_string.argtypes = [ci]
@@ -378,6 +384,37 @@ def _group(ctx, Ws, masks, W_outs, want_mask, inplace):
         optr, _, _, ldo = _matrix(W_outs[i], "W_out")
         arr[i] = Matrix(ptr, R, ld, _ptr(masks[i]), optr, ldo)
     return arr, k, dtype, masks, W_outs
+
+
+def sp_select_unstructured_multi(ctxs, Ws, sparsity=None, *, params: EwmaParams | None = None,
+                                 masks=None, W_outs=None, inplace=False, want_mask=True,
+                                 counters=None, stream=None):
+    """Algorithm 1 on matrices that read different layer inputs, in one call: Ws[i] is pruned
+    with the statistics of ctxs[i] (contexts may repeat).  Returns (masks, W_outs)."""
+    k = len(Ws)
+    if k != len(ctxs) or k < 1:
+        raise SpError(SP_ERR_INVALID_ARG, "one context per matrix")
+    masks = list(masks) if masks is not None else [None] * k
+    W_outs = list(W_outs) if W_outs is not None else [None] * k
+    arr = (Matrix * k)()
+    handles = (ctypes.c_void_p * k)()
+    dtype = _dtype_of(Ws[0])
+    for i, (ctx, W) in enumerate(zip(ctxs, Ws)):
+        ptr, R, n, ld = _matrix(W, "W")
+        ctx._check_width(n)
+        if _dtype_of(W) != dtype:
+            raise SpError(SP_ERR_DTYPE, "all matrices of a call must have the same dtype")
+        masks[i], W_outs[i] = ctx._outputs(W, masks[i], W_outs[i], want_mask, inplace)
+        optr, _, _, ldo = _matrix(W_outs[i], "W_out")
+        arr[i] = Matrix(ptr, R, ld, _ptr(masks[i]), optr, ldo)
+        handles[i] = ctx._h
+    if params is not None:
+        _check(lib.sp_select_unstructured_multi_ex(handles, arr, k, dtype, ctypes.byref(params),
+                                                   _ptr(counters), _stream(stream)))
+    else:
+        _check(lib.sp_select_unstructured_multi(handles, arr, k, dtype, float(sparsity),
+                                                _ptr(counters), _stream(stream)))
+    return masks, W_outs
 
 
 def sp_apply_mask(W: torch.Tensor, mask: torch.Tensor, W_out: torch.Tensor | None = None,

@@ -1,5 +1,6 @@
 // C ABI of the library: argument validation on the host, context management, dispatch to
 // the kernel launchers.  Nothing here synchronises unless the header says so.
+#include <algorithm>
 #include <atomic>
 #include <cmath>
 #include <cstdio>
@@ -65,6 +66,16 @@ class CallRange {
 #define SP_CALL_RANGE() CallRange sp_call_range__(__func__)
 
 static bool valid_dtype(sp_dtype d) { return d == SP_F16 || d == SP_BF16; }
+
+static bool ewma_params_valid(const sp_ewma_params *params) {
+    if (params == nullptr) return false;
+    if (!(params->alpha > 0.0f) || !(params->alpha <= 1.0f) || !(params->beta > 0.0f) ||
+        !(params->beta <= 1.0f) || !std::isfinite(params->la))
+        return false;
+    return params->s_update == SP_S_GATED || params->s_update == SP_S_FROZEN ||
+           params->s_update == SP_S_LITERAL_W2 || params->s_update == SP_S_READING_X2 ||
+           params->s_update == SP_S_LITERAL_SCAN;
+}
 
 static sp_status ensure_finalized(sp_ctx *ctx, cudaStream_t stream) {
     if (ctx->n_tokens <= 0) return SP_ERR_STATE;
@@ -302,14 +313,7 @@ sp_status sp_select_unstructured_ex(sp_ctx *ctx, const void *W, sp_dtype dtype, 
     SP_CALL_RANGE();
     sp_status st = check_matrix_args(ctx, W, dtype, n_rows, ldw, W_out, ldo);
     if (st != SP_OK) return st;
-    if (params == nullptr) return SP_ERR_INVALID_ARG;
-    if (!(params->alpha > 0.0f) || !(params->alpha <= 1.0f) || !(params->beta > 0.0f) ||
-        !(params->beta <= 1.0f) || !std::isfinite(params->la))
-        return SP_ERR_INVALID_ARG;
-    if (params->s_update != SP_S_GATED && params->s_update != SP_S_FROZEN &&
-        params->s_update != SP_S_LITERAL_W2 && params->s_update != SP_S_READING_X2 &&
-        params->s_update != SP_S_LITERAL_SCAN)
-        return SP_ERR_INVALID_ARG;
+    if (!ewma_params_valid(params)) return SP_ERR_INVALID_ARG;
     if (ctx->n_tokens <= 0) return SP_ERR_STATE;
     DeviceGuard guard(ctx->device);
     if (guard.error() != cudaSuccess) return cuda_fail(guard.error());
@@ -354,14 +358,7 @@ sp_status sp_select_unstructured_group_ex(sp_ctx *ctx, const sp_matrix *mats, in
     EwmaLaunchJob jobs[SP_MAX_GROUP];
     sp_status st = group_jobs(ctx, mats, n_mats, dtype, jobs);
     if (st != SP_OK) return st;
-    if (params == nullptr) return SP_ERR_INVALID_ARG;
-    if (!(params->alpha > 0.0f) || !(params->alpha <= 1.0f) || !(params->beta > 0.0f) ||
-        !(params->beta <= 1.0f) || !std::isfinite(params->la))
-        return SP_ERR_INVALID_ARG;
-    if (params->s_update != SP_S_GATED && params->s_update != SP_S_FROZEN &&
-        params->s_update != SP_S_LITERAL_W2 && params->s_update != SP_S_READING_X2 &&
-        params->s_update != SP_S_LITERAL_SCAN)
-        return SP_ERR_INVALID_ARG;
+    if (!ewma_params_valid(params)) return SP_ERR_INVALID_ARG;
     if (ctx->n_tokens <= 0) return SP_ERR_STATE;
     DeviceGuard guard(ctx->device);
     if (guard.error() != cudaSuccess) return cuda_fail(guard.error());
@@ -382,6 +379,51 @@ sp_status sp_select_unstructured_group(sp_ctx *ctx, const sp_matrix *mats, int n
     sp_status st = sp_la_for_sparsity(sparsity, &p.la);
     if (st != SP_OK) return st;
     return sp_select_unstructured_group_ex(ctx, mats, n_mats, dtype, &p, counters, stream);
+}
+
+sp_status sp_select_unstructured_multi_ex(sp_ctx *const *ctxs, const sp_matrix *mats, int n_items,
+                                          sp_dtype dtype, const sp_ewma_params *params,
+                                          unsigned long long *counters, sp_stream stream) {
+    SP_CALL_RANGE();
+    if (ctxs == nullptr || mats == nullptr) return SP_ERR_INVALID_ARG;
+    if (n_items < 1 || n_items > SP_MAX_MULTI) return SP_ERR_INVALID_ARG;
+    if (!ewma_params_valid(params)) return SP_ERR_INVALID_ARG;
+    EwmaLaunchJob jobs[SP_MAX_MULTI];
+    for (int i = 0; i < n_items; ++i) {
+        const sp_matrix &m = mats[i];
+        if (ctxs[i] == nullptr) return SP_ERR_INVALID_ARG;
+        sp_status st = check_matrix_args(ctxs[i], m.W, dtype, m.n_rows, m.ldw, m.W_out, m.ldo);
+        if (st != SP_OK) return st;
+        if (ctxs[i]->device != ctxs[0]->device) return SP_ERR_INVALID_ARG;
+        if (ctxs[i]->n_tokens <= 0) return SP_ERR_STATE;
+        jobs[i] = EwmaLaunchJob{m.W, m.W_out, m.mask_out, m.n_rows, m.ldw, m.ldo, ctxs[i]};
+    }
+    // Longest rows first: the CTAs of a launch start in this order, and the launch ends soonest
+    // when the rows that take longest are not the ones left for its tail.
+    std::stable_sort(jobs, jobs + n_items, [](const EwmaLaunchJob &x, const EwmaLaunchJob &y) {
+        return x.ctx->d_in > y.ctx->d_in;
+    });
+    DeviceGuard guard(ctxs[0]->device);
+    if (guard.error() != cudaSuccess) return cuda_fail(guard.error());
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    for (int i = 0; i < n_items; ++i) {
+        sp_status st = ensure_finalized(ctxs[i], s);  // no work for a context seen before
+        if (st != SP_OK) return st;
+    }
+    return launch_select_ewma(ctxs[0], jobs, n_items, dtype, *params, counters, s);
+}
+
+sp_status sp_select_unstructured_multi(sp_ctx *const *ctxs, const sp_matrix *mats, int n_items,
+                                       sp_dtype dtype, float sparsity,
+                                       unsigned long long *counters, sp_stream stream) {
+    SP_CALL_RANGE();
+    sp_ewma_params p;
+    p.alpha = 0.125f;  // Section 4.2
+    p.beta = 0.125f;
+    p.s_update = SP_S_GATED;
+    sp_status st = sp_la_for_sparsity(sparsity, &p.la);
+    if (st != SP_OK) return st;
+    return sp_select_unstructured_multi_ex(ctxs, mats, n_items, dtype, &p, counters, stream);
 }
 
 sp_status sp_select_nm_group(sp_ctx *ctx, const sp_matrix *mats, int n_mats, sp_dtype dtype, int N,

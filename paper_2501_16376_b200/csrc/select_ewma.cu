@@ -67,17 +67,24 @@ __device__ __forceinline__ float lane_affine_scan(float x, const float (&step)[5
     return x;
 }
 
-// The matrices of one launch.  Rows are numbered through all jobs.
+// The matrices of one launch, each with the statistics it is pruned with (matrices that read
+// different layer inputs can share a launch).  A job owns a whole number of CTAs, so the job of a
+// CTA - and with it the row length and every pointer - is the same for all its warps.
 struct EwmaJob {
     const uint16_t *W;
     uint16_t *W_out;  // nullable
     uint32_t *mask;   // nullable
+    const float *factor_pairs;
+    const DeviceScalars *scalars;
+    const double *colsq;
+    const float *factor;
     int ldw, ldo, n_rows;
-    int first_row;
+    int n, mask_words;
+    int first_cta;
 };
 struct EwmaJobTable {
     int count;
-    int total_rows;
+    int total_ctas;
     EwmaJob job[kEwmaMaxJobs];
 };
 
@@ -290,28 +297,28 @@ struct TileConstants {
 
 template <bool BF16, bool FULL, bool COUNT, bool GATE>
 __global__ void __launch_bounds__(kPairThreads, SP_EWMA_PAIR_MIN_BLOCKS)
-ewma_pair_scan_kernel(const __grid_constant__ EwmaJobTable jobs, int n,
-                      const float *__restrict__ factor_pairs,
-                      const DeviceScalars *__restrict__ scalars,
+ewma_pair_scan_kernel(const __grid_constant__ EwmaJobTable jobs,
                       const __grid_constant__ ScanConstants sc,
                       const __grid_constant__ PairConstants pc,
-                      const __grid_constant__ TileConstants wc, int mask_words,
-                      unsigned long long *__restrict__ counters,
-                      const double *__restrict__ colsq, const float *__restrict__ factor) {
+                      const __grid_constant__ TileConstants wc,
+                      unsigned long long *__restrict__ counters) {
     constexpr int kTile = 512;
     pdl_launch_dependents();
     pdl_wait();  // the per-channel factors come from an earlier kernel of the stream
     const int lane = threadIdx.x & 31;
-    const int grow = blockIdx.x * kPairWarps + (threadIdx.x >> 5);  // row among all jobs
-    if (grow >= jobs.total_rows) return;  // warp-uniform
-    int jk = 0;
-    while (jk + 1 < jobs.count && grow >= jobs.job[jk + 1].first_row) ++jk;
-    const int row = grow - jobs.job[jk].first_row;
-    const int ldw = jobs.job[jk].ldw;
-    const uint16_t *wrow = jobs.job[jk].W + static_cast<int64_t>(row) * ldw;
-    uint16_t *const W_out = jobs.job[jk].W_out;
-    uint32_t *const mask = jobs.job[jk].mask;
-    uint16_t *olane = W_out != nullptr ? W_out + static_cast<int64_t>(row) * jobs.job[jk].ldo + lane * 16 : nullptr;
+    int jk = 0;  // the job of this CTA
+    while (jk + 1 < jobs.count && static_cast<int>(blockIdx.x) >= jobs.job[jk + 1].first_cta) ++jk;
+    const EwmaJob &job = jobs.job[jk];
+    const int row = (static_cast<int>(blockIdx.x) - job.first_cta) * kPairWarps + (threadIdx.x >> 5);
+    if (row >= job.n_rows) return;  // warp-uniform
+    const int n = job.n;
+    const int mask_words = job.mask_words;
+    const float *__restrict__ factor_pairs = job.factor_pairs;
+    const DeviceScalars *__restrict__ scalars = job.scalars;
+    const uint16_t *wrow = job.W + static_cast<int64_t>(row) * job.ldw;
+    uint16_t *const W_out = job.W_out;
+    uint32_t *const mask = job.mask;
+    uint16_t *olane = W_out != nullptr ? W_out + static_cast<int64_t>(row) * job.ldo + lane * 16 : nullptr;
     uint16_t *mlane = mask != nullptr
                           ? reinterpret_cast<uint16_t *>(mask + static_cast<int64_t>(row) * mask_words) + lane
                           : nullptr;
@@ -513,7 +520,7 @@ ewma_pair_scan_kernel(const __grid_constant__ EwmaJobTable jobs, int n,
                 if (!in_row[x]) keep8 = 0u;
                 keep16 |= keep8 << (8 * x);
                 if (olane != nullptr && in_row[x] &&
-                    SP_IN_RANGE(col + 8 * x + 7, jobs.job[jk].ldo, kDbgEwmaColumn)) {
+                    SP_IN_RANGE(col + 8 * x + 7, job.ldo, kDbgEwmaColumn)) {
 #pragma unroll
                     for (int k = 0; k < 4; ++k) p[x][k] &= ~pm[k];
                     __stcs(reinterpret_cast<uint4 *>(olane + tile * kTile + 8 * x),
@@ -537,10 +544,10 @@ ewma_pair_scan_kernel(const __grid_constant__ EwmaJobTable jobs, int n,
             kept = static_cast<uint32_t>(snap[4 + lane]);  // kept before that column
             if (is_lane0)
                 walked = gate_walk<BF16>(
-                    wrow, W_out != nullptr ? W_out + static_cast<int64_t>(row) * jobs.job[jk].ldo : nullptr,
+                    wrow, W_out != nullptr ? W_out + static_cast<int64_t>(row) * job.ldo : nullptr,
                     mask != nullptr ? mask + static_cast<int64_t>(row) * mask_words : nullptr, n,
                     snap[0], __fmul_rn(sc.alpha, __int_as_float(snap[1])),
-                    __fmul_rn(pc.unit_b[0], __int_as_float(snap[2])), colsq, factor, scalars,
+                    __fmul_rn(pc.unit_b[0], __int_as_float(snap[2])), job.colsq, job.factor, scalars,
                     sc.alpha, sc.beta, la, counters);
         }
     }
@@ -655,24 +662,37 @@ bool job_is_vector(const EwmaLaunchJob &j, int64_t n) {
            (j.W_out == nullptr || (aligned16(j.W_out) && j.ldo % 8 == 0));
 }
 
+// Statistics a job is pruned with: its own context's, else those of the call's context.
+inline const sp_ctx *job_ctx(const EwmaLaunchJob &j, const sp_ctx *ctx) {
+    return j.ctx != nullptr ? j.ctx : ctx;
+}
+
 // Device-side table of the jobs [first, first + count); false if there are too many rows.
-bool fill_job_table(const EwmaLaunchJob *jobs, int first, int count, EwmaJobTable &t) {
+bool fill_job_table(const sp_ctx *ctx, const EwmaLaunchJob *jobs, int first, int count,
+                    EwmaJobTable &t) {
     t.count = count;
-    int64_t rows = 0;
+    int64_t ctas = 0;
     for (int i = 0; i < count; ++i) {
         const EwmaLaunchJob &j = jobs[first + i];
+        const sp_ctx *c = job_ctx(j, ctx);
         EwmaJob &d = t.job[i];
         d.W = static_cast<const uint16_t *>(j.W);
         d.W_out = static_cast<uint16_t *>(j.W_out);
         d.mask = j.mask;
+        d.factor_pairs = c->factor_pairs;
+        d.scalars = c->scalars;
+        d.colsq = c->colsq;
+        d.factor = c->factor;
         d.ldw = static_cast<int>(j.ldw);
         d.ldo = static_cast<int>(j.ldo);
         d.n_rows = static_cast<int>(j.n_rows);
-        d.first_row = static_cast<int>(rows);
-        rows += j.n_rows;
+        d.n = static_cast<int>(c->d_in);
+        d.mask_words = static_cast<int>((c->d_in + 31) / 32);
+        d.first_cta = static_cast<int>(ctas);
+        ctas += (j.n_rows + kPairWarps - 1) / kPairWarps;
     }
-    t.total_rows = static_cast<int>(rows);
-    return rows <= kEwmaMaxLaunchRows;
+    t.total_ctas = static_cast<int>(ctas);
+    return ctas <= 0x7fffffffLL;
 }
 
 // The frozen-S scan (with the drift gate, if asked for) over jobs that share one launch: all of
@@ -681,21 +701,17 @@ sp_status launch_scan_group(const sp_ctx *ctx, const EwmaLaunchJob *jobs, int fi
                             sp_dtype dtype, const sp_ewma_params &p,
                             unsigned long long *counters, cudaStream_t stream,
                             bool la_from_device) {
-    const int64_t n = ctx->d_in;
     const bool bf16 = dtype == SP_BF16;
     const bool gated = p.s_update == SP_S_GATED;
-    const int words = static_cast<int>((n + 31) / 32);
     EwmaJobTable table{};
-    if (!fill_job_table(jobs, first, count, table)) return SP_ERR_SHAPE;
-    if (table.total_rows == 0) return SP_OK;
+    if (!fill_job_table(ctx, jobs, first, count, table)) return SP_ERR_SHAPE;
+    if (table.total_ctas == 0) return SP_OK;
 
     ScanConstants sc;
     fill_scan_constants(p, sc);
-    const DeviceScalars *scalars = ctx->scalars;
-    const double *colsq = ctx->colsq;
-    const float *factor = ctx->factor;
     cudaError_t launch_err = cudaSuccess;
-    const bool vec = job_is_vector(jobs[first], n);  // groups are uniform in this respect
+    const sp_ctx *c0 = job_ctx(jobs[first], ctx);
+    const bool vec = job_is_vector(jobs[first], c0->d_in);  // groups are uniform in this respect
     if (vec) {
         const double a = static_cast<double>(sc.a), b = static_cast<double>(sc.b);
         PairConstants pc{};
@@ -713,14 +729,12 @@ sp_status launch_scan_group(const sp_ctx *ctx, const EwmaLaunchJob *jobs, int fi
         }
         wc.a8 = sc.a_step[0];
         wc.b8 = sc.b_step[0];
-        const bool full_tiles = n % 512 == 0;
-        PdlConfig pdlp(dim3(static_cast<unsigned>((table.total_rows + kPairWarps - 1) / kPairWarps)),
-                       dim3(kPairThreads), stream);
-        const float *factor_pairs = ctx->factor_pairs;
+        bool full_tiles = true;  // every row of the launch a whole number of tiles
+        for (int i = 0; i < count; ++i) full_tiles = full_tiles && table.job[i].n % 512 == 0;
+        PdlConfig pdlp(dim3(static_cast<unsigned>(table.total_ctas)), dim3(kPairThreads), stream);
 #define SP_LAUNCH_P(B, F, C, G)                                                              \
-    launch_err = cudaLaunchKernelEx(&pdlp.cfg, ewma_pair_scan_kernel<B, F, C, G>, table,      \
-                                    static_cast<int>(n), factor_pairs, scalars, sc, pc, wc,   \
-                                    words, counters, colsq, factor)
+    launch_err = cudaLaunchKernelEx(&pdlp.cfg, ewma_pair_scan_kernel<B, F, C, G>, table, sc,  \
+                                    pc, wc, counters)
 #define SP_LAUNCH_PC(B, F, C)                                                                \
     do {                                                                                     \
         if (gated) SP_LAUNCH_P(B, F, C, true); else SP_LAUNCH_P(B, F, C, false);             \
@@ -739,12 +753,17 @@ sp_status launch_scan_group(const sp_ctx *ctx, const EwmaLaunchJob *jobs, int fi
 #undef SP_LAUNCH_P
     } else {
         const EwmaJob &j = table.job[0];
+        const int n = j.n, words = j.mask_words;
+        const float *factor = j.factor;
+        const DeviceScalars *scalars = j.scalars;
+        const double *colsq = j.colsq;
+        const int64_t ldw = j.ldw, ldo = j.ldo, n_rows = j.n_rows;
         PdlConfig pdl(dim3(static_cast<unsigned>((j.n_rows + kEwmaWarps - 1) / kEwmaWarps)),
                       dim3(kEwmaThreads), stream);
 #define SP_LAUNCH_S(B, C, G)                                                                 \
-    launch_err = cudaLaunchKernelEx(&pdl.cfg, ewma_scan_kernel<B, C, G>, j.W, j.ldw, j.n_rows, \
-                                    static_cast<int>(n), factor, scalars, sc, j.mask, words,  \
-                                    j.W_out, j.ldo, counters, colsq)
+    launch_err = cudaLaunchKernelEx(&pdl.cfg, ewma_scan_kernel<B, C, G>, j.W, ldw, n_rows, n, \
+                                    factor, scalars, sc, j.mask, words, j.W_out, ldo,         \
+                                    counters, colsq)
 #define SP_LAUNCH_SC(B, C)                                                                   \
     do {                                                                                     \
         if (gated) SP_LAUNCH_S(B, C, true); else SP_LAUNCH_S(B, C, false);                   \
@@ -791,13 +810,12 @@ sp_status launch_literal(const sp_ctx *ctx, const EwmaLaunchJob &j, sp_dtype dty
 sp_status launch_select_ewma(const sp_ctx *ctx, const EwmaLaunchJob *jobs_in, int n_jobs,
                              sp_dtype dtype, const sp_ewma_params &p, unsigned long long *counters,
                              cudaStream_t stream, bool la_from_device) {
-    const int64_t n = ctx->d_in;
-    const int64_t words = (n + 31) / 32;
     // Cut every matrix into pieces of at most kEwmaMaxLaunchRows rows ...
     EwmaLaunchJob pieces[64];
     int n_pieces = 0;
     for (int i = 0; i < n_jobs; ++i) {
         const EwmaLaunchJob &j = jobs_in[i];
+        const int64_t words = (job_ctx(j, ctx)->d_in + 31) / 32;
         if (j.n_rows < 0 || j.ldw > 0x7fffffffLL || j.ldo > 0x7fffffffLL) return SP_ERR_SHAPE;
         for (int64_t r0 = 0; r0 < j.n_rows; r0 += kEwmaMaxLaunchRows) {
             if (n_pieces == 64) return SP_ERR_SHAPE;
@@ -812,15 +830,15 @@ sp_status launch_select_ewma(const sp_ctx *ctx, const EwmaLaunchJob *jobs_in, in
     if (p.s_update == SP_S_LITERAL_SCAN) {
         for (int i = 0; i < n_pieces; ++i) {
             const EwmaLaunchJob &j = pieces[i];
-            sp_status st = launch_ewma_sweep(ctx, j.W, dtype, j.n_rows, j.ldw, p, j.mask, j.W_out,
-                                             j.ldo, counters, stream);
+            sp_status st = launch_ewma_sweep(job_ctx(j, ctx), j.W, dtype, j.n_rows, j.ldw, p, j.mask,
+                                             j.W_out, j.ldo, counters, stream);
             if (st != SP_OK) return st;
         }
         return SP_OK;
     }
     if (p.s_update == SP_S_LITERAL_W2 || p.s_update == SP_S_READING_X2) {
         for (int i = 0; i < n_pieces; ++i) {
-            sp_status st = launch_literal(ctx, pieces[i], dtype, p, counters, stream);
+            sp_status st = launch_literal(job_ctx(pieces[i], ctx), pieces[i], dtype, p, counters, stream);
             if (st != SP_OK) return st;
         }
         return SP_OK;
@@ -829,10 +847,10 @@ sp_status launch_select_ewma(const sp_ctx *ctx, const EwmaLaunchJob *jobs_in, in
     int first = 0;
     while (first < n_pieces) {
         int count = 1;
-        if (job_is_vector(pieces[first], n)) {
+        if (job_is_vector(pieces[first], job_ctx(pieces[first], ctx)->d_in)) {
             int64_t bits = pieces[first].n_rows;
             while (first + count < n_pieces && count < kEwmaMaxJobs &&
-                   job_is_vector(pieces[first + count], n)) {
+                   job_is_vector(pieces[first + count], job_ctx(pieces[first + count], ctx)->d_in)) {
                 const int64_t more = pieces[first + count].n_rows;
                 if (bits + more > kEwmaMaxLaunchRows) break;
                 bits += more;

@@ -39,7 +39,7 @@ namespace sp {
 #ifndef SP_NM_THREADS
 #define SP_NM_THREADS 128
 #endif
-constexpr int kNmMaxJobs = kEwmaMaxJobs;  // matrices one launch can cover
+constexpr int kNmMaxJobs = 8;  // matrices one launch can cover
 constexpr int kNmThreads = SP_NM_THREADS;
 constexpr int kNmWarps = kNmThreads / 32;
 constexpr int kNmRowsInFlight = SP_NM_ROWS_IN_FLIGHT;

@@ -18,7 +18,7 @@ constexpr int64_t kMaxDin = 1 << 20;
 constexpr int kFlagDegenerate = 1;
 
 constexpr int64_t kEwmaMaxLaunchRows = int64_t(1) << 30;  // rows one EWMA launch can cover
-constexpr int kEwmaMaxJobs = 8;                            // weight matrices, likewise
+constexpr int kEwmaMaxJobs = 16;                           // weight matrices, likewise
 
 // Scalars produced by finalisation; lives in device memory inside the context.
 struct DeviceScalars {
@@ -101,12 +101,13 @@ sp_status launch_select_24_compressed(const sp_ctx *ctx, const void *W, sp_dtype
                                       int64_t n_rows, int64_t ldw, void *values, int64_t ldv,
                                       uint32_t *meta, cudaStream_t stream);
 
-// One weight matrix of a selection launch that covers several (layers reading the same input).
+// One weight matrix of a selection launch that covers several.
 struct EwmaLaunchJob {
     const void *W;
     void *W_out;     // nullable
     uint32_t *mask;  // nullable
     int64_t n_rows, ldw, ldo;
+    const sp_ctx *ctx = nullptr;  // statistics to prune it with; null: those of the call's context
 };
 
 // select_nm.cu: N:M selection of up to kEwmaMaxJobs matrices that share the context
@@ -120,8 +121,8 @@ inline sp_status launch_select_nm(const sp_ctx *ctx, const void *W, sp_dtype dty
 }
 
 // select_ewma.cu
-// Algorithm 1 on up to kEwmaMaxJobs matrices that share the context (and dtype), in as few
-// launches as their layouts allow.
+// Algorithm 1 on several matrices of one dtype (each with the statistics of its own context, or
+// of `ctx`), in as few launches as their layouts allow.
 sp_status launch_select_ewma(const sp_ctx *ctx, const EwmaLaunchJob *jobs, int n_jobs,
                              sp_dtype dtype, const sp_ewma_params &p, unsigned long long *counters,
                              cudaStream_t stream, bool la_from_device = false);

@@ -99,23 +99,39 @@ def select_group(ctx: sp.Context, w: synth.Workload, Ws, masks, W_outs, mode_arg
         ctx.sp_select_unstructured_group(Ws, mode_arg, masks=masks, W_outs=W_outs, stream=stream)
 
 
+def select_block(mb: ModelBuffers, b: int, sparsity, stream=None):
+    """Algorithm 1 on every layer of block b in one call, each layer with the statistics of the
+    input it reads (sp_select_unstructured_multi)."""
+    w = mb.workload
+    sp.sp_select_unstructured_multi([mb.ctxs[layer.input] for layer in w.layers], mb.weights[b],
+                                    sparsity, masks=mb.masks[b], W_outs=mb.outputs[b],
+                                    stream=stream)
+
+
 def prune_model(mb: ModelBuffers, mode_arg, batch_tokens: int, phase_events=None, stream=None,
-                grouped: bool = True):
+                grouped: bool = True, per_block: bool | None = None):
     """One pass of the whole hot path over the model: for every block and every distinct layer
     input, accumulate the calibration statistics, finalise them, then select + write back every
     layer that reads this input.  phase_events, if given, is a list that receives
-    (kind, start_event, end_event, units) tuples per layer input: "calib" (units = activation
-    elements, brackets its back-to-back accumulate launches), "finalize", and "select" (units =
-    weights, brackets the back-to-back selection launches of the layers reading this input);
-    with phase_events the calls are issued strictly input by input so that the brackets are
+    (kind, start_event, end_event, units) tuples: "calib" (units = activation elements, brackets
+    the back-to-back accumulate launches of one layer input), "finalize", and "select" (units =
+    weights, brackets the back-to-back selection launches of one layer input, or of one block);
+    with phase_events the calls are issued strictly phase by phase so that the brackets are
     clean, without it the next input's calibration is enqueued ahead of the current input's
-    selections (same calls, same results).  With grouped (the default) the layers that read one
-    input are selected by one grouped call (one launch when their layouts allow); otherwise by
-    one call each.  Returns launch counts."""
+    selections where there are any (same calls, same results).
+
+    Selection calls: per_block (the default for unstructured pruning; N:M has no such call) prunes
+    all layers of a block with one call once all its inputs are calibrated; otherwise grouped
+    (the default) gives the layers that read one input one grouped call (one launch when their
+    layouts allow), else every layer gets a call of its own.  Returns launch counts."""
     w = mb.workload
     n_calib = n_select = n_final = 0
     if stream is None:
         stream = torch.cuda.current_stream()   # looked up once, not once per call
+    if per_block is None:
+        per_block = grouped and w.mode != "nm"
+    if per_block and w.mode == "nm":
+        raise ValueError("N:M selection has no per-block call")
 
     def mark():
         e = torch.cuda.Event(enable_timing=True)
@@ -135,6 +151,32 @@ def prune_model(mb: ModelBuffers, mode_arg, batch_tokens: int, phase_events=None
                              mode_arg, stream)
         n_select += sp.sp_launch_count() - before
         return sum(w.layers[li].d_out * w.layers[li].d_in for li in idx)
+
+    if per_block:
+        # calibrate + finalise every input of the block (the next input's accumulate launches
+        # follow an input's finalisation directly and stream under it), then one selection call
+        block_weights = sum(layer.d_out * layer.d_in for layer in w.layers)
+        last = mark() if phase_events is not None else None
+        for b in range(w.blocks):
+            for name, d_in in w.input_widths().items():
+                ctx = mb.ctxs[name]
+                n_calib += calibrate_input(ctx, mb.acts[name], batch_tokens, stream, True)
+                e1 = mark() if phase_events is not None else None
+                ctx.sp_score(None, stream=stream)          # finalisation only
+                n_final += 1
+                if phase_events is not None:
+                    e2 = mark()
+                    phase_events.append(("calib", last, e1, mb.acts[name].shape[0] * d_in))
+                    phase_events.append(("finalize", e1, e2, d_in))
+                    last = e2
+            before = sp.sp_launch_count()
+            select_block(mb, b, mode_arg, stream)
+            n_select += sp.sp_launch_count() - before
+            if phase_events is not None:
+                e3 = mark()
+                phase_events.append(("select", last, e3, block_weights))
+                last = e3
+        return {"calib": n_calib, "finalize": n_final, "select": n_select}
 
     if phase_events is None:
         # Plain pass.  The calibration of the next input is enqueued between an input's
@@ -226,15 +268,15 @@ def prune_model_split(mb: ModelBuffers, mode_arg, batch_tokens: int, rank: int, 
     return {"calib": n_calib, "finalize": n_final, "select": n_select}
 
 
-def capture_model_graph(mb: ModelBuffers, mode_arg, batch_tokens: int):
+def capture_model_graph(mb: ModelBuffers, mode_arg, batch_tokens: int, **how):
     """Captures one whole-model pass into a CUDA graph (for models whose layers are so small
     that the pass is bound by launch overhead).  The library's calls only enqueue kernels on the
     current stream, so they can be captured as they are.  Returns (graph, launch counts)."""
-    prune_model(mb, mode_arg, batch_tokens)       # everything allocated and finalised once
+    prune_model(mb, mode_arg, batch_tokens, **how)   # everything allocated and finalised once
     torch.cuda.synchronize()
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.graph(graph):
-        counts = prune_model(mb, mode_arg, batch_tokens)
+        counts = prune_model(mb, mode_arg, batch_tokens, **how)
     return graph, counts
 
 

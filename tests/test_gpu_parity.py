@@ -577,6 +577,53 @@ def test_whole_pass_can_be_captured_and_replayed_as_a_cuda_graph(sp):
         mb.close()
 
 
+def test_unstructured_pass_per_block_per_input_and_per_layer_calls_agree(sp):
+    from paper_2501_16376_b200 import pipeline, synth
+    w = synth.scaled(synth.WORKLOADS["llama3-8b"], blocks=2, n_seqs=4, seq_len=128, shrink=16)
+    mb = pipeline.allocate_model(w, "cuda")
+    try:
+        batch_tokens = 2 * w.seq_len
+        results = {}
+        for how, kw in (("block", {}), ("input", {"per_block": False}),
+                        ("layer", {"per_block": False, "grouped": False})):
+            for ms, os_ in zip(mb.masks, mb.outputs):
+                for m, o in zip(ms, os_):
+                    m.zero_()
+                    o.zero_()
+            counts = pipeline.prune_model(mb, 0.5, batch_tokens, **kw)
+            torch.cuda.synchronize()
+            results[how] = ([[m.clone() for m in ms] for ms in mb.masks],
+                            [[o.clone() for o in os_] for os_ in mb.outputs], counts)
+        assert results["block"][2]["select"] == w.blocks                 # one launch per block
+        assert results["input"][2]["select"] == w.blocks * len(w.input_widths())
+        assert results["layer"][2]["select"] == w.blocks * len(w.layers)
+        for how in ("input", "layer"):
+            for b in range(w.blocks):
+                for li in range(len(w.layers)):
+                    assert torch.equal(results["block"][0][b][li], results[how][0][b][li])
+                    assert torch.equal(results["block"][1][b][li].view(torch.int16),
+                                       results[how][1][b][li].view(torch.int16))
+        # the per-block pass under graph replay, with phase events, gives the same again
+        graph, counts = pipeline.capture_model_graph(mb, 0.5, batch_tokens)
+        for ms, os_ in zip(mb.masks, mb.outputs):
+            for m, o in zip(ms, os_):
+                m.zero_()
+                o.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert counts["select"] == w.blocks
+        events = []
+        pipeline.prune_model(mb, 0.5, batch_tokens, events)
+        torch.cuda.synchronize()
+        assert sum(1 for k, *_ in events if k == "select") == w.blocks
+        assert sum(u for k, _, _, u in events if k == "select") == w.total_weights()
+        for b in range(w.blocks):
+            for li in range(len(w.layers)):
+                assert torch.equal(mb.masks[b][li], results["block"][0][b][li])
+    finally:
+        mb.close()
+
+
 # ------------------------------------------------------------------ compressed 2:4 emission
 
 @pytest.mark.parametrize("R,n,dtype", [(130, 2048, torch.float16), (65, 520, torch.bfloat16),
@@ -677,6 +724,67 @@ def test_grouped_nm_selection_equals_single_calls_and_oracle(sp, N, M):
         if i < 2:
             assert torch.equal(mask, masks2[i]) and outs2[i].data_ptr() == clones[i].data_ptr()
             assert np.array_equal(P.bits(clones[i]), sel.W_out)
+
+
+@pytest.mark.parametrize("dtype,widths", [
+    (torch.float16, [512, 2048, 1024, 2048]),        # whole tiles everywhere, one context twice
+    (torch.bfloat16, [1536, 520, 4096, 1001]),       # ragged tiles; 1001: no 16-byte access
+])
+def test_multi_context_ewma_selection_equals_single_calls_and_oracle(sp, dtype, widths):
+    # one call, matrices that read different inputs (different widths and statistics)
+    rows = [37, 130, 64, 9, 21]
+    ctxs, Ws, owner = {}, [], []
+    for k, n in enumerate(widths):
+        if n not in ctxs:
+            ctxs[n] = _ctx_with_stats(sp, [_activations(90 + k, 1024, n, dtype)], n)
+        Ws.append(_gen(700 + k, (rows[k], n), dtype, 0.02))
+        owner.append(ctxs[n])
+    Ws.append(_gen(777, (rows[4], widths[0]), dtype, 0.02))   # a second matrix on the first input
+    owner.append(ctxs[widths[0]])
+    counters = sp.new_counters()
+    prm = sp.EwmaParams(0.125, 0.125, 0.2, sp.SP_S_GATED)
+    try:
+        masks, outs = sp.sp_select_unstructured_multi(owner, Ws, params=prm, counters=counters)
+        kept = 0
+        for ctx, W, mask, out in zip(owner, Ws, masks, outs):
+            n = W.shape[1]
+            m1, o1 = ctx.sp_select_unstructured(W, params=prm)
+            assert torch.equal(mask, m1)
+            assert torch.equal(out.contiguous().view(torch.int16), o1.contiguous().view(torch.int16))
+            st = so.Stats(ctx.sp_get_stats()[0].numpy().copy(), 1)
+            sel = so.select_ewma(P.bits(W), P.odtype(W), st, 0.2, want_trace=True)
+            P.check_selection(mask, out, W, sel, P.ewma_allowed_flips(sel))
+            kept += int(so.unpack_mask(P.mask_np(mask), n).sum())
+        assert int(counters[sp.SP_COUNTER_KEPT]) == kept
+        # the sparsity form, and the sequential modes through the same entry point
+        m2, o2 = sp.sp_select_unstructured_multi(owner[:2], Ws[:2], 0.6)
+        for ctx, W, mask, out in zip(owner[:2], Ws[:2], m2, o2):
+            m1, o1 = ctx.sp_select_unstructured(W, 0.6)
+            assert torch.equal(mask, m1) and torch.equal(out.view(torch.int16), o1.view(torch.int16))
+        lit = sp.EwmaParams(0.125, 0.125, 0.2, sp.SP_S_LITERAL_W2)
+        m3, o3 = sp.sp_select_unstructured_multi(owner[:3], Ws[:3], params=lit)
+        for ctx, W, mask, out in zip(owner[:3], Ws[:3], m3, o3):
+            m1, o1 = ctx.sp_select_unstructured(W, params=lit)
+            assert torch.equal(mask, m1) and torch.equal(out.view(torch.int16), o1.view(torch.int16))
+    finally:
+        for ctx in ctxs.values():
+            ctx.close()
+
+
+def test_multi_context_selection_rejects_bad_calls(sp):
+    W = _gen(3, (8, 512), torch.float16, 0.02)
+    X = _activations(4, 256, 512, torch.float16)
+    with _ctx_with_stats(sp, [X], 512) as ctx, sp.Context(512) as empty, sp.Context(1024) as wide:
+        with pytest.raises(sp.SpError) as e:
+            sp.sp_select_unstructured_multi([ctx] * (sp.SP_MAX_MULTI + 1),
+                                            [W] * (sp.SP_MAX_MULTI + 1), 0.5)
+        assert e.value.status == sp.SP_ERR_INVALID_ARG
+        with pytest.raises(sp.SpError) as e:
+            sp.sp_select_unstructured_multi([ctx, empty], [W, W], 0.5)     # no calibration data
+        assert e.value.status == sp.SP_ERR_STATE
+        with pytest.raises(sp.SpError) as e:
+            sp.sp_select_unstructured_multi([ctx, wide], [W, W], 0.5)      # W narrower than d_in
+        assert e.value.status == sp.SP_ERR_SHAPE
 
 
 def test_grouped_selection_rejects_bad_groups(sp):

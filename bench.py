@@ -39,14 +39,17 @@ CALIB_BYTES_PER_ELEMENT = 2.0
 
 # DRAM bytes (read + write) per launch from ncu captures of the kernels as committed
 # (summarised under profiles/), for the launch shapes of the default configuration
-# (32768-token calibration batches; selection launches grouped per layer input).
-# Keys: calibration -> d_in; selection -> (total rows of the launch, d_in).  Shapes that were
+# (32768-token calibration batches; selection launches per block or grouped per layer input).
+# Keys: calibration -> d_in; selection -> (total rows of the launch, d_in), or
+# ("block", workload) for one launch over all layers of a block.  Shapes that were
 # not captured, and kernels changed since, report null.
 NCU_CALIB_TRAFFIC = {4096: 272.0e6, 11008: 725.1e6}
 NCU_SELECT_TRAFFIC = {
     "select_nm_stream_kernel": {(12288, 4096): 156.0e6, (4096, 4096): 34.3e6,
                                 (22016, 4096): 318.4e6, (4096, 11008): 131.4e6},
-    "ewma_pair_scan_kernel": {},
+    "ewma_pair_scan_kernel": {("block", "llama3-8b"): 845.2e6,
+                              (6144, 4096): 54.2e6, (4096, 4096): 33.6e6,
+                              (28672, 4096): 426.1e6, (4096, 14336): 184.8e6},
 }
 
 

@@ -45,8 +45,7 @@ CALIB_BYTES_PER_ELEMENT = 2.0
 # not captured, and kernels changed since, report null.
 NCU_CALIB_TRAFFIC = {4096: 272.0e6, 11008: 725.1e6}
 NCU_SELECT_TRAFFIC = {
-    "select_nm_stream_kernel": {(12288, 4096): 156.0e6, (4096, 4096): 34.3e6,
-                                (22016, 4096): 318.4e6, (4096, 11008): 131.4e6},
+    "select_nm_stream_kernel": {},
     "ewma_pair_scan_kernel": {("block", "llama3-8b"): 845.2e6,
                               (6144, 4096): 54.2e6, (4096, 4096): 33.6e6,
                               (28672, 4096): 426.1e6, (4096, 14336): 184.8e6},
@@ -61,9 +60,8 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama2-7b")
     ap.add_argument("--select-launch", default="auto", choices=["auto", "block", "input", "layer"],
-                    help="selection calls of the pass: one per block (unstructured only), one per "
-                         "layer input (grouped), or one per layer; auto = block for unstructured "
-                         "workloads, input for N:M")
+                    help="selection calls of the pass: one per block, one per layer input "
+                         "(grouped), or one per layer; auto = block (input with --split)")
     ap.add_argument("--batch-seqs", type=int, default=16,
                     help="calibration sequences per sp_calib_accumulate call")
     ap.add_argument("--e2e-steps", type=int, default=1)
@@ -395,9 +393,9 @@ def gpu_arm(args):
 
     select_launch = args.select_launch
     if select_launch == "auto":
-        select_launch = "block" if w.mode != "nm" and not shared else "input"
-    if select_launch == "block" and (w.mode == "nm" or shared):
-        raise SystemExit("--select-launch block: unstructured single-model passes only")
+        select_launch = "input" if shared else "block"
+    if select_launch == "block" and shared:
+        raise SystemExit("--select-launch block: single-model passes only")
     how = {"grouped": select_launch != "layer", "per_block": select_launch == "block"}
 
     def one_pass():
@@ -513,29 +511,44 @@ def gpu_arm(args):
                     "block" if select_launch == "block" else "layer input"),
     }
 
-    # The same select kernel timed alone on the largest layer shape: back-to-back launches over
-    # every block's own weights / outputs (distinct buffers, far more than L2), statistics in place.
+    # The same select kernel timed alone on the largest layer shape: one launch per block over
+    # every block's own weights / outputs (distinct buffers, far more than L2), statistics in
+    # place, the sequence replayed as one CUDA graph so that the host's enqueue rate does not
+    # set the pace.
     li = max(range(len(w.layers)), key=lambda i: w.layers[i].d_out * w.layers[i].d_in)
     big = w.layers[li]
     if w.blocks * big.d_out * big.d_in * 4 > 256e6:
         ctx_big = mb.ctxs[big.input]
-        t0 = torch.cuda.Event(enable_timing=True)
-        t1 = torch.cuda.Event(enable_timing=True)
-        for rep in range(2):   # the first repetition warms up
-            t0.record()
+
+        def big_layer_launches():
             for b in range(w.blocks):
                 pipeline.select_layer(ctx_big, w, mb.weights[b][li], mb.masks[b][li],
                                       mb.outputs[b][li], arg)
+        big_layer_launches()
+        torch.cuda.synchronize()
+        alone_graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(alone_graph):
+            big_layer_launches()
+        t0 = torch.cuda.Event(enable_timing=True)
+        t1 = torch.cuda.Event(enable_timing=True)
+        alone_ms = None
+        for rep in range(3):   # the first repetition warms up
+            t0.record()
+            alone_graph.replay()
             t1.record()
             torch.cuda.synchronize()
-        alone_ms = t0.elapsed_time(t1) / w.blocks
+            if rep:
+                ms = t0.elapsed_time(t1) / w.blocks
+                alone_ms = ms if alone_ms is None else min(alone_ms, ms)
+        del alone_graph
         alone_gbs = SELECT_BYTES_PER_WEIGHT * big.d_out * big.d_in / (alone_ms * 1e-3) / 1e9
         roofline_select["alone"] = {
             "layer": "%dx%d" % (big.d_out, big.d_in), "launches": w.blocks,
             "avg_launch_ms": alone_ms, "achieved": alone_gbs, "frac": alone_gbs / peak,
             "frac_of_8TBs": alone_gbs / 8000.0,
-            "note": "select launches only, back to back over all blocks (no calibration traffic "
-                    "in between, so the SM clock is not held down by the power cap)",
+            "note": "select launches of this one layer only, back to back over all blocks as one "
+                    "CUDA graph (no calibration traffic in between, so the SM clock is not held "
+                    "down by the power cap)",
         }
 
     line = {

@@ -319,13 +319,18 @@ sp_status sp_select_nm_group(sp_ctx *ctx, const sp_matrix *mats /* host */, int 
  * each matrix is identical to that of its own sp_select_unstructured[_ex] call on its context;
  * what changes is the cost: one launch, whose tail the short rows fill, instead of one launch
  * and one ramp-up per layer input.  Every context with batches pending is finalised on `stream`
- * first.  counters (nullable, device) are totals over all items.
+ * first.  counters (nullable, device) are totals over all items.  sp_select_nm_multi is the
+ * same for the N:M rule of Section 3.3 (every ctxs[i]'s d_in a multiple of M, else
+ * SP_ERR_SHAPE; matrices that ask for different outputs than their neighbours, or do not allow
+ * 16-byte access, get launches of their own).
  */
 enum { SP_MAX_MULTI = 16 };
 sp_status sp_select_unstructured_multi(sp_ctx *const *ctxs /* host */,
                                        const sp_matrix *mats /* host */, int n_items,
                                        sp_dtype dtype, float sparsity,
                                        unsigned long long *counters, sp_stream stream);
+sp_status sp_select_nm_multi(sp_ctx *const *ctxs /* host */, const sp_matrix *mats /* host */,
+                             int n_items, sp_dtype dtype, int N, int M, sp_stream stream);
 sp_status sp_select_unstructured_multi_ex(sp_ctx *const *ctxs /* host */,
                                           const sp_matrix *mats /* host */, int n_items,
                                           sp_dtype dtype, const sp_ewma_params *params /* host */,

@@ -32,7 +32,7 @@ EXPORTS = (
     "sp_select_unstructured_ex", "sp_search_la", "sp_ewma_trace", "sp_select_nm", "sp_select_24_compressed", "sp_apply_mask", "sp_calib_accumulate_host",
     "sp_select_nm_host", "sp_select_unstructured_host", "sp_select_unstructured_group",
     "sp_select_unstructured_group_ex", "sp_select_nm_group", "sp_select_unstructured_multi",
-    "sp_select_unstructured_multi_ex", "sp_debug_status", "sp_status_string",
+    "sp_select_unstructured_multi_ex", "sp_select_nm_multi", "sp_debug_status", "sp_status_string",
     "sp_last_cuda_error", "sp_launch_count",
 )
 
@@ -95,6 +95,8 @@ def _load() -> ctypes.CDLL:
                                                  ci, f32, vp, vp]
     lib.sp_select_unstructured_multi_ex.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(Matrix), ci,
                                                     ci, ctypes.POINTER(EwmaParams), vp, vp]
+    lib.sp_select_nm_multi.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(Matrix), ci, ci, ci, ci,
+                                       vp]
     lib.sp_debug_status.argtypes = [ctypes.POINTER(ci), ctypes.POINTER(ci), ctypes.POINTER(i64),
                                     ctypes.POINTER(i64), ci]
     lib.sp_status_string.argtypes = [ci]
@@ -386,11 +388,8 @@ def _group(ctx, Ws, masks, W_outs, want_mask, inplace):
     return arr, k, dtype, masks, W_outs
 
 
-def sp_select_unstructured_multi(ctxs, Ws, sparsity=None, *, params: EwmaParams | None = None,
-                                 masks=None, W_outs=None, inplace=False, want_mask=True,
-                                 counters=None, stream=None):
-    """Algorithm 1 on matrices that read different layer inputs, in one call: Ws[i] is pruned
-    with the statistics of ctxs[i] (contexts may repeat).  Returns (masks, W_outs)."""
+def _multi(ctxs, Ws, masks, W_outs, want_mask, inplace):
+    """Marshals matrices with a context each into an sp_matrix array and a handle array."""
     k = len(Ws)
     if k != len(ctxs) or k < 1:
         raise SpError(SP_ERR_INVALID_ARG, "one context per matrix")
@@ -408,12 +407,30 @@ def sp_select_unstructured_multi(ctxs, Ws, sparsity=None, *, params: EwmaParams 
         optr, _, _, ldo = _matrix(W_outs[i], "W_out")
         arr[i] = Matrix(ptr, R, ld, _ptr(masks[i]), optr, ldo)
         handles[i] = ctx._h
+    return handles, arr, k, dtype, masks, W_outs
+
+
+def sp_select_unstructured_multi(ctxs, Ws, sparsity=None, *, params: EwmaParams | None = None,
+                                 masks=None, W_outs=None, inplace=False, want_mask=True,
+                                 counters=None, stream=None):
+    """Algorithm 1 on matrices that read different layer inputs, in one call: Ws[i] is pruned
+    with the statistics of ctxs[i] (contexts may repeat).  Returns (masks, W_outs)."""
+    handles, arr, k, dtype, masks, W_outs = _multi(ctxs, Ws, masks, W_outs, want_mask, inplace)
     if params is not None:
         _check(lib.sp_select_unstructured_multi_ex(handles, arr, k, dtype, ctypes.byref(params),
                                                    _ptr(counters), _stream(stream)))
     else:
         _check(lib.sp_select_unstructured_multi(handles, arr, k, dtype, float(sparsity),
                                                 _ptr(counters), _stream(stream)))
+    return masks, W_outs
+
+
+def sp_select_nm_multi(ctxs, Ws, N: int, M: int, *, masks=None, W_outs=None, inplace=False,
+                       want_mask=True, stream=None):
+    """N:M selection of matrices that read different layer inputs, in one call: Ws[i] is pruned
+    with the statistics of ctxs[i].  Returns (masks, W_outs)."""
+    handles, arr, k, dtype, masks, W_outs = _multi(ctxs, Ws, masks, W_outs, want_mask, inplace)
+    _check(lib.sp_select_nm_multi(handles, arr, k, dtype, int(N), int(M), _stream(stream)))
     return masks, W_outs
 
 

@@ -444,6 +444,34 @@ sp_status sp_select_nm_group(sp_ctx *ctx, const sp_matrix *mats, int n_mats, sp_
     return launch_select_nm(ctx, jobs, n_mats, dtype, N, M, s);
 }
 
+sp_status sp_select_nm_multi(sp_ctx *const *ctxs, const sp_matrix *mats, int n_items,
+                             sp_dtype dtype, int N, int M, sp_stream stream) {
+    SP_CALL_RANGE();
+    if (ctxs == nullptr || mats == nullptr) return SP_ERR_INVALID_ARG;
+    if (n_items < 1 || n_items > SP_MAX_MULTI) return SP_ERR_INVALID_ARG;
+    if (M != 4 && M != 8) return SP_ERR_INVALID_ARG;
+    if (N <= 0 || N >= M) return SP_ERR_INVALID_ARG;
+    EwmaLaunchJob jobs[SP_MAX_MULTI];
+    for (int i = 0; i < n_items; ++i) {
+        const sp_matrix &m = mats[i];
+        if (ctxs[i] == nullptr) return SP_ERR_INVALID_ARG;
+        sp_status st = check_matrix_args(ctxs[i], m.W, dtype, m.n_rows, m.ldw, m.W_out, m.ldo);
+        if (st != SP_OK) return st;
+        if (ctxs[i]->device != ctxs[0]->device) return SP_ERR_INVALID_ARG;
+        if (ctxs[i]->d_in % M != 0) return SP_ERR_SHAPE;
+        if (ctxs[i]->n_tokens <= 0) return SP_ERR_STATE;
+        jobs[i] = EwmaLaunchJob{m.W, m.W_out, m.mask_out, m.n_rows, m.ldw, m.ldo, ctxs[i]};
+    }
+    DeviceGuard guard(ctxs[0]->device);
+    if (guard.error() != cudaSuccess) return cuda_fail(guard.error());
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    for (int i = 0; i < n_items; ++i) {
+        sp_status st = ensure_finalized(ctxs[i], s);  // no work for a context seen before
+        if (st != SP_OK) return st;
+    }
+    return launch_select_nm(ctxs[0], jobs, n_items, dtype, N, M, s);
+}
+
 sp_status sp_ewma_trace(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows, int64_t ldw,
                         const sp_ewma_params *params, float *est_out, float *dev_out,
                         float *scores_out, sp_stream stream) {

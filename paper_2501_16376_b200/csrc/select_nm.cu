@@ -39,7 +39,7 @@ namespace sp {
 #ifndef SP_NM_THREADS
 #define SP_NM_THREADS 128
 #endif
-constexpr int kNmMaxJobs = 8;  // matrices one launch can cover
+constexpr int kNmMaxJobs = 16;  // matrices one launch can cover
 constexpr int kNmThreads = SP_NM_THREADS;
 constexpr int kNmWarps = kNmThreads / 32;
 constexpr int kNmRowsInFlight = SP_NM_ROWS_IN_FLIGHT;
@@ -148,38 +148,45 @@ select_nm_kernel(const uint16_t *__restrict__ W, int ldw, int n_rows, int64_t n,
 // little-endian mask word holds columns 8k .. 8k+7) instead of assembling words across lanes,
 // and when the strip is whole (FULL: d_in a multiple of 256) there are no column guards.
 // OUT / MASK: the pruned weights / the keep mask are requested.  The launch covers a table of
-// matrices that share the context (layers reading the same input); slabs are numbered through
-// all of them.
+// matrices, each with the per-channel factors of the input it reads (layers of one input, or all
+// layers of a block).  A matrix owns whole CTAs - strips x groups of kNmWarps slabs, strips
+// fastest - so the matrix of a CTA, and with it the width and every pointer, is CTA-uniform.
 struct NmJob {
     const uint16_t *W;
     uint16_t *W_out;  // nullable
     uint32_t *mask;   // nullable
+    const float *factor;
     int ldw, ldo, n_rows;
-    int first_slab;
+    int n, mask_words, strips;
+    int first_cta;
 };
 struct NmJobTable {
     int count;
-    int total_slabs;
+    int total_ctas;
     NmJob job[kNmMaxJobs];
 };
 
 template <bool BF16, bool FULL, int M, bool OUT, bool MASK>
 __global__ void __launch_bounds__(kNmThreads, SP_NM_MIN_BLOCKS)
-select_nm_stream_kernel(const __grid_constant__ NmJobTable jobs, int n, int rows_per_warp,
-                        const float *__restrict__ factor, int prune_count, int mask_words) {
+select_nm_stream_kernel(const __grid_constant__ NmJobTable jobs, int rows_per_warp,
+                        int prune_count) {
     pdl_launch_dependents();
     pdl_wait();  // the per-channel factors come from an earlier kernel of the stream
     const int lane = threadIdx.x & 31;
-    const int col = blockIdx.x * kStripChannels + lane * 8;
-    const int gslab = blockIdx.y * kNmWarps + (threadIdx.x >> 5);
-    if (gslab >= jobs.total_slabs) return;  // warp-uniform
-    int jk = 0;
-    while (jk + 1 < jobs.count && gslab >= jobs.job[jk + 1].first_slab) ++jk;
-    const uint16_t *const W = jobs.job[jk].W;
-    uint16_t *const W_out = jobs.job[jk].W_out;
-    uint32_t *const mask = jobs.job[jk].mask;
-    const int ldw = jobs.job[jk].ldw, ldo = jobs.job[jk].ldo, n_rows = jobs.job[jk].n_rows;
-    const int row_begin = (gslab - jobs.job[jk].first_slab) * rows_per_warp;  // < n_rows
+    int jk = 0;  // the matrix of this CTA
+    while (jk + 1 < jobs.count && static_cast<int>(blockIdx.x) >= jobs.job[jk + 1].first_cta) ++jk;
+    const NmJob &job = jobs.job[jk];
+    const int local = static_cast<int>(blockIdx.x) - job.first_cta;
+    const int slab_group = local / job.strips;
+    const int col = (local - slab_group * job.strips) * kStripChannels + lane * 8;
+    const int n = job.n, mask_words = job.mask_words;
+    const float *__restrict__ factor = job.factor;
+    const uint16_t *const W = job.W;
+    uint16_t *const W_out = job.W_out;
+    uint32_t *const mask = job.mask;
+    const int ldw = job.ldw, ldo = job.ldo, n_rows = job.n_rows;
+    const int row_begin = (slab_group * kNmWarps + (threadIdx.x >> 5)) * rows_per_warp;
+    if (row_begin >= n_rows) return;  // warp-uniform
     const int rows = min(n_rows - row_begin, rows_per_warp);
     const bool in_row = FULL || col < n;  // d_in % 8 == 0: a chunk is inside or outside as a whole
 
@@ -266,60 +273,83 @@ bool nm_job_is_vector(const EwmaLaunchJob &j, int64_t n) {
            (j.W_out == nullptr || (aligned16(j.W_out) && j.ldo % 8 == 0));
 }
 
+inline const sp_ctx *nm_job_ctx(const EwmaLaunchJob &j, const sp_ctx *ctx) {
+    return j.ctx != nullptr ? j.ctx : ctx;
+}
+
 // Jobs [first, first + count) in one launch: either all of them allow 16-byte access and ask
 // for the same outputs, or count == 1.
 sp_status launch_nm_group(const sp_ctx *ctx, const EwmaLaunchJob *jobs, int first, int count,
                           sp_dtype dtype, int N, int M, cudaStream_t stream) {
-    const int64_t n = ctx->d_in;
-    const int strips = ctx->strips;
-    int64_t total_rows = 0;
-    for (int i = 0; i < count; ++i) total_rows += jobs[first + i].n_rows;
+    int64_t row_strips = 0, total_rows = 0;  // warps' worth of work: rows x 256-column strips
+    for (int i = 0; i < count; ++i) {
+        row_strips += jobs[first + i].n_rows * nm_job_ctx(jobs[first + i], ctx)->strips;
+        total_rows += jobs[first + i].n_rows;
+    }
     if (total_rows == 0) return SP_OK;
     // Short slabs, i.e. many warps (measured: 8 rows per warp for the LLaMA-sized layers is 3-7 %
     // faster than 16-32, and than 4 once the SM clock is held down by the power cap).
     const int64_t target_warps = static_cast<int64_t>(ctx->sm_count) * SP_NM_TARGET_WARPS;
-    int64_t rows_per_warp = (total_rows * strips + target_warps - 1) / target_warps;
+    int64_t rows_per_warp = (row_strips + target_warps - 1) / target_warps;
     rows_per_warp = (rows_per_warp + kNmRowsInFlight - 1) / kNmRowsInFlight * kNmRowsInFlight;
     if (rows_per_warp < SP_NM_MIN_ROWS) rows_per_warp = SP_NM_MIN_ROWS;
-    const int64_t max_grid_y = 65535;
-    if ((total_rows + rows_per_warp * kNmWarps - 1) / (rows_per_warp * kNmWarps) + count > max_grid_y) {
-        // keep gridDim.y legal for very tall matrices by giving each warp more rows
-        rows_per_warp = (total_rows + (max_grid_y - count) * kNmWarps - 1) / ((max_grid_y - count) * kNmWarps);
-        rows_per_warp = (rows_per_warp + kNmRowsInFlight - 1) / kNmRowsInFlight * kNmRowsInFlight;
-    }
-    if (rows_per_warp > 0x7fffffffLL) return SP_ERR_SHAPE;
 
-    NmJobTable table{};
-    table.count = count;
-    int64_t slabs = 0;
-    for (int i = 0; i < count; ++i) {
-        const EwmaLaunchJob &j = jobs[first + i];
-        if (j.n_rows > 0x7fffffffLL || j.ldw > 0x7fffffffLL || j.ldo > 0x7fffffffLL) return SP_ERR_SHAPE;
-        NmJob &d = table.job[i];
-        d.W = static_cast<const uint16_t *>(j.W);
-        d.W_out = static_cast<uint16_t *>(j.W_out);
-        d.mask = j.mask;
-        d.ldw = static_cast<int>(j.ldw);
-        d.ldo = static_cast<int>(j.ldo);
-        d.n_rows = static_cast<int>(j.n_rows);
-        d.first_slab = static_cast<int>(slabs);
-        slabs += (j.n_rows + rows_per_warp - 1) / rows_per_warp;
-    }
-    if (slabs > 0x7fffffffLL) return SP_ERR_SHAPE;
-    table.total_slabs = static_cast<int>(slabs);
-    const dim3 grid(static_cast<unsigned>(strips),
-                    static_cast<unsigned>((slabs + kNmWarps - 1) / kNmWarps));
     const EwmaLaunchJob &j0 = jobs[first];
+    const sp_ctx *c0 = nm_job_ctx(j0, ctx);
+    const int64_t n = c0->d_in;
     const bool vec = nm_job_is_vector(j0, n);
+    if (!vec) {
+        // element-wise kernel (a single matrix, grid = strips x slab groups): keep gridDim.y legal
+        // for very tall matrices by giving each warp more rows
+        const int64_t max_grid_y = 65535;
+        if ((j0.n_rows + rows_per_warp * kNmWarps - 1) / (rows_per_warp * kNmWarps) > max_grid_y) {
+            rows_per_warp = (j0.n_rows + max_grid_y * kNmWarps - 1) / (max_grid_y * kNmWarps);
+            rows_per_warp = (rows_per_warp + kNmRowsInFlight - 1) / kNmRowsInFlight * kNmRowsInFlight;
+        }
+        if (rows_per_warp > 0x7fffffffLL) return SP_ERR_SHAPE;
+    }
+    NmJobTable table{};
+    int64_t ctas = 0;
+    for (;;) {  // the CTAs of the launch; a grid that would not fit gets longer slabs
+        table.count = count;
+        ctas = 0;
+        for (int i = 0; i < count; ++i) {
+            const EwmaLaunchJob &j = jobs[first + i];
+            const sp_ctx *c = nm_job_ctx(j, ctx);
+            if (j.n_rows > 0x7fffffffLL || j.ldw > 0x7fffffffLL || j.ldo > 0x7fffffffLL) return SP_ERR_SHAPE;
+            NmJob &d = table.job[i];
+            d.W = static_cast<const uint16_t *>(j.W);
+            d.W_out = static_cast<uint16_t *>(j.W_out);
+            d.mask = j.mask;
+            d.factor = c->factor;
+            d.ldw = static_cast<int>(j.ldw);
+            d.ldo = static_cast<int>(j.ldo);
+            d.n_rows = static_cast<int>(j.n_rows);
+            d.n = static_cast<int>(c->d_in);
+            d.mask_words = static_cast<int>((c->d_in + 31) / 32);
+            d.strips = c->strips;
+            d.first_cta = static_cast<int>(ctas);
+            const int64_t slabs = (j.n_rows + rows_per_warp - 1) / rows_per_warp;
+            ctas += (slabs + kNmWarps - 1) / kNmWarps * c->strips;
+        }
+        if (ctas <= 0x7fffffffLL) break;
+        rows_per_warp *= 2;
+        if (rows_per_warp > 0x7fffffffLL) return SP_ERR_SHAPE;
+    }
+    table.total_ctas = static_cast<int>(ctas);
     const uint16_t *Wp = static_cast<const uint16_t *>(j0.W);
     uint16_t *Op = static_cast<uint16_t *>(j0.W_out);
     uint32_t *mask = j0.mask;
     const int words = static_cast<int>((n + 31) / 32);
     const int prune_count = M - N;
     const int rpw = static_cast<int>(rows_per_warp);
-    PdlConfig pdl(grid, dim3(kNmThreads), stream);
-    const float *factor = ctx->factor;
+    const float *factor = c0->factor;
     cudaError_t launch_err = cudaSuccess;
+    const int64_t slabs0 = (j0.n_rows + rows_per_warp - 1) / rows_per_warp;
+    PdlConfig pdl(vec ? dim3(static_cast<unsigned>(ctas))
+                      : dim3(static_cast<unsigned>(c0->strips),
+                             static_cast<unsigned>((slabs0 + kNmWarps - 1) / kNmWarps)),
+                  dim3(kNmThreads), stream);
 #define SP_LAUNCH(B, MM)                                                                     \
     launch_err = cudaLaunchKernelEx(&pdl.cfg, select_nm_kernel<B, MM>, Wp,                    \
                                     static_cast<int>(j0.ldw), static_cast<int>(j0.n_rows), n, \
@@ -331,7 +361,7 @@ sp_status launch_nm_group(const sp_ctx *ctx, const EwmaLaunchJob *jobs, int firs
     } while (0)
 #define SP_LAUNCH_ST(B, F, MM, O, K)                                                         \
     launch_err = cudaLaunchKernelEx(&pdl.cfg, select_nm_stream_kernel<B, F, MM, O, K>, table, \
-                                    static_cast<int>(n), rpw, factor, prune_count, words)
+                                    rpw, prune_count)
 #define SP_LAUNCH_STO(B, F, MM)                                                               \
     do {                                                                                      \
         if (Op != nullptr && mask != nullptr) SP_LAUNCH_ST(B, F, MM, true, true);             \
@@ -342,7 +372,8 @@ sp_status launch_nm_group(const sp_ctx *ctx, const EwmaLaunchJob *jobs, int firs
     do {                                                                                      \
         if (M == 8) SP_LAUNCH_STO(B, F, 8); else SP_LAUNCH_STO(B, F, 4);                      \
     } while (0)
-    const bool full = n % kStripChannels == 0;
+    bool full = true;  // every matrix a whole number of strips wide
+    for (int i = 0; i < count; ++i) full = full && table.job[i].n % kStripChannels == 0;
     if (vec) {
         if (dtype == SP_BF16) {
             if (full) SP_LAUNCH_STM(true, true); else SP_LAUNCH_STM(true, false);
@@ -367,7 +398,6 @@ sp_status launch_nm_group(const sp_ctx *ctx, const EwmaLaunchJob *jobs, int firs
 
 sp_status launch_select_nm(const sp_ctx *ctx, const EwmaLaunchJob *jobs_in, int n_jobs,
                            sp_dtype dtype, int N, int M, cudaStream_t stream) {
-    const int64_t n = ctx->d_in;
     // jobs that produce nothing are dropped; consecutive jobs that allow 16-byte access and ask
     // for the same outputs share a launch
     EwmaLaunchJob jobs[kNmMaxJobs];
@@ -380,8 +410,9 @@ sp_status launch_select_nm(const sp_ctx *ctx, const EwmaLaunchJob *jobs_in, int 
     int first = 0;
     while (first < count) {
         int group = 1;
-        if (nm_job_is_vector(jobs[first], n)) {
-            while (first + group < count && nm_job_is_vector(jobs[first + group], n) &&
+        if (nm_job_is_vector(jobs[first], nm_job_ctx(jobs[first], ctx)->d_in)) {
+            while (first + group < count &&
+                   nm_job_is_vector(jobs[first + group], nm_job_ctx(jobs[first + group], ctx)->d_in) &&
                    (jobs[first + group].mask != nullptr) == (jobs[first].mask != nullptr) &&
                    (jobs[first + group].W_out != nullptr) == (jobs[first].W_out != nullptr))
                 ++group;

@@ -99,13 +99,18 @@ def select_group(ctx: sp.Context, w: synth.Workload, Ws, masks, W_outs, mode_arg
         ctx.sp_select_unstructured_group(Ws, mode_arg, masks=masks, W_outs=W_outs, stream=stream)
 
 
-def select_block(mb: ModelBuffers, b: int, sparsity, stream=None):
-    """Algorithm 1 on every layer of block b in one call, each layer with the statistics of the
-    input it reads (sp_select_unstructured_multi)."""
+def select_block(mb: ModelBuffers, b: int, mode_arg, stream=None):
+    """Every layer of block b in one call, each layer with the statistics of the input it reads
+    (sp_select_unstructured_multi / sp_select_nm_multi)."""
     w = mb.workload
-    sp.sp_select_unstructured_multi([mb.ctxs[layer.input] for layer in w.layers], mb.weights[b],
-                                    sparsity, masks=mb.masks[b], W_outs=mb.outputs[b],
-                                    stream=stream)
+    ctxs = [mb.ctxs[layer.input] for layer in w.layers]
+    if w.mode == "nm":
+        N, M = mode_arg
+        sp.sp_select_nm_multi(ctxs, mb.weights[b], N, M, masks=mb.masks[b], W_outs=mb.outputs[b],
+                              stream=stream)
+    else:
+        sp.sp_select_unstructured_multi(ctxs, mb.weights[b], mode_arg, masks=mb.masks[b],
+                                        W_outs=mb.outputs[b], stream=stream)
 
 
 def prune_model(mb: ModelBuffers, mode_arg, batch_tokens: int, phase_events=None, stream=None,
@@ -120,18 +125,16 @@ def prune_model(mb: ModelBuffers, mode_arg, batch_tokens: int, phase_events=None
     clean, without it the next input's calibration is enqueued ahead of the current input's
     selections where there are any (same calls, same results).
 
-    Selection calls: per_block (the default for unstructured pruning; N:M has no such call) prunes
-    all layers of a block with one call once all its inputs are calibrated; otherwise grouped
-    (the default) gives the layers that read one input one grouped call (one launch when their
-    layouts allow), else every layer gets a call of its own.  Returns launch counts."""
+    Selection calls: per_block (the default) prunes all layers of a block with one call once
+    all its inputs are calibrated; otherwise grouped gives the layers that read one input one
+    grouped call (one launch when their layouts allow), else every layer gets a call of its
+    own.  Returns launch counts."""
     w = mb.workload
     n_calib = n_select = n_final = 0
     if stream is None:
         stream = torch.cuda.current_stream()   # looked up once, not once per call
     if per_block is None:
-        per_block = grouped and w.mode != "nm"
-    if per_block and w.mode == "nm":
-        raise ValueError("N:M selection has no per-block call")
+        per_block = grouped
 
     def mark():
         e = torch.cuda.Event(enable_timing=True)

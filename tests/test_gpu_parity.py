@@ -567,7 +567,7 @@ def test_whole_pass_can_be_captured_and_replayed_as_a_cuda_graph(sp):
                 o.zero_()
         graph.replay()
         torch.cuda.synchronize()
-        assert counts["select"] == 2 * len(w.input_widths())   # one grouped launch per input
+        assert counts["select"] == w.blocks                    # one launch per block
         for b in range(w.blocks):
             for li in range(len(w.layers)):
                 assert torch.equal(mb.masks[b][li], want_masks[b][li])
@@ -577,9 +577,11 @@ def test_whole_pass_can_be_captured_and_replayed_as_a_cuda_graph(sp):
         mb.close()
 
 
-def test_unstructured_pass_per_block_per_input_and_per_layer_calls_agree(sp):
+@pytest.mark.parametrize("name,arg", [("llama3-8b", 0.5), ("llama2-7b", (2, 4)),
+                                      ("llama2-13b", (4, 8))])
+def test_pass_with_per_block_per_input_and_per_layer_calls_agree(sp, name, arg):
     from paper_2501_16376_b200 import pipeline, synth
-    w = synth.scaled(synth.WORKLOADS["llama3-8b"], blocks=2, n_seqs=4, seq_len=128, shrink=16)
+    w = synth.scaled(synth.WORKLOADS[name], blocks=2, n_seqs=4, seq_len=128, shrink=16)
     mb = pipeline.allocate_model(w, "cuda")
     try:
         batch_tokens = 2 * w.seq_len
@@ -590,7 +592,7 @@ def test_unstructured_pass_per_block_per_input_and_per_layer_calls_agree(sp):
                 for m, o in zip(ms, os_):
                     m.zero_()
                     o.zero_()
-            counts = pipeline.prune_model(mb, 0.5, batch_tokens, **kw)
+            counts = pipeline.prune_model(mb, arg, batch_tokens, **kw)
             torch.cuda.synchronize()
             results[how] = ([[m.clone() for m in ms] for ms in mb.masks],
                             [[o.clone() for o in os_] for os_ in mb.outputs], counts)
@@ -604,7 +606,7 @@ def test_unstructured_pass_per_block_per_input_and_per_layer_calls_agree(sp):
                     assert torch.equal(results["block"][1][b][li].view(torch.int16),
                                        results[how][1][b][li].view(torch.int16))
         # the per-block pass under graph replay, with phase events, gives the same again
-        graph, counts = pipeline.capture_model_graph(mb, 0.5, batch_tokens)
+        graph, counts = pipeline.capture_model_graph(mb, arg, batch_tokens)
         for ms, os_ in zip(mb.masks, mb.outputs):
             for m, o in zip(ms, os_):
                 m.zero_()
@@ -613,7 +615,7 @@ def test_unstructured_pass_per_block_per_input_and_per_layer_calls_agree(sp):
         torch.cuda.synchronize()
         assert counts["select"] == w.blocks
         events = []
-        pipeline.prune_model(mb, 0.5, batch_tokens, events)
+        pipeline.prune_model(mb, arg, batch_tokens, events)
         torch.cuda.synchronize()
         assert sum(1 for k, *_ in events if k == "select") == w.blocks
         assert sum(u for k, _, _, u in events if k == "select") == w.total_weights()
@@ -771,6 +773,41 @@ def test_multi_context_ewma_selection_equals_single_calls_and_oracle(sp, dtype, 
             ctx.close()
 
 
+@pytest.mark.parametrize("dtype,widths,N,M", [
+    (torch.float16, [512, 2048, 1024, 2048], 2, 4),     # whole strips everywhere
+    (torch.bfloat16, [1536, 520, 4096, 1004], 2, 4),    # ragged strips; 1004: no 16-byte access
+    (torch.float16, [1024, 264, 2048, 512], 4, 8),
+])
+def test_multi_context_nm_selection_equals_single_calls_and_oracle(sp, dtype, widths, N, M):
+    rows = [37, 130, 64, 9, 21]
+    ctxs, Ws, owner = {}, [], []
+    for k, n in enumerate(widths):
+        if n not in ctxs:
+            ctxs[n] = _ctx_with_stats(sp, [_activations(190 + k, 1024, n, dtype)], n)
+        Ws.append(_gen(800 + k, (rows[k], n), dtype, 0.02))
+        owner.append(ctxs[n])
+    Ws.append(_gen(877, (rows[4], widths[0]), dtype, 0.02))
+    owner.append(ctxs[widths[0]])
+    try:
+        masks, outs = sp.sp_select_nm_multi(owner, Ws, N, M)
+        for ctx, W, mask, out in zip(owner, Ws, masks, outs):
+            m1, o1 = ctx.sp_select_nm(W, N, M)
+            assert torch.equal(mask, m1)
+            assert torch.equal(out.contiguous().view(torch.int16), o1.contiguous().view(torch.int16))
+            st = so.Stats(ctx.sp_get_stats()[0].numpy().copy(), 1)
+            sel = so.select_nm(P.bits(W), P.odtype(W), st, N, M)
+            P.check_selection(mask, out, W, sel, None, strict=True)
+        # members that ask for different outputs (in place, no mask): launches of their own
+        clones = [W.clone() for W in Ws[:3]]
+        m2, o2 = sp.sp_select_nm_multi(owner[:3], clones, N, M, inplace=True, want_mask=False)
+        for i in range(3):
+            assert m2[i] is None and o2[i].data_ptr() == clones[i].data_ptr()
+            assert torch.equal(clones[i].view(torch.int16), outs[i].view(torch.int16))
+    finally:
+        for ctx in ctxs.values():
+            ctx.close()
+
+
 def test_multi_context_selection_rejects_bad_calls(sp):
     W = _gen(3, (8, 512), torch.float16, 0.02)
     X = _activations(4, 256, 512, torch.float16)
@@ -784,6 +821,17 @@ def test_multi_context_selection_rejects_bad_calls(sp):
         assert e.value.status == sp.SP_ERR_STATE
         with pytest.raises(sp.SpError) as e:
             sp.sp_select_unstructured_multi([ctx, wide], [W, W], 0.5)      # W narrower than d_in
+        assert e.value.status == sp.SP_ERR_SHAPE
+        with pytest.raises(sp.SpError) as e:
+            sp.sp_select_nm_multi([ctx, empty], [W, W], 2, 4)
+        assert e.value.status == sp.SP_ERR_STATE
+        with pytest.raises(sp.SpError) as e:
+            sp.sp_select_nm_multi([ctx], [W], 4, 4)
+        assert e.value.status == sp.SP_ERR_INVALID_ARG
+    W6 = _gen(5, (8, 516), torch.float16, 0.02)
+    with _ctx_with_stats(sp, [_activations(6, 64, 516, torch.float16)], 516) as c6:
+        with pytest.raises(sp.SpError) as e:
+            sp.sp_select_nm_multi([c6], [W6], 4, 8)                        # 516 % 8 != 0
         assert e.value.status == sp.SP_ERR_SHAPE
 
 

@@ -1,6 +1,5 @@
 """GPU parity at the full layer sizes of the five synthetic workloads, in the launch configuration
-the benchmark times (same calibration batch size; one selection call per block for the
-unstructured workloads, one grouped call per layer input for N:M).
+the benchmark times (same calibration batch size; one selection call per block).
 
 For the first and the last block of every model-shaped workload, every row of every layer is
 selected on the GPU and by the oracle and compared entry by entry.  The statistics of the first
@@ -89,41 +88,29 @@ def _run_workload(sp, name, modes):
         try:
             for input_name, d_in in w.input_widths().items():
                 ctxs[input_name] = _calibrate(sp, w, block, input_name, d_in, all_tokens=block == 0)
-            if w.mode != "nm":
-                # unstructured: one call per block over all its layers, as bench.py's pass makes it
-                Ws = [synth.gen_weight(w, block, l, "cuda") for l in w.layers]
-                owners = [ctxs[l.input][0] for l in w.layers]
-                for mode in modes:
+            # one call per block over all its layers, as bench.py's pass makes it
+            Ws = [synth.gen_weight(w, block, l, "cuda") for l in w.layers]
+            owners = [ctxs[l.input][0] for l in w.layers]
+            for mode in modes:
+                nm = mode if isinstance(mode, tuple) else None
+                if nm is not None:
+                    masks, outs = sp.sp_select_nm_multi(owners, Ws, nm[0], nm[1])
+                else:
                     masks, outs = sp.sp_select_unstructured_multi(owners, Ws, mode)
-                    for layer, W, mask, out in zip(w.layers, Ws, masks, outs):
-                        sel = so.select_unstructured(P.bits(W), P.odtype(W), ctxs[layer.input][1],
-                                                     mode, want_trace=True, threads=threads)
-                        f, e, achieved = _compare_layer(W, mask, out, sel, layer.d_in, None)
-                        flips += f
-                        entries += e
-                        report.append((block, layer.name, mode, round(achieved, 4)))
-                        del sel
-                    del masks, outs
-                del Ws
-                continue
-            for input_name, d_in in w.input_widths().items():
-                ctx, st = ctxs[input_name]
-                layers = [l for l in w.layers if l.input == input_name]
-                Ws = [synth.gen_weight(w, block, l, "cuda") for l in layers]
-                for nm in modes:
-                    if len(Ws) > 1:                          # the calls bench.py's driver makes
-                        masks, outs = ctx.sp_select_nm_group(Ws, nm[0], nm[1])
-                    else:
-                        masks, outs = (list(x) for x in zip(ctx.sp_select_nm(Ws[0], nm[0], nm[1])))
-                    for layer, W, mask, out in zip(layers, Ws, masks, outs):
+                for layer, W, mask, out in zip(w.layers, Ws, masks, outs):
+                    st = ctxs[layer.input][1]
+                    if nm is not None:
                         sel = so.select_nm(P.bits(W), P.odtype(W), st, nm[0], nm[1], threads=threads)
-                        f, e, achieved = _compare_layer(W, mask, out, sel, layer.d_in, nm)
-                        flips += f
-                        entries += e
-                        report.append((block, layer.name, nm, round(achieved, 4)))
-                        del sel
-                    del masks, outs
-                del Ws
+                    else:
+                        sel = so.select_unstructured(P.bits(W), P.odtype(W), st, mode,
+                                                     want_trace=True, threads=threads)
+                    f, e, achieved = _compare_layer(W, mask, out, sel, layer.d_in, nm)
+                    flips += f
+                    entries += e
+                    report.append((block, layer.name, mode, round(achieved, 4)))
+                    del sel
+                del masks, outs
+            del Ws
         finally:
             for ctx, _ in ctxs.values():
                 ctx.close()

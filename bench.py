@@ -45,7 +45,9 @@ CALIB_BYTES_PER_ELEMENT = 2.0
 # not captured, and kernels changed since, report null.
 NCU_CALIB_TRAFFIC = {4096: 272.0e6, 11008: 725.1e6}
 NCU_SELECT_TRAFFIC = {
-    "select_nm_stream_kernel": {},
+    "select_nm_stream_kernel": {("block", "llama2-7b"): 782.4e6,
+                                (12288, 4096): 154.9e6, (4096, 4096): 33.6e6,
+                                (22016, 4096): 314.6e6, (4096, 11008): 127.7e6},
     "ewma_pair_scan_kernel": {("block", "llama3-8b"): 845.2e6,
                               (6144, 4096): 54.2e6, (4096, 4096): 33.6e6,
                               (28672, 4096): 426.1e6, (4096, 14336): 184.8e6},
@@ -479,7 +481,8 @@ def gpu_arm(args):
     sel_traffic = None
     table = NCU_SELECT_TRAFFIC[sel_kernel]
     if select_launch == "block":     # one launch per block
-        sel_traffic = table.get(("block", w.name))
+        if w.mode != "nm" or arg == (2, 4):
+            sel_traffic = table.get(("block", w.name))
     elif select_launch == "input":   # one grouped launch per layer input: (total rows, d_in)
         shapes = []
         for name, d_in in w.input_widths().items():

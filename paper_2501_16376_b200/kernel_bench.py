@@ -13,8 +13,10 @@ fraction of the measured copy rate when MEASURED_PEAKS.json is present.
 
 Calls: ewma (default mode, drift gate on) | ewma-frozen | ewma-literal | ewma-literal-scan |
 ewma-x2 | nm |
-compressed24 | calib | search (24 counting passes).  --few N limits the number of buffers (for a
-profiler capture that should see only a handful of launches).
+compressed24 | calib | search (24 counting passes) | block (all layers of one block of
+--workload in one call: sp_select_nm_multi / sp_select_unstructured_multi; --shape is ignored).
+--few N limits the number of buffers (for a profiler capture that should see only a handful of
+launches).
 """
 from __future__ import annotations
 
@@ -128,6 +130,49 @@ def run(call: str, rows: int, cols: int, dtype, nm=(2, 4), reps: int = 5, few: i
             "frac_of_8TBs": gbs / 8000.0}
 
 
+def run_block(workload: str, blocks: int = 6, reps: int = 5):
+    """One selection call per block of a synthetic model (every layer with the statistics of the
+    input it reads), over `blocks` blocks' distinct buffers, replayed as one CUDA graph."""
+    from . import pipeline, synth
+    dev = torch.device("cuda", torch.cuda.current_device())
+    w0 = synth.WORKLOADS[workload]
+    w = synth.Workload(**{**w0.__dict__, "blocks": blocks, "n_seqs": 2})
+    mb = pipeline.allocate_model(w, dev)
+    for name in w.input_widths():
+        pipeline.calibrate_input(mb.ctxs[name], mb.acts[name], 4096)
+        mb.ctxs[name].sp_score(None)
+    arg = w.patterns[0] if w.mode == "nm" else w.sparsities[0]
+
+    def all_blocks():
+        for b in range(blocks):
+            pipeline.select_block(mb, b, arg)
+    all_blocks()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        all_blocks()
+    graph.replay()
+    torch.cuda.synchronize()
+    best = None
+    for _ in range(reps):
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        e0.record()
+        graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        t = e0.elapsed_time(e1) / blocks
+        best = t if best is None else min(best, t)
+    mb.close()
+    weights = sum(l.d_out * l.d_in for l in w.layers)
+    gbs = weights * 4.125 / (best * 1e-3) / 1e9
+    peak = _peak()
+    return {"call": "block", "workload": workload, "mode": w.mode, "mode_arg": str(arg),
+            "weights_per_block": weights, "blocks": blocks, "us_per_call": best * 1e3,
+            "algorithmic_GBs": gbs, "frac_of_measured_copy_rate": gbs / peak if peak else None,
+            "frac_of_8TBs": gbs / 8000.0}
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawTextHelpFormatter)
     ap.add_argument("--call", default="ewma")
@@ -139,9 +184,13 @@ def main(argv=None):
     ap.add_argument("--stats-scale", type=float, default=0.0,
                     help="replace the calibration statistics by uniform(1,2) * SCALE per channel "
                          "(e.g. 1e-3: S small enough for Algorithm 1's S update to matter)")
+    ap.add_argument("--workload", default="llama2-7b", help="model shape for --call block")
     args = ap.parse_args(argv)
     if not torch.cuda.is_available():
         raise SystemExit("kernel_bench needs a CUDA device")
+    if args.call == "block":
+        print(json.dumps(run_block(args.workload, args.few or 6, args.reps)), flush=True)
+        return 0
     dtype = torch.float16 if args.dtype == "f16" else torch.bfloat16
     nm = tuple(int(v) for v in args.nm.split(":"))
     for shape in args.shape or ["4096x4096"]:

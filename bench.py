@@ -63,7 +63,7 @@ def parse_args():
     ap.add_argument("--workload", default="llama2-7b")
     ap.add_argument("--select-launch", default="auto", choices=["auto", "block", "input", "layer"],
                     help="selection calls of the pass: one per block, one per layer input "
-                         "(grouped), or one per layer; auto = block (input with --split)")
+                         "(grouped), or one per layer; auto = block")
     ap.add_argument("--batch-seqs", type=int, default=16,
                     help="calibration sequences per sp_calib_accumulate call")
     ap.add_argument("--e2e-steps", type=int, default=1)
@@ -395,9 +395,9 @@ def gpu_arm(args):
 
     select_launch = args.select_launch
     if select_launch == "auto":
-        select_launch = "input" if shared else "block"
-    if select_launch == "block" and shared:
-        raise SystemExit("--select-launch block: single-model passes only")
+        select_launch = "block"
+    if select_launch != "block" and shared:
+        raise SystemExit("--split passes make one selection call per block")
     how = {"grouped": select_launch != "layer", "per_block": select_launch == "block"}
 
     def one_pass():

@@ -229,7 +229,7 @@ def prune_model_split(mb: ModelBuffers, mode_arg, batch_tokens: int, rank: int, 
     split == "tokens": for every block and layer input, rank r accumulates its share of the
     calibration tokens, the ranks sum their column sums of squares with one all-reduce of
     d_in + 1 doubles (sharding.merge_calibration), and rank r then prunes its share of the rows
-    of every layer that reads the input.  Masks and outputs of rows a rank does not own are left
+    of every layer of the block with one call.  Masks and outputs of rows a rank does not own are left
     untouched.  Returns launch counts."""
     from . import sharding
     w = mb.workload
@@ -252,22 +252,25 @@ def prune_model_split(mb: ModelBuffers, mode_arg, batch_tokens: int, rank: int, 
                 n_calib += calibrate_input(ctx, X, batch_tokens, stream, True)
             ctx.sp_score(None, stream=stream)
             n_final += 1
-            idx = [li for li, layer in enumerate(w.layers) if layer.input == name]
-            Ws, masks, outs = [], [], []
-            for li in idx:
-                rows = (sharding.row_share(w.layers[li].d_out, world, rank)
-                        if split == "tokens" else range(w.layers[li].d_out))
-                if len(rows) == 0:
-                    continue
-                Ws.append(mb.weights[b][li][rows.start:rows.stop])
-                masks.append(mb.masks[b][li][rows.start:rows.stop])
-                outs.append(mb.outputs[b][li][rows.start:rows.stop])
-            before = sp.sp_launch_count()
-            if len(Ws) > 1:
-                select_group(ctx, w, Ws, masks, outs, mode_arg, stream)
-            elif len(Ws) == 1:
-                select_layer(ctx, w, Ws[0], masks[0], outs[0], mode_arg, stream)
-            n_select += sp.sp_launch_count() - before
+        # this rank's rows of every layer of the block, in one call
+        ctxs, Ws, masks, outs = [], [], [], []
+        for li, layer in enumerate(w.layers):
+            rows = (sharding.row_share(layer.d_out, world, rank)
+                    if split == "tokens" else range(layer.d_out))
+            if len(rows) == 0:
+                continue
+            ctxs.append(mb.ctxs[layer.input])
+            Ws.append(mb.weights[b][li][rows.start:rows.stop])
+            masks.append(mb.masks[b][li][rows.start:rows.stop])
+            outs.append(mb.outputs[b][li][rows.start:rows.stop])
+        before = sp.sp_launch_count()
+        if Ws and w.mode == "nm":
+            sp.sp_select_nm_multi(ctxs, Ws, mode_arg[0], mode_arg[1], masks=masks, W_outs=outs,
+                                  stream=stream)
+        elif Ws:
+            sp.sp_select_unstructured_multi(ctxs, Ws, mode_arg, masks=masks, W_outs=outs,
+                                            stream=stream)
+        n_select += sp.sp_launch_count() - before
     return {"calib": n_calib, "finalize": n_final, "select": n_select}
 
 

@@ -626,6 +626,47 @@ def test_pass_with_per_block_per_input_and_per_layer_calls_agree(sp, name, arg):
         mb.close()
 
 
+@pytest.mark.parametrize("name,arg", [("llama3-8b", 0.5), ("llama2-7b", (2, 4))])
+def test_one_model_split_over_ranks_gives_the_single_rank_result(sp, name, arg):
+    # the strong-scaling pass, its ranks played one after the other on this GPU (the block split
+    # has no exchange; the token split of a single rank is the plain pass)
+    from paper_2501_16376_b200 import pipeline, synth
+    w = synth.scaled(synth.WORKLOADS[name], blocks=3, n_seqs=4, seq_len=128, shrink=16)
+    mb = pipeline.allocate_model(w, "cuda")
+    try:
+        batch_tokens = 2 * w.seq_len
+        pipeline.prune_model(mb, arg, batch_tokens)
+        torch.cuda.synchronize()
+        want_masks = [[m.clone() for m in ms] for ms in mb.masks]
+        want_out = [[o.clone() for o in os_] for os_ in mb.outputs]
+
+        def clear():
+            for ms, os_ in zip(mb.masks, mb.outputs):
+                for m, o in zip(ms, os_):
+                    m.zero_()
+                    o.zero_()
+
+        def check():
+            torch.cuda.synchronize()
+            for b in range(w.blocks):
+                for li in range(len(w.layers)):
+                    assert torch.equal(mb.masks[b][li], want_masks[b][li])
+                    assert torch.equal(mb.outputs[b][li].view(torch.int16),
+                                       want_out[b][li].view(torch.int16))
+        clear()
+        selects = 0
+        for rank in range(2):
+            selects += pipeline.prune_model_split(mb, arg, batch_tokens, rank, 2, "blocks")["select"]
+        assert selects == w.blocks
+        check()
+        clear()
+        counts = pipeline.prune_model_split(mb, arg, batch_tokens, 0, 1, "tokens")
+        assert counts["select"] == w.blocks
+        check()
+    finally:
+        mb.close()
+
+
 # ------------------------------------------------------------------ compressed 2:4 emission
 
 @pytest.mark.parametrize("R,n,dtype", [(130, 2048, torch.float16), (65, 520, torch.bfloat16),

@@ -110,7 +110,8 @@ struct EwmaLaunchJob {
     const sp_ctx *ctx = nullptr;  // statistics to prune it with; null: those of the call's context
 };
 
-// select_nm.cu: N:M selection of up to kEwmaMaxJobs matrices that share the context
+// select_nm.cu: N:M selection of up to kEwmaMaxJobs matrices (each with the statistics of its
+// own context, or of `ctx`), in as few launches as their layouts and requested outputs allow
 sp_status launch_select_nm(const sp_ctx *ctx, const EwmaLaunchJob *jobs, int n_jobs, sp_dtype dtype,
                            int N, int M, cudaStream_t stream);
 inline sp_status launch_select_nm(const sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows,

@@ -85,3 +85,42 @@ def test_random_ewma_cases(sp, seed):
         assert np.array_equal(P.bits(out), np.where(keep, P.bits(W_ref), 0))
         if counters is not None:
             assert int(counters[sp.SP_COUNTER_KEPT]) == int(keep.sum())
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_multi_context_calls_equal_single_calls(sp, seed):
+    # several random matrices with a context each (widths repeat, so contexts do), one call;
+    # every matrix must come out exactly as from its own call (those are checked above)
+    rng = np.random.default_rng(3000 + seed)
+    nm = seed % 2 == 1
+    N, M = [(2, 4), (4, 8), (3, 4)][(seed // 2) % 3]
+    k = int(rng.integers(2, 7))
+    dtype = torch.float16 if seed % 4 < 2 else torch.bfloat16
+    ctxs, owners, Ws = {}, [], []
+    try:
+        for _ in range(k):
+            while True:
+                R, n, W, big, colsq = _case(rng, need_multiple=M if nm else 1)
+                if W.dtype == dtype:
+                    break
+            if n not in ctxs:
+                ctxs[n] = sp.Context(n)
+                ctxs[n].sp_set_stats(torch.from_numpy(colsq), 5)
+            owners.append(ctxs[n])
+            Ws.append(W)
+        if nm:
+            masks, outs = sp.sp_select_nm_multi(owners, Ws, N, M)
+            singles = [c.sp_select_nm(W, N, M) for c, W in zip(owners, Ws)]
+        else:
+            counters = sp.new_counters()
+            prm = sp.EwmaParams(0.125, 0.25, float(rng.choice([0.5, -0.2, 1.0])), sp.SP_S_GATED)
+            masks, outs = sp.sp_select_unstructured_multi(owners, Ws, params=prm, counters=counters)
+            singles = [c.sp_select_unstructured(W, params=prm) for c, W in zip(owners, Ws)]
+            kept = sum(int(so.unpack_mask(P.mask_np(m), W.shape[1]).sum()) for m, W in zip(masks, Ws))
+            assert int(counters[sp.SP_COUNTER_KEPT]) == kept
+        for (m1, o1), m, o in zip(singles, masks, outs):
+            assert torch.equal(m, m1)
+            assert np.array_equal(P.bits(o), P.bits(o1))
+    finally:
+        for c in ctxs.values():
+            c.close()

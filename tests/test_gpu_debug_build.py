@@ -1,5 +1,6 @@
 """The debug build of the library (index checks compiled in: an out-of-range store is skipped
-and recorded, nothing traps) run over ragged, strided and grouped cases in a process of its own:
+and recorded, nothing traps) run over ragged, strided, grouped and multi-context cases in a
+process of its own:
 it must record no violation and give the release build's results."""
 import json
 import os
@@ -27,6 +28,7 @@ def digest(*tensors):
 
 g = torch.Generator(device="cuda").manual_seed(3)
 out = {}
+kept = {}
 for n, R, dtype in ((520, 77, torch.float16), (1536, 130, torch.bfloat16), (8704, 9, torch.float16)):
     W = (torch.randn(R, n, device="cuda", generator=g) * 0.02).to(dtype)
     X = torch.randn(700, n, device="cuda", generator=g).to(dtype)
@@ -41,6 +43,19 @@ for n, R, dtype in ((520, 77, torch.float16), (1536, 130, torch.bfloat16), (8704
         m4, o4 = ctx.sp_select_unstructured(W, params=sp.EwmaParams(0.125, 0.125, 0.5, sp.SP_S_LITERAL_SCAN))
         colsq = ctx.sp_get_stats()[0]
     out[str(n)] = digest(m1, o1, m2, o2, *ms, *os_, *mn, *on, m3, o3, m4, o4, colsq)
+    if dtype == torch.float16:
+        kept[n] = (W, X)
+# matrices that read different inputs, in one call each
+ctxs = {n: sp.Context(n) for n in kept}
+for n, (W, X) in kept.items():
+    ctxs[n].sp_calib_accumulate(X)
+owners = [ctxs[n] for n in kept] + [ctxs[520]]
+Ws = [kept[n][0] for n in kept] + [kept[520][0][:33]]
+mu, ou = sp.sp_select_unstructured_multi(owners, Ws, 0.5)
+mm, om = sp.sp_select_nm_multi(owners, Ws, 2, 4)
+out["multi"] = digest(*mu, *ou, *mm, *om)
+for c in ctxs.values():
+    c.close()
 out["debug_status"] = list(sp.sp_debug_status())
 print(json.dumps(out))
 """

@@ -210,7 +210,7 @@ void spo_select_ewma_f32(const uint16_t *W, int dtype, int64_t R, int64_t n, int
 #ifdef _OPENMP
 #pragma omp parallel for schedule(static) num_threads(nthreads > 0 ? nthreads : 1)
 #endif
-    for (int64_t r = 0; r < R; ++r) { /* "Parallel calculation for each row" */
+    for (int64_t r = 0; r < R; ++r) { /* rows are independent problems (the row loop of Algorithm 1 is parallel) */
         uint32_t *mrow = mask + r * words;
         for (int64_t k = 0; k < words; ++k)
             mrow[k] = 0;

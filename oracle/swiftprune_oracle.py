@@ -61,7 +61,9 @@ _lib = None
 def _load():
     global _lib
     if _lib is None:
-        lib = ctypes.CDLL(build())
+        # SWIFTPRUNE_ORACLE_LIBRARY: a library built elsewhere from (a copy of) the C source; the
+        # mutation test uses it to check that the pins catch planted mistakes
+        lib = ctypes.CDLL(os.environ.get("SWIFTPRUNE_ORACLE_LIBRARY") or build())
         i64, f32, f64, ci, vp = (ctypes.c_int64, ctypes.c_float, ctypes.c_double,
                                  ctypes.c_int, ctypes.c_void_p)
         lib.spo_decode_array.argtypes = [vp, ci, i64, vp]

@@ -1040,6 +1040,61 @@ def test_x2_reading_of_the_S_update_is_bit_exact(sp, R, n, misalign):
     assert not np.array_equal(other.mask, sel.mask)
 
 
+def _golden_trace(name):
+    import os
+    g = {}
+    with open(os.path.join(os.path.dirname(__file__), "golden", name)) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                key, *vals = line.split()
+                g[key] = vals
+    return g
+
+
+@pytest.mark.parametrize("name", ["ewma_hand_trace.txt", "ewma_hand_trace_alpha_ne_beta.txt"])
+@pytest.mark.parametrize("pad", [0, 2, 10])     # 6 columns: general kernel; 8, 16: paired-chain kernel
+def test_fixed_S_hand_traces_through_the_scan_kernels(sp, name, pad):
+    # the paper-derived hand evaluations, not the oracle, are the expected values here
+    g = _golden_trace(name)
+    w = [float(v) for v in g["w"]] + [0.0] * pad          # extra columns: w = 0, after the trace
+    colsq = [float(v) for v in g["colsq"]] + [0.0] * pad
+    n0, n = len(g["w"]), len(w)
+    W = torch.tensor([w, w], dtype=torch.float16, device="cuda")
+    prm = sp.EwmaParams(float(g["alpha"][0]), float(g["beta"][0]), float(g["la"][0]), sp.SP_S_FROZEN)
+    with sp.Context(n) as ctx:
+        ctx.sp_set_stats(torch.tensor(colsq, dtype=torch.float64), 1)
+        mask, out = ctx.sp_select_unstructured(W, params=prm)
+        est, dev, L = ctx.sp_ewma_trace(W, prm)
+    keep = so.unpack_mask(P.mask_np(mask), n)
+    want = [int(v) for v in g["keep"]]
+    assert keep[0, :n0].astype(int).tolist() == want and keep[1, :n0].astype(int).tolist() == want
+    assert out[0, :n0].float().cpu().tolist() == [wi if k else 0.0 for wi, k in zip(w, want)]
+    assert L.cpu().numpy()[0, :n0].tolist() == [float(v) for v in g["L"]]
+    thr = (est - prm.la * dev).cpu().numpy()[0, :n0].tolist()
+    assert thr == [float(v) for v in g["thr"]]
+
+
+@pytest.mark.parametrize("mode", ["literal", "gated"])
+def test_literal_S_hand_trace_through_the_library(sp, mode):
+    # S = 16 and w^2 up to 64: every pruned weight moves S, so the default (gated) call must
+    # give the printed algorithm's hand-evaluated decisions too
+    g = _golden_trace("ewma_hand_trace_literal_s.txt")
+    W = torch.tensor([[float(v) for v in g["w"]]], dtype=torch.float16, device="cuda")
+    n = W.shape[1]
+    prm = sp.EwmaParams(float(g["alpha"][0]), float(g["beta"][0]), float(g["la"][0]),
+                        sp.SP_S_LITERAL_W2 if mode == "literal" else sp.SP_S_GATED)
+    with sp.Context(n) as ctx:
+        ctx.sp_set_stats(torch.tensor([float(v) for v in g["colsq"]], dtype=torch.float64), 1)
+        mask, out = ctx.sp_select_unstructured(W, params=prm)
+        est, dev, L = ctx.sp_ewma_trace(W, prm)
+    keep = so.unpack_mask(P.mask_np(mask), n)[0].astype(int).tolist()
+    assert keep == [int(v) for v in g["keep"]]
+    thr = (est - prm.la * dev).cpu().numpy()[0].tolist()
+    assert thr == [float(v) for v in g["thr"]]
+    assert np.allclose(L.cpu().numpy()[0], [float(v) for v in g["L"]], rtol=3e-7)
+
+
 def test_x2_reading_hand_trace_through_the_library(sp):
     import os
     g = {}

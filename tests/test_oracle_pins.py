@@ -200,6 +200,17 @@ def test_hand_trace_fixed_S(precision):
 
 
 @pytest.mark.parametrize("precision", ["f32", "f64"])
+def test_hand_trace_with_different_alpha_and_beta(precision):
+    # alpha belongs to est, beta to dev: a mix-up changes the thresholds from column 2 on
+    g = _read_golden("ewma_hand_trace_alpha_ne_beta.txt")
+    sel = _run_trace(g, so.S_FROZEN, precision)
+    n = len(g["w"])
+    assert sel.L[0].tolist() == [float(v) for v in g["L"]]
+    assert sel.thr[0].tolist() == [float(v) for v in g["thr"]]
+    assert sel.keep_bool(n)[0].astype(int).tolist() == [int(v) for v in g["keep"]]
+
+
+@pytest.mark.parametrize("precision", ["f32", "f64"])
 def test_hand_trace_literal_S_update(precision):
     g = _read_golden("ewma_hand_trace_literal_s.txt")
     n = len(g["w"])

@@ -64,6 +64,10 @@ def parse_args():
     ap.add_argument("--select-launch", default="auto", choices=["auto", "block", "input", "layer"],
                     help="selection calls of the pass: one per block, one per layer input "
                          "(grouped), or one per layer; auto = block")
+    ap.add_argument("--calib-launch", default="auto", choices=["auto", "input", "shared"],
+                    help="accumulate launches: one per layer input and batch, or shared by the "
+                         "inputs of a block (sp_calib_accumulate_multi); auto = shared when a "
+                         "batch of the widest input is at most 64 MiB")
     ap.add_argument("--batch-seqs", type=int, default=16,
                     help="calibration sequences per sp_calib_accumulate call")
     ap.add_argument("--e2e-steps", type=int, default=1)
@@ -399,6 +403,10 @@ def gpu_arm(args):
     if select_launch != "block" and shared:
         raise SystemExit("--split passes make one selection call per block")
     how = {"grouped": select_launch != "layer", "per_block": select_launch == "block"}
+    if args.calib_launch != "auto":
+        if args.calib_launch == "shared" and select_launch != "block":
+            raise SystemExit("--calib-launch shared needs --select-launch block")
+        how["multi_calib"] = args.calib_launch == "shared"
 
     def one_pass():
         if shared:
@@ -569,6 +577,9 @@ def gpu_arm(args):
                              sum(x.numel() * 2 for x in mb.acts.values()) / 1e9,
                              min(x.numel() * 2 for x in mb.acts.values()) / 1e9),
                    "launch": "cuda graph replay" if graph is not None else "stream launches",
+                   "calib_launch": ("one per layer input and batch" if counts["calib"] ==
+                                    w.blocks * len(w.input_widths()) * -(-w.tokens // batch_tokens)
+                                    or shared else "shared by the inputs of a block"),
                    "calib_flags": "SP_CALIB_X_COMPLETE (the activations are resident and complete "
                                   "long before the step starts)",
                    "parallelism": ("single GPU" if world == 1 else

@@ -142,6 +142,34 @@ sp_status sp_calib_accumulate_ex(sp_ctx *ctx, const void *X, sp_dtype dtype, int
                                  int64_t ldx, unsigned flags, sp_stream stream);
 
 /*
+ * One batch for each of several layer inputs (the inputs of one transformer block, say) in one
+ * launch: exactly the effect of sp_calib_accumulate_ex(ctxs[i], batches[i].X, dtype,
+ * batches[i].n_tokens, batches[i].ldx, flags, stream) for every i, bit for bit - Algorithm 1's
+ * step 1 is a sum per channel, and the channels of different inputs have nothing to do with
+ * each other.  For inputs so narrow or batches so short that a launch of their own would be
+ * mostly ramp-up.  ctxs and batches are HOST arrays of n_items entries (1 <= n_items <=
+ * SP_MAX_MULTI); the contexts must all be different (two batches of one launch cannot update
+ * the same sums: SP_ERR_INVALID_ARG) and on one device; a batch with n_tokens == 0 is skipped;
+ * batches that do not allow 16-byte access get launches of their own.
+ */
+typedef struct {
+    const void *X;    /* device, [n_tokens, d_in of its context] of the call's dtype */
+    int64_t n_tokens;
+    int64_t ldx;      /* elements */
+} sp_batch;
+sp_status sp_calib_accumulate_multi(sp_ctx *const *ctxs /* host */,
+                                    const sp_batch *batches /* host */, int n_items,
+                                    sp_dtype dtype, unsigned flags, sp_stream stream);
+
+/*
+ * Finalisation of several contexts at once: S and the per-channel factors of Eq. 8 for every
+ * listed context that has batches pending, by one launch (what sp_score(ctx, NULL, ...) does for
+ * one context; the selection calls do it implicitly).  A context without calibration data gives
+ * SP_ERR_STATE; a context may appear more than once.
+ */
+sp_status sp_finalize_multi(sp_ctx *const *ctxs /* host */, int n_items, sp_stream stream);
+
+/*
  * Reads the statistics back to HOST buffers (any may be NULL) and synchronises
  * the stream: colsq_host[d_in] (fp64), *S_host, factor_host[d_in] (the fp32
  * per-channel factor c_q = 1/(2(1 - colsq[q]/S)) of Eq. 8), *n_tokens_host.
@@ -319,7 +347,7 @@ sp_status sp_select_nm_group(sp_ctx *ctx, const sp_matrix *mats /* host */, int 
  * each matrix is identical to that of its own sp_select_unstructured[_ex] call on its context;
  * what changes is the cost: one launch, whose tail the short rows fill, instead of one launch
  * and one ramp-up per layer input.  Every context with batches pending is finalised on `stream`
- * first.  counters (nullable, device) are totals over all items.  sp_select_nm_multi is the
+ * first (all of them by one launch).  counters (nullable, device) are totals over all items.  sp_select_nm_multi is the
  * same for the N:M rule of Section 3.3 (every ctxs[i]'s d_in a multiple of M, else
  * SP_ERR_SHAPE; matrices that ask for different outputs than their neighbours, or do not allow
  * 16-byte access, get launches of their own).

@@ -26,7 +26,7 @@ SP_CALIB_X_COMPLETE = 1
 
 #: every symbol include/swiftprune.h declares
 EXPORTS = (
-    "sp_create", "sp_destroy", "sp_calib_reset", "sp_calib_accumulate", "sp_calib_accumulate_ex",
+    "sp_create", "sp_destroy", "sp_calib_reset", "sp_calib_accumulate", "sp_calib_accumulate_ex", "sp_calib_accumulate_multi", "sp_finalize_multi",
     "sp_get_stats",
     "sp_set_stats", "sp_calib_stats_noalloc", "sp_score", "sp_la_for_sparsity", "sp_select_unstructured",
     "sp_select_unstructured_ex", "sp_search_la", "sp_ewma_trace", "sp_select_nm", "sp_select_24_compressed", "sp_apply_mask", "sp_calib_accumulate_host",
@@ -52,6 +52,11 @@ class Matrix(ctypes.Structure):
     """sp_matrix: one weight matrix of a grouped selection call."""
     _fields_ = [("W", ctypes.c_void_p), ("n_rows", ctypes.c_int64), ("ldw", ctypes.c_int64),
                 ("mask_out", ctypes.c_void_p), ("W_out", ctypes.c_void_p), ("ldo", ctypes.c_int64)]
+
+
+class Batch(ctypes.Structure):
+    """sp_batch: one batch of calibration activations of a multi-input call."""
+    _fields_ = [("X", ctypes.c_void_p), ("n_tokens", ctypes.c_int64), ("ldx", ctypes.c_int64)]
 
 
 SP_MAX_GROUP = 8
@@ -95,6 +100,9 @@ def _load() -> ctypes.CDLL:
                                                  ci, f32, vp, vp]
     lib.sp_select_unstructured_multi_ex.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(Matrix), ci,
                                                     ci, ctypes.POINTER(EwmaParams), vp, vp]
+    lib.sp_calib_accumulate_multi.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(Batch), ci, ci,
+                                              ctypes.c_uint, vp]
+    lib.sp_finalize_multi.argtypes = [ctypes.POINTER(vp), ci, vp]
     lib.sp_select_nm_multi.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(Matrix), ci, ci, ci, ci,
                                        vp]
     lib.sp_debug_status.argtypes = [ctypes.POINTER(ci), ctypes.POINTER(ci), ctypes.POINTER(i64),
@@ -386,6 +394,34 @@ def _group(ctx, Ws, masks, W_outs, want_mask, inplace):
         optr, _, _, ldo = _matrix(W_outs[i], "W_out")
         arr[i] = Matrix(ptr, R, ld, _ptr(masks[i]), optr, ldo)
     return arr, k, dtype, masks, W_outs
+
+
+def sp_calib_accumulate_multi(ctxs, Xs, stream=None, x_complete: bool = False):
+    """One batch for each of several layer inputs in one call: Xs[i] ([tokens, d_in of ctxs[i]],
+    all of one dtype) is added to the statistics of ctxs[i]; the contexts must all differ."""
+    k = len(Xs)
+    if k != len(ctxs) or k < 1:
+        raise SpError(SP_ERR_INVALID_ARG, "one context per batch")
+    arr = (Batch * k)()
+    handles = (ctypes.c_void_p * k)()
+    dtype = _dtype_of(Xs[0])
+    for i, (ctx, X) in enumerate(zip(ctxs, Xs)):
+        ptr, T, n, ld = _matrix(X, "X")
+        if n != ctx.d_in:
+            raise SpError(SP_ERR_SHAPE, "X has %d channels, context has %d" % (n, ctx.d_in))
+        if _dtype_of(X) != dtype:
+            raise SpError(SP_ERR_DTYPE, "all batches of a call must have the same dtype")
+        arr[i] = Batch(ptr, T, ld)
+        handles[i] = ctx._h
+    _check(lib.sp_calib_accumulate_multi(handles, arr, k, dtype,
+                                         SP_CALIB_X_COMPLETE if x_complete else 0,
+                                         _stream(stream)))
+
+
+def sp_finalize_multi(ctxs, stream=None):
+    """S and the per-channel factors of every listed context with batches pending, one launch."""
+    handles = (ctypes.c_void_p * len(ctxs))(*[c._h for c in ctxs])
+    _check(lib.sp_finalize_multi(handles, len(ctxs), _stream(stream)))
 
 
 def _multi(ctxs, Ws, masks, W_outs, want_mask, inplace):

@@ -200,6 +200,57 @@ sp_status sp_calib_accumulate_ex(sp_ctx *ctx, const void *X, sp_dtype dtype, int
                                    (flags & SP_CALIB_X_COMPLETE) != 0u);
 }
 
+sp_status sp_calib_accumulate_multi(sp_ctx *const *ctxs, const sp_batch *batches, int n_items,
+                                    sp_dtype dtype, unsigned flags, sp_stream stream) {
+    SP_CALL_RANGE();
+    if (ctxs == nullptr || batches == nullptr) return SP_ERR_INVALID_ARG;
+    if (n_items < 1 || n_items > SP_MAX_MULTI) return SP_ERR_INVALID_ARG;
+    if (!valid_dtype(dtype)) return SP_ERR_DTYPE;
+    if ((flags & ~static_cast<unsigned>(SP_CALIB_X_COMPLETE)) != 0u) return SP_ERR_INVALID_ARG;
+    for (int i = 0; i < n_items; ++i) {
+        if (ctxs[i] == nullptr || batches[i].n_tokens < 0) return SP_ERR_INVALID_ARG;
+        if (batches[i].n_tokens > 0 && batches[i].X == nullptr) return SP_ERR_INVALID_ARG;
+        if (batches[i].ldx < ctxs[i]->d_in) return SP_ERR_SHAPE;
+        if (ctxs[i]->device != ctxs[0]->device) return SP_ERR_INVALID_ARG;
+        for (int k = 0; k < i; ++k)  // two batches of one launch cannot update the same sums
+            if (ctxs[k] == ctxs[i]) return SP_ERR_INVALID_ARG;
+    }
+    DeviceGuard guard(ctxs[0]->device);
+    if (guard.error() != cudaSuccess) return cuda_fail(guard.error());
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const bool x_complete = (flags & SP_CALIB_X_COMPLETE) != 0u;
+    // batches that allow 16-byte access share launches of up to 8; the others go one by one
+    sp_ctx *group_ctx[8];
+    CalibItem group[8];
+    int n_group = 0;
+    auto flush = [&]() -> sp_status {
+        sp_status st = SP_OK;
+        if (n_group == 1)
+            st = launch_calib_accumulate(group_ctx[0], group[0].X, dtype, group[0].n_tokens,
+                                         group[0].ldx, s, x_complete);
+        else if (n_group > 1)
+            st = launch_calib_accumulate_multi(group_ctx, group, n_group, dtype, s, x_complete);
+        n_group = 0;
+        return st;
+    };
+    for (int i = 0; i < n_items; ++i) {
+        const sp_batch &b = batches[i];
+        if (b.n_tokens == 0) continue;
+        if (!calib_multi_applies(ctxs[i], b.X, b.ldx)) {
+            sp_status st = launch_calib_accumulate(ctxs[i], b.X, dtype, b.n_tokens, b.ldx, s, x_complete);
+            if (st != SP_OK) return st;
+            continue;
+        }
+        group_ctx[n_group] = ctxs[i];
+        group[n_group] = CalibItem{b.X, b.n_tokens, b.ldx};
+        if (++n_group == 8) {
+            sp_status st = flush();
+            if (st != SP_OK) return st;
+        }
+    }
+    return flush();
+}
+
 sp_status sp_calib_accumulate(sp_ctx *ctx, const void *X, sp_dtype dtype, int64_t n_tokens,
                               int64_t ldx, sp_stream stream) {
     SP_CALL_RANGE();
@@ -280,6 +331,18 @@ sp_status sp_score(sp_ctx *ctx, const void *W, sp_dtype dtype, int64_t n_rows, i
     sp_status st = ensure_finalized(ctx, s);
     if (st != SP_OK || scores_out == nullptr) return st;
     return launch_score(ctx, W, dtype, n_rows, ldw, scores_out, s);
+}
+
+sp_status sp_finalize_multi(sp_ctx *const *ctxs, int n_items, sp_stream stream) {
+    SP_CALL_RANGE();
+    if (ctxs == nullptr || n_items < 1 || n_items > SP_MAX_MULTI) return SP_ERR_INVALID_ARG;
+    for (int i = 0; i < n_items; ++i) {
+        if (ctxs[i] == nullptr || ctxs[i]->device != ctxs[0]->device) return SP_ERR_INVALID_ARG;
+        if (ctxs[i]->n_tokens <= 0) return SP_ERR_STATE;
+    }
+    DeviceGuard guard(ctxs[0]->device);
+    if (guard.error() != cudaSuccess) return cuda_fail(guard.error());
+    return launch_finalize_pending(ctxs, n_items, static_cast<cudaStream_t>(stream));
 }
 
 sp_status sp_la_for_sparsity(float sparsity, float *la_out) {
@@ -406,10 +469,8 @@ sp_status sp_select_unstructured_multi_ex(sp_ctx *const *ctxs, const sp_matrix *
     DeviceGuard guard(ctxs[0]->device);
     if (guard.error() != cudaSuccess) return cuda_fail(guard.error());
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    for (int i = 0; i < n_items; ++i) {
-        sp_status st = ensure_finalized(ctxs[i], s);  // no work for a context seen before
-        if (st != SP_OK) return st;
-    }
+    sp_status fin = launch_finalize_pending(ctxs, n_items, s);  // one launch for all that need it
+    if (fin != SP_OK) return fin;
     return launch_select_ewma(ctxs[0], jobs, n_items, dtype, *params, counters, s);
 }
 
@@ -465,10 +526,8 @@ sp_status sp_select_nm_multi(sp_ctx *const *ctxs, const sp_matrix *mats, int n_i
     DeviceGuard guard(ctxs[0]->device);
     if (guard.error() != cudaSuccess) return cuda_fail(guard.error());
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    for (int i = 0; i < n_items; ++i) {
-        sp_status st = ensure_finalized(ctxs[i], s);  // no work for a context seen before
-        if (st != SP_OK) return st;
-    }
+    sp_status fin = launch_finalize_pending(ctxs, n_items, s);  // one launch for all that need it
+    if (fin != SP_OK) return fin;
     return launch_select_nm(ctxs[0], jobs, n_items, dtype, N, M, s);
 }
 

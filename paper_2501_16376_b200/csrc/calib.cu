@@ -21,12 +21,15 @@ constexpr int kCalibWarps = kCalibThreads / 32;
 constexpr int kRowsInFlight = 8;
 constexpr int kFinalGroups = 4;  // slab groups summed in parallel by the finalisation kernel
 constexpr int kFinalThreads = kFinalGroups * kStripChannels;
+constexpr int kFinalMaxJobs = 16;  // contexts one finalisation launch can cover
 
+// The work of one CTA: cell (strip, slab) of one activation matrix.
 template <bool BF16, bool VEC>
-__global__ void __launch_bounds__(kCalibThreads)
-calib_accumulate_kernel(const uint16_t *__restrict__ X, int64_t ldx, int64_t n_tokens, int64_t n,
-                        int64_t rows_per_slab, double *__restrict__ partial, int64_t n_pad,
-                        int first_fresh_slab, int x_complete) {
+__device__ __forceinline__ void calib_cell(const uint16_t *__restrict__ X, int64_t ldx,
+                                           int64_t n_tokens, int64_t n, int64_t rows_per_slab,
+                                           double *__restrict__ partial, int64_t n_pad,
+                                           int first_fresh_slab, int x_complete, int strip,
+                                           int slab) {
     // Programmatic dependent launch: the next kernel in the stream may start as soon as this
     // grid's CTAs are all resident.  X is read only after everything queued earlier on the
     // stream has completed - the kernel before this one may be the one that writes X - unless
@@ -37,8 +40,6 @@ calib_accumulate_kernel(const uint16_t *__restrict__ X, int64_t ldx, int64_t n_t
     if (!x_complete) pdl_wait();
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-    const int strip = blockIdx.x;
-    const int slab = blockIdx.y;
     const int64_t col = static_cast<int64_t>(strip) * kStripChannels + lane * 8;
     const int64_t row_begin = static_cast<int64_t>(slab) * rows_per_slab;
     const int64_t row_end = min(n_tokens, row_begin + rows_per_slab);
@@ -94,17 +95,52 @@ calib_accumulate_kernel(const uint16_t *__restrict__ X, int64_t ldx, int64_t n_t
     }
 }
 
+template <bool BF16, bool VEC>
+__global__ void __launch_bounds__(kCalibThreads)
+calib_accumulate_kernel(const uint16_t *__restrict__ X, int64_t ldx, int64_t n_tokens, int64_t n,
+                        int64_t rows_per_slab, double *__restrict__ partial, int64_t n_pad,
+                        int first_fresh_slab, int x_complete) {
+    calib_cell<BF16, VEC>(X, ldx, n_tokens, n, rows_per_slab, partial, n_pad, first_fresh_slab,
+                          x_complete, blockIdx.x, blockIdx.y);
+}
+
+// Several activation matrices (the inputs of one transformer block, say) in one launch: a
+// matrix owns strips x slabs consecutive CTAs, strips fastest.  For inputs so small that a launch
+// of their own would be mostly ramp-up.
+constexpr int kCalibMaxJobs = 8;
+struct CalibJob {
+    const uint16_t *X;
+    double *partial;
+    int64_t ldx, n_tokens, n, n_pad, rows_per_slab;
+    int strips, first_fresh_slab, first_cta;
+};
+struct CalibJobTable {
+    int count;
+    CalibJob job[kCalibMaxJobs];
+};
+
+template <bool BF16>
+__global__ void __launch_bounds__(kCalibThreads, 4)  // the occupancy of the single-matrix kernel
+calib_accumulate_multi_kernel(const __grid_constant__ CalibJobTable jobs, int x_complete) {
+    int jk = 0;
+    while (jk + 1 < jobs.count && static_cast<int>(blockIdx.x) >= jobs.job[jk + 1].first_cta) ++jk;
+    const CalibJob &j = jobs.job[jk];
+    const int local = static_cast<int>(blockIdx.x) - j.first_cta;
+    const int slab = local / j.strips;
+    calib_cell<BF16, true>(j.X, j.ldx, j.n_tokens, j.n, j.rows_per_slab, j.partial, j.n_pad,
+                           j.first_fresh_slab, x_complete, local - slab * j.strips, slab);
+}
+
 // Finalisation.  CTA `strip` sums its 256 channels over the valid slab rows (four slab groups
 // in parallel, each in ascending order, then the groups in order), writes colsq and its strip
 // total; the last CTA to arrive adds the strip totals in
 // ascending order to S and writes the per-channel factor for every channel:
 //     u = colsq32 / S32 ;  den = 1 - u ;  c = 0.5 / den          (binary32, round to nearest)
 // No CTA waits for another one (the last arrival does the tail), so the kernel cannot hang.
-__global__ void __launch_bounds__(kFinalThreads)
-finalize_kernel(const double *__restrict__ partial, int slabs_valid, int64_t n, int64_t n_pad,
-                int strips, double *__restrict__ colsq, double *__restrict__ strip_sum,
-                float *__restrict__ factor, float *__restrict__ factor_pairs,
-                DeviceScalars *__restrict__ scalars) {
+__device__ __forceinline__ void finalize_strip(
+    const double *__restrict__ partial, int slabs_valid, int64_t n, int64_t n_pad, int strips,
+    double *__restrict__ colsq, double *__restrict__ strip_sum, float *__restrict__ factor,
+    float *__restrict__ factor_pairs, DeviceScalars *__restrict__ scalars, int strip) {
     __shared__ double part[kFinalGroups][kStripChannels];
     __shared__ double red[kStripChannels];
     __shared__ bool is_last;
@@ -112,7 +148,7 @@ finalize_kernel(const double *__restrict__ partial, int slabs_valid, int64_t n, 
     pdl_wait();  // all partial sums are in place
     const int t = threadIdx.x & (kStripChannels - 1);  // channel within the strip
     const int g = threadIdx.x / kStripChannels;        // slab group
-    const int64_t ch = static_cast<int64_t>(blockIdx.x) * kStripChannels + t;
+    const int64_t ch = static_cast<int64_t>(strip) * kStripChannels + t;
     // Group g adds a contiguous range of slabs in ascending order (eight loads in flight);
     // the groups are then added in ascending order: a fixed summation order.
     const int per_group = (slabs_valid + kFinalGroups - 1) / kFinalGroups;
@@ -146,7 +182,7 @@ finalize_kernel(const double *__restrict__ partial, int slabs_valid, int64_t n, 
         __syncthreads();
     }
     if (threadIdx.x == 0) {
-        strip_sum[blockIdx.x] = red[0];
+        strip_sum[strip] = red[0];
         __threadfence();
         unsigned int ticket = atomicAdd(&scalars->ticket, 1u);
         is_last = (ticket == static_cast<unsigned int>(strips) - 1u);
@@ -220,6 +256,39 @@ finalize_kernel(const double *__restrict__ partial, int slabs_valid, int64_t n, 
     }
 }
 
+__global__ void __launch_bounds__(kFinalThreads)
+finalize_kernel(const double *__restrict__ partial, int slabs_valid, int64_t n, int64_t n_pad,
+                int strips, double *__restrict__ colsq, double *__restrict__ strip_sum,
+                float *__restrict__ factor, float *__restrict__ factor_pairs,
+                DeviceScalars *__restrict__ scalars) {
+    finalize_strip(partial, slabs_valid, n, n_pad, strips, colsq, strip_sum, factor, factor_pairs,
+                   scalars, blockIdx.x);
+}
+
+// Several contexts in one launch: context j owns the CTAs [first_cta, first_cta + strips) and has
+// its own arrival counter, so the contexts do not wait for each other either.
+struct FinalJob {
+    const double *partial;
+    double *colsq, *strip_sum;
+    float *factor, *factor_pairs;
+    DeviceScalars *scalars;
+    int64_t n, n_pad;
+    int slabs_valid, strips, first_cta;
+};
+struct FinalJobTable {
+    int count;
+    FinalJob job[kFinalMaxJobs];
+};
+
+__global__ void __launch_bounds__(kFinalThreads)
+finalize_multi_kernel(const __grid_constant__ FinalJobTable jobs) {
+    int jk = 0;
+    while (jk + 1 < jobs.count && static_cast<int>(blockIdx.x) >= jobs.job[jk + 1].first_cta) ++jk;
+    const FinalJob &j = jobs.job[jk];
+    finalize_strip(j.partial, j.slabs_valid, j.n, j.n_pad, j.strips, j.colsq, j.strip_sum, j.factor,
+                   j.factor_pairs, j.scalars, static_cast<int>(blockIdx.x) - j.first_cta);
+}
+
 template <bool BF16, bool VEC>
 static int query_blocks_per_sm() {
     int blocks = 0;
@@ -231,20 +300,28 @@ static int query_blocks_per_sm() {
 
 int calib_query_blocks_per_sm() { return query_blocks_per_sm<false, true>(); }
 
-sp_status launch_calib_accumulate(sp_ctx *ctx, const void *X, sp_dtype dtype, int64_t n_tokens,
-                                  int64_t ldx, cudaStream_t stream, bool x_complete) {
-    const int64_t n = ctx->d_in;
+// Slabs and rows per slab for one activation matrix of a launch that covers `total_strips`
+// strips in all (its own, plus those of the other matrices of a multi-input launch).
+static void calib_partition(const sp_ctx *ctx, int64_t n_tokens, int64_t total_strips,
+                            int64_t &slabs, int64_t &rows_per_slab) {
     // One resident wave: strips x slabs CTAs fill the GPU once, every CTA gets the same rows.
     const int64_t resident = static_cast<int64_t>(ctx->sm_count) * ctx->calib_blocks_per_sm;
-    int64_t slabs = resident / ctx->strips;
+    slabs = resident / total_strips;
     if (slabs < 1) slabs = 1;
     if (slabs > kMaxSlabs) slabs = kMaxSlabs;
     const int64_t min_rows = kCalibWarps * kRowsInFlight;  // at least one full step per warp
-    int64_t max_slabs_by_rows = (n_tokens + min_rows - 1) / min_rows;
+    const int64_t max_slabs_by_rows = (n_tokens + min_rows - 1) / min_rows;
     if (slabs > max_slabs_by_rows) slabs = max_slabs_by_rows;
-    int64_t rows_per_slab = (n_tokens + slabs - 1) / slabs;
+    rows_per_slab = (n_tokens + slabs - 1) / slabs;
     rows_per_slab = (rows_per_slab + kCalibWarps - 1) / kCalibWarps * kCalibWarps;
     slabs = (n_tokens + rows_per_slab - 1) / rows_per_slab;
+}
+
+sp_status launch_calib_accumulate(sp_ctx *ctx, const void *X, sp_dtype dtype, int64_t n_tokens,
+                                  int64_t ldx, cudaStream_t stream, bool x_complete) {
+    const int64_t n = ctx->d_in;
+    int64_t slabs, rows_per_slab;
+    calib_partition(ctx, n_tokens, ctx->strips, slabs, rows_per_slab);
 
     const bool vec = aligned16(X) && (ldx % 8 == 0) && (n % 8 == 0);
     const bool bf16 = dtype == SP_BF16;
@@ -271,6 +348,102 @@ sp_status launch_calib_accumulate(sp_ctx *ctx, const void *X, sp_dtype dtype, in
     if (slabs > ctx->slabs_valid) ctx->slabs_valid = static_cast<int>(slabs);
     ctx->n_tokens += n_tokens;
     ctx->dirty = true;
+    return SP_OK;
+}
+
+bool calib_multi_applies(const sp_ctx *ctx, const void *X, int64_t ldx) {
+    return aligned16(X) && ldx % 8 == 0 && ctx->d_in % 8 == 0;
+}
+
+sp_status launch_calib_accumulate_multi(sp_ctx *const *ctxs, const CalibItem *items, int count,
+                                        sp_dtype dtype, cudaStream_t stream, bool x_complete) {
+    if (count > kCalibMaxJobs) return SP_ERR_INVALID_ARG;
+    int64_t total_strips = 0;
+    for (int i = 0; i < count; ++i) total_strips += ctxs[i]->strips;
+    CalibJobTable table{};
+    table.count = count;
+    int64_t ctas = 0;
+    int64_t slabs_of[kCalibMaxJobs];
+    for (int i = 0; i < count; ++i) {
+        sp_ctx *c = ctxs[i];
+        int64_t slabs, rows_per_slab;
+        calib_partition(c, items[i].n_tokens, total_strips, slabs, rows_per_slab);
+        slabs_of[i] = slabs;
+        CalibJob &j = table.job[i];
+        j.X = static_cast<const uint16_t *>(items[i].X);
+        j.partial = c->partial;
+        j.ldx = items[i].ldx;
+        j.n_tokens = items[i].n_tokens;
+        j.n = c->d_in;
+        j.n_pad = c->n_pad;
+        j.rows_per_slab = rows_per_slab;
+        j.strips = c->strips;
+        j.first_fresh_slab = c->slabs_valid;
+        j.first_cta = static_cast<int>(ctas);
+        ctas += slabs * c->strips;
+    }
+    PdlConfig pdl(dim3(static_cast<unsigned>(ctas)), dim3(kCalibThreads), stream);
+    const int x_ok = x_complete ? 1 : 0;
+    cudaError_t e = dtype == SP_BF16
+                        ? cudaLaunchKernelEx(&pdl.cfg, calib_accumulate_multi_kernel<true>, table, x_ok)
+                        : cudaLaunchKernelEx(&pdl.cfg, calib_accumulate_multi_kernel<false>, table, x_ok);
+    if (e != cudaSuccess) return cuda_fail(e);
+    sp_status st = check_launch();
+    if (st != SP_OK) return st;
+    for (int i = 0; i < count; ++i) {
+        sp_ctx *c = ctxs[i];
+        if (slabs_of[i] > c->slabs_valid) c->slabs_valid = static_cast<int>(slabs_of[i]);
+        c->n_tokens += items[i].n_tokens;
+        c->dirty = true;
+    }
+    return SP_OK;
+}
+
+// Finalises every context of the list that has batches pending, in one launch when there are
+// several (a context may appear more than once).
+sp_status launch_finalize_pending(sp_ctx *const *ctxs, int count, cudaStream_t stream) {
+    sp_ctx *todo[kFinalMaxJobs];
+    int n_todo = 0;
+    for (int i = 0; i < count; ++i) {
+        sp_ctx *c = ctxs[i];
+        if (!c->dirty) continue;
+        bool seen = false;
+        for (int k = 0; k < n_todo; ++k) seen = seen || todo[k] == c;
+        if (seen) continue;
+        if (n_todo == kFinalMaxJobs) {  // more distinct contexts than one table holds
+            sp_status st = launch_finalize(c, stream);
+            if (st != SP_OK) return st;
+            continue;
+        }
+        todo[n_todo++] = c;
+    }
+    if (n_todo == 0) return SP_OK;
+    if (n_todo == 1) return launch_finalize(todo[0], stream);
+    FinalJobTable table{};
+    table.count = n_todo;
+    int ctas = 0;
+    for (int i = 0; i < n_todo; ++i) {
+        sp_ctx *c = todo[i];
+        FinalJob &j = table.job[i];
+        j.partial = c->partial;
+        j.colsq = c->colsq;
+        j.strip_sum = c->strip_sum;
+        j.factor = c->factor;
+        j.factor_pairs = c->factor_pairs;
+        j.scalars = c->scalars;
+        j.n = c->d_in;
+        j.n_pad = c->n_pad;
+        j.slabs_valid = c->slabs_valid;
+        j.strips = c->strips;
+        j.first_cta = ctas;
+        ctas += c->strips;
+    }
+    PdlConfig pdl(dim3(static_cast<unsigned>(ctas)), dim3(kFinalThreads), stream);
+    cudaError_t e = cudaLaunchKernelEx(&pdl.cfg, finalize_multi_kernel, table);
+    if (e != cudaSuccess) return cuda_fail(e);
+    sp_status st = check_launch();
+    if (st != SP_OK) return st;
+    for (int i = 0; i < n_todo; ++i) todo[i]->dirty = false;
     return SP_OK;
 }
 

@@ -84,6 +84,16 @@ int calib_query_blocks_per_sm();
 sp_status launch_calib_accumulate(sp_ctx *ctx, const void *X, sp_dtype dtype, int64_t n_tokens,
                                   int64_t ldx, cudaStream_t stream, bool x_complete = false);
 sp_status launch_finalize(sp_ctx *ctx, cudaStream_t stream);
+sp_status launch_finalize_pending(sp_ctx *const *ctxs, int count, cudaStream_t stream);
+// One batch for each of several contexts (all different) in one launch; every item must satisfy
+// calib_multi_applies (16-byte access).
+struct CalibItem {
+    const void *X;
+    int64_t n_tokens, ldx;
+};
+bool calib_multi_applies(const sp_ctx *ctx, const void *X, int64_t ldx);
+sp_status launch_calib_accumulate_multi(sp_ctx *const *ctxs, const CalibItem *items, int count,
+                                        sp_dtype dtype, cudaStream_t stream, bool x_complete);
 int64_t calib_static_max_d_in();
 sp_status launch_calib_stats_static(int device, const void *X, sp_dtype dtype, int64_t n_tokens,
                                     int64_t d_in, int64_t ldx, double *colsq_out,

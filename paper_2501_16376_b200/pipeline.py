@@ -113,8 +113,29 @@ def select_block(mb: ModelBuffers, b: int, mode_arg, stream=None):
                                         W_outs=mb.outputs[b], stream=stream)
 
 
+#: up to this many bytes per accumulate launch, the inputs of a block share their launches
+MULTI_CALIB_BYTES = 64 << 20
+
+
+def calibrate_block(mb: ModelBuffers, batch_tokens: int, stream=None) -> int:
+    """Statistics of all layer inputs of a block with shared launches: per batch one
+    sp_calib_accumulate_multi over the inputs, then one finalisation launch.  Returns the number
+    of accumulate launches."""
+    names = list(mb.workload.input_widths())
+    ctxs = [mb.ctxs[name] for name in names]
+    for ctx in ctxs:
+        ctx.sp_calib_reset(stream)
+    T = mb.workload.tokens
+    before = sp.sp_launch_count()
+    for t0 in range(0, T, batch_tokens):
+        sp.sp_calib_accumulate_multi(ctxs, [mb.acts[name][t0:min(T, t0 + batch_tokens)]
+                                            for name in names], stream, True)
+    return sp.sp_launch_count() - before
+
+
 def prune_model(mb: ModelBuffers, mode_arg, batch_tokens: int, phase_events=None, stream=None,
-                grouped: bool = True, per_block: bool | None = None):
+                grouped: bool = True, per_block: bool | None = None,
+                multi_calib: bool | None = None):
     """One pass of the whole hot path over the model: for every block and every distinct layer
     input, accumulate the calibration statistics, finalise them, then select + write back every
     layer that reads this input.  phase_events, if given, is a list that receives
@@ -128,13 +149,20 @@ def prune_model(mb: ModelBuffers, mode_arg, batch_tokens: int, phase_events=None
     Selection calls: per_block (the default) prunes all layers of a block with one call once
     all its inputs are calibrated; otherwise grouped gives the layers that read one input one
     grouped call (one launch when their layouts allow), else every layer gets a call of its
-    own.  Returns launch counts."""
+    own.  multi_calib (per-block passes; the default when one input's batch is below
+    MULTI_CALIB_BYTES): the inputs of a block share their accumulate launches and their
+    finalisation launch.  Returns launch counts."""
     w = mb.workload
     n_calib = n_select = n_final = 0
     if stream is None:
         stream = torch.cuda.current_stream()   # looked up once, not once per call
     if per_block is None:
         per_block = grouped
+    if multi_calib is None:
+        multi_calib = per_block and len(w.input_widths()) > 1 and \
+            batch_tokens * max(w.input_widths().values()) * 2 <= MULTI_CALIB_BYTES
+    if multi_calib and not per_block:
+        raise ValueError("multi_calib needs per_block")
 
     def mark():
         e = torch.cuda.Event(enable_timing=True)
@@ -160,8 +188,20 @@ def prune_model(mb: ModelBuffers, mode_arg, batch_tokens: int, phase_events=None
         # follow an input's finalisation directly and stream under it), then one selection call
         block_weights = sum(layer.d_out * layer.d_in for layer in w.layers)
         last = mark() if phase_events is not None else None
+        all_ctxs = [mb.ctxs[name] for name in w.input_widths()]
+        x_elements = sum(mb.acts[name].shape[0] * d_in for name, d_in in w.input_widths().items())
         for b in range(w.blocks):
-            for name, d_in in w.input_widths().items():
+            if multi_calib:
+                n_calib += calibrate_block(mb, batch_tokens, stream)
+                e1 = mark() if phase_events is not None else None
+                sp.sp_finalize_multi(all_ctxs, stream)
+                n_final += 1
+                if phase_events is not None:
+                    e2 = mark()
+                    phase_events.append(("calib", last, e1, x_elements))
+                    phase_events.append(("finalize", e1, e2, sum(w.input_widths().values())))
+                    last = e2
+            for name, d_in in ([] if multi_calib else w.input_widths().items()):
                 ctx = mb.ctxs[name]
                 n_calib += calibrate_input(ctx, mb.acts[name], batch_tokens, stream, True)
                 e1 = mark() if phase_events is not None else None

@@ -586,8 +586,9 @@ def test_pass_with_per_block_per_input_and_per_layer_calls_agree(sp, name, arg):
     try:
         batch_tokens = 2 * w.seq_len
         results = {}
-        for how, kw in (("block", {}), ("input", {"per_block": False}),
-                        ("layer", {"per_block": False, "grouped": False})):
+        for how, kw in (("block", {"multi_calib": False}), ("input", {"per_block": False}),
+                        ("layer", {"per_block": False, "grouped": False}),
+                        ("shared", {"multi_calib": True})):
             for ms, os_ in zip(mb.masks, mb.outputs):
                 for m, o in zip(ms, os_):
                     m.zero_()
@@ -599,7 +600,11 @@ def test_pass_with_per_block_per_input_and_per_layer_calls_agree(sp, name, arg):
         assert results["block"][2]["select"] == w.blocks                 # one launch per block
         assert results["input"][2]["select"] == w.blocks * len(w.input_widths())
         assert results["layer"][2]["select"] == w.blocks * len(w.layers)
-        for how in ("input", "layer"):
+        batches = w.tokens // batch_tokens
+        assert results["block"][2]["calib"] == w.blocks * len(w.input_widths()) * batches
+        assert results["shared"][2] == {"calib": w.blocks * batches, "finalize": w.blocks,
+                                        "select": w.blocks}
+        for how in ("input", "layer", "shared"):
             for b in range(w.blocks):
                 for li in range(len(w.layers)):
                     assert torch.equal(results["block"][0][b][li], results[how][0][b][li])
@@ -887,6 +892,75 @@ def test_grouped_selection_rejects_bad_groups(sp):
         with pytest.raises(sp.SpError) as e:
             ctx.sp_select_unstructured_group([W, W.to(torch.bfloat16)], 0.5)
         assert e.value.status == sp.SP_ERR_DTYPE
+
+
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+def test_multi_input_calibration_equals_single_calls_bit_for_bit_and_the_oracle(sp, dtype):
+    # four inputs of different widths (one ragged strip, one without 16-byte access, one with a
+    # padded row stride), three batches of different lengths, one launch per batch
+    widths = [1024, 520, 1001, 4096]
+    lengths = [700, 64, 1300]
+    Xs = {n: _activations(300 + n, sum(lengths), n, dtype) for n in widths}
+    padded = torch.zeros(sum(lengths), 520 + 24, dtype=dtype, device="cuda")
+    padded[:, :520] = Xs[520]
+    Xs[520] = padded[:, :520]
+    multi = {n: sp.Context(n) for n in widths}
+    single = {n: sp.Context(n) for n in widths}
+    try:
+        t0 = 0
+        launches = sp.sp_launch_count()
+        for T in lengths:
+            sp.sp_calib_accumulate_multi([multi[n] for n in widths],
+                                         [Xs[n][t0:t0 + T] for n in widths])
+            t0 += T
+        assert sp.sp_launch_count() - launches == 2 * len(lengths)   # 3 inputs together + 1001 alone
+        t0 = 0
+        for T in lengths:
+            for n in widths:
+                single[n].sp_calib_accumulate(Xs[n][t0:t0 + T])
+            t0 += T
+        launches = sp.sp_launch_count()
+        sp.sp_finalize_multi([multi[n] for n in widths] + [multi[1024]])
+        assert sp.sp_launch_count() - launches == 1
+        sp.sp_finalize_multi([multi[n] for n in widths])              # nothing pending: no launch
+        assert sp.sp_launch_count() - launches == 1
+        for n in widths:
+            cm, Sm, fm, tm = multi[n].sp_get_stats()
+            cs, Ss, fs, ts = single[n].sp_get_stats()
+            assert tm == ts == sum(lengths)
+            assert torch.equal(cm, cs) and Sm == Ss and torch.equal(fm, fs)
+            st = P.oracle_stats([Xs[n]], n)
+            assert P.rel_err(cm.numpy(), st.colsq) <= P.SCORE_RTOL
+            assert np.array_equal(fm.numpy(), so.Stats(cm.numpy().copy(), tm).channel_factor32())
+        # the EWMA kernel's own copy of the factors comes out of the multi finalisation too
+        W = _gen(11, (40, 1024), dtype, 0.02)
+        m1, o1 = multi[1024].sp_select_unstructured(W, 0.5)
+        m2, o2 = single[1024].sp_select_unstructured(W, 0.5)
+        assert torch.equal(m1, m2) and torch.equal(o1.view(torch.int16), o2.view(torch.int16))
+    finally:
+        for c in list(multi.values()) + list(single.values()):
+            c.close()
+
+
+def test_multi_input_calibration_rejects_bad_calls(sp):
+    X = _activations(5, 64, 512, torch.float16)
+    with sp.Context(512) as a, sp.Context(512) as b, sp.Context(256) as c:
+        with pytest.raises(sp.SpError) as e:
+            sp.sp_calib_accumulate_multi([a, a], [X, X])                  # the same sums twice
+        assert e.value.status == sp.SP_ERR_INVALID_ARG
+        with pytest.raises(sp.SpError) as e:
+            sp.sp_calib_accumulate_multi([a, c], [X, X])                  # width mismatch
+        assert e.value.status == sp.SP_ERR_SHAPE
+        with pytest.raises(sp.SpError) as e:
+            sp.sp_calib_accumulate_multi([a, b], [X, X.to(torch.bfloat16)])
+        assert e.value.status == sp.SP_ERR_DTYPE
+        with pytest.raises(sp.SpError) as e:
+            sp.sp_finalize_multi([a, b])                                  # no calibration data
+        assert e.value.status == sp.SP_ERR_STATE
+        sp.sp_calib_accumulate_multi([a, b], [X, X[:0]])                  # an empty batch is skipped
+        assert a.sp_get_stats()[3] == 64
+        with pytest.raises(sp.SpError):
+            b.sp_get_stats()
 
 
 def test_calib_accumulate_ex_flag_changes_ordering_only(sp):

@@ -236,7 +236,7 @@ sp_status sp_calib_accumulate_multi(sp_ctx *const *ctxs, const sp_batch *batches
     for (int i = 0; i < n_items; ++i) {
         const sp_batch &b = batches[i];
         if (b.n_tokens == 0) continue;
-        if (!calib_multi_applies(ctxs[i], b.X, b.ldx)) {
+        if (!calib_multi_applies(ctxs[i], b.X, b.ldx, b.n_tokens)) {
             sp_status st = launch_calib_accumulate(ctxs[i], b.X, dtype, b.n_tokens, b.ldx, s, x_complete);
             if (st != SP_OK) return st;
             continue;

@@ -23,13 +23,48 @@ constexpr int kFinalGroups = 4;  // slab groups summed in parallel by the finali
 constexpr int kFinalThreads = kFinalGroups * kStripChannels;
 constexpr int kFinalMaxJobs = 16;  // contexts one finalisation launch can cover
 
-// The work of one CTA: cell (strip, slab) of one activation matrix.
-template <bool BF16, bool VEC>
-__device__ __forceinline__ void calib_cell(const uint16_t *__restrict__ X, int64_t ldx,
-                                           int64_t n_tokens, int64_t n, int64_t rows_per_slab,
-                                           double *__restrict__ partial, int64_t n_pad,
-                                           int first_fresh_slab, int x_complete, int strip,
-                                           int slab) {
+// One activation matrix of an accumulate launch.  I: the type of its sizes - 64-bit for a single
+// matrix, whose sizes the kernel reads from the constant bank wherever it uses them; 32-bit for a
+// table of matrices, where the sizes of the CTA's matrix live in registers for the whole kernel.
+template <class I>
+struct CalibMatrixT {
+    const uint16_t *X;
+    double *partial;
+    I ldx, n_tokens, n, n_pad, rows_per_slab;
+    int strips, first_fresh_slab, first_cta;
+};
+
+// Launch arguments, in two shapes with one kernel body.  CalibOne: a single matrix on a
+// strips x slabs grid.  CalibMany: several matrices (the inputs of one transformer block, say)
+// in one launch for inputs so small that a launch of their own would be mostly ramp-up; a matrix
+// owns strips x slabs consecutive CTAs of a 1-D grid, strips fastest.
+struct CalibOne {
+    using Matrix = CalibMatrixT<int64_t>;
+    Matrix m;
+    __device__ __forceinline__ const Matrix &cell(int &strip, int &slab) const {
+        strip = blockIdx.x;
+        slab = blockIdx.y;
+        return m;
+    }
+};
+constexpr int kCalibMaxJobs = 8;
+struct CalibMany {
+    using Matrix = CalibMatrixT<int>;
+    int count;
+    Matrix job[kCalibMaxJobs];
+    __device__ __forceinline__ const Matrix &cell(int &strip, int &slab) const {
+        int jk = 0;
+        while (jk + 1 < count && static_cast<int>(blockIdx.x) >= job[jk + 1].first_cta) ++jk;
+        const int local = static_cast<int>(blockIdx.x) - job[jk].first_cta;
+        slab = local / job[jk].strips;
+        strip = local - slab * job[jk].strips;
+        return job[jk];
+    }
+};
+
+template <bool BF16, bool VEC, class Args>
+__global__ void __launch_bounds__(kCalibThreads, VEC ? 4 : 1)  // 16-byte path: 4 CTAs per SM
+calib_accumulate_kernel(const __grid_constant__ Args args, int x_complete) {
     // Programmatic dependent launch: the next kernel in the stream may start as soon as this
     // grid's CTAs are all resident.  X is read only after everything queued earlier on the
     // stream has completed - the kernel before this one may be the one that writes X - unless
@@ -38,23 +73,28 @@ __device__ __forceinline__ void calib_cell(const uint16_t *__restrict__ X, int64
     // sums below waits for it.
     pdl_launch_dependents();
     if (!x_complete) pdl_wait();
+    int strip, slab;
+    const typename Args::Matrix &a = args.cell(strip, slab);
+    using I = decltype(a.ldx);
+    const uint16_t *__restrict__ X = a.X;
+    const I ldx = a.ldx, n = a.n;
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-    const int64_t col = static_cast<int64_t>(strip) * kStripChannels + lane * 8;
-    const int64_t row_begin = static_cast<int64_t>(slab) * rows_per_slab;
-    const int64_t row_end = min(n_tokens, row_begin + rows_per_slab);
+    const I col = static_cast<I>(strip) * kStripChannels + lane * 8;
+    const I row_begin = static_cast<I>(slab) * a.rows_per_slab;
+    const I row_end = min(a.n_tokens, row_begin + a.rows_per_slab);
 
     double acc[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) acc[j] = 0.0;
 
-    for (int64_t r = row_begin + warp; r < row_end; r += kCalibWarps * kRowsInFlight) {
+    for (I r = row_begin + warp; r < row_end; r += kCalibWarps * kRowsInFlight) {
         uint32_t v[kRowsInFlight][4];
 #pragma unroll
         for (int u = 0; u < kRowsInFlight; ++u) {
-            const int64_t rr = r + static_cast<int64_t>(u) * kCalibWarps;
+            const I rr = r + static_cast<I>(u) * kCalibWarps;
             if (rr < row_end) {
-                load8<VEC, true>(X + rr * ldx, col, n, v[u]);
+                load8<VEC, true>(X + static_cast<int64_t>(rr) * ldx, col, n, v[u]);
             } else {
                 v[u][0] = v[u][1] = v[u][2] = v[u][3] = 0u;
             }
@@ -79,56 +119,24 @@ __device__ __forceinline__ void calib_cell(const uint16_t *__restrict__ X, int64
     for (int j = 0; j < 8; ++j) sm[warp][lane * 8 + j] = acc[j];
     __syncthreads();
     pdl_wait();  // earlier kernels' partial sums are final
+    // (the matrix is looked up again rather than carried through the loop in registers)
+    int strip_out, slab_out;
+    const typename Args::Matrix &b = args.cell(strip_out, slab_out);
     const int t = threadIdx.x;
-    const int64_t ch = static_cast<int64_t>(strip) * kStripChannels + t;
-    if (ch < n) {
+    const int64_t ch = static_cast<int64_t>(strip_out) * kStripChannels + t;
+    if (ch < b.n) {
         double sum = 0.0;
 #pragma unroll
         for (int w = 0; w < kCalibWarps; ++w) sum += sm[w][t];
-        double *dst = partial + static_cast<int64_t>(slab) * n_pad + ch;
-        if (SP_IN_RANGE(static_cast<int64_t>(slab) * n_pad + ch, kMaxSlabs * n_pad, kDbgCalibPartial)) {
-            if (slab >= first_fresh_slab)
+        const int64_t at = static_cast<int64_t>(slab_out) * b.n_pad + ch;
+        double *dst = b.partial + at;
+        if (SP_IN_RANGE(at, kMaxSlabs * static_cast<int64_t>(b.n_pad), kDbgCalibPartial)) {
+            if (slab_out >= b.first_fresh_slab)
                 *dst = sum;
             else
                 *dst += sum;
         }
     }
-}
-
-template <bool BF16, bool VEC>
-__global__ void __launch_bounds__(kCalibThreads)
-calib_accumulate_kernel(const uint16_t *__restrict__ X, int64_t ldx, int64_t n_tokens, int64_t n,
-                        int64_t rows_per_slab, double *__restrict__ partial, int64_t n_pad,
-                        int first_fresh_slab, int x_complete) {
-    calib_cell<BF16, VEC>(X, ldx, n_tokens, n, rows_per_slab, partial, n_pad, first_fresh_slab,
-                          x_complete, blockIdx.x, blockIdx.y);
-}
-
-// Several activation matrices (the inputs of one transformer block, say) in one launch: a
-// matrix owns strips x slabs consecutive CTAs, strips fastest.  For inputs so small that a launch
-// of their own would be mostly ramp-up.
-constexpr int kCalibMaxJobs = 8;
-struct CalibJob {
-    const uint16_t *X;
-    double *partial;
-    int64_t ldx, n_tokens, n, n_pad, rows_per_slab;
-    int strips, first_fresh_slab, first_cta;
-};
-struct CalibJobTable {
-    int count;
-    CalibJob job[kCalibMaxJobs];
-};
-
-template <bool BF16>
-__global__ void __launch_bounds__(kCalibThreads, 4)  // the occupancy of the single-matrix kernel
-calib_accumulate_multi_kernel(const __grid_constant__ CalibJobTable jobs, int x_complete) {
-    int jk = 0;
-    while (jk + 1 < jobs.count && static_cast<int>(blockIdx.x) >= jobs.job[jk + 1].first_cta) ++jk;
-    const CalibJob &j = jobs.job[jk];
-    const int local = static_cast<int>(blockIdx.x) - j.first_cta;
-    const int slab = local / j.strips;
-    calib_cell<BF16, true>(j.X, j.ldx, j.n_tokens, j.n, j.rows_per_slab, j.partial, j.n_pad,
-                           j.first_fresh_slab, x_complete, local - slab * j.strips, slab);
 }
 
 // Finalisation.  CTA `strip` sums its 256 channels over the valid slab rows (four slab groups
@@ -293,7 +301,7 @@ template <bool BF16, bool VEC>
 static int query_blocks_per_sm() {
     int blocks = 0;
     cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-        &blocks, calib_accumulate_kernel<BF16, VEC>, kCalibThreads, 0);
+        &blocks, calib_accumulate_kernel<BF16, VEC, CalibOne>, kCalibThreads, 0);
     if (e != cudaSuccess || blocks < 1) blocks = 1;
     return blocks;
 }
@@ -326,16 +334,22 @@ sp_status launch_calib_accumulate(sp_ctx *ctx, const void *X, sp_dtype dtype, in
     const bool vec = aligned16(X) && (ldx % 8 == 0) && (n % 8 == 0);
     const bool bf16 = dtype == SP_BF16;
     dim3 grid(static_cast<unsigned>(ctx->strips), static_cast<unsigned>(slabs));
-    const uint16_t *Xp = static_cast<const uint16_t *>(X);
     PdlConfig pdl(grid, dim3(kCalibThreads), stream);
-    double *partial = ctx->partial;
-    int64_t n_pad = ctx->n_pad;
-    int first_fresh = ctx->slabs_valid;
+    CalibOne args{};
+    args.m.X = static_cast<const uint16_t *>(X);
+    args.m.partial = ctx->partial;
+    args.m.ldx = ldx;
+    args.m.n_tokens = n_tokens;
+    args.m.n = n;
+    args.m.n_pad = ctx->n_pad;
+    args.m.rows_per_slab = rows_per_slab;
+    args.m.strips = ctx->strips;
+    args.m.first_fresh_slab = ctx->slabs_valid;
+    args.m.first_cta = 0;
     const int x_ok = x_complete ? 1 : 0;
     cudaError_t launch_err = cudaSuccess;
-#define SP_LAUNCH(B, V)                                                                       \
-    launch_err = cudaLaunchKernelEx(&pdl.cfg, calib_accumulate_kernel<B, V>, Xp, ldx, n_tokens, n, \
-                                    rows_per_slab, partial, n_pad, first_fresh, x_ok)
+#define SP_LAUNCH(B, V) \
+    launch_err = cudaLaunchKernelEx(&pdl.cfg, calib_accumulate_kernel<B, V, CalibOne>, args, x_ok)
     if (bf16) {
         if (vec) SP_LAUNCH(true, true); else SP_LAUNCH(true, false);
     } else {
@@ -351,8 +365,9 @@ sp_status launch_calib_accumulate(sp_ctx *ctx, const void *X, sp_dtype dtype, in
     return SP_OK;
 }
 
-bool calib_multi_applies(const sp_ctx *ctx, const void *X, int64_t ldx) {
-    return aligned16(X) && ldx % 8 == 0 && ctx->d_in % 8 == 0;
+bool calib_multi_applies(const sp_ctx *ctx, const void *X, int64_t ldx, int64_t n_tokens) {
+    return aligned16(X) && ldx % 8 == 0 && ctx->d_in % 8 == 0 && ldx < (int64_t(1) << 30) &&
+           n_tokens < (int64_t(1) << 30);  // the table kernel computes with 32-bit sizes
 }
 
 sp_status launch_calib_accumulate_multi(sp_ctx *const *ctxs, const CalibItem *items, int count,
@@ -360,7 +375,7 @@ sp_status launch_calib_accumulate_multi(sp_ctx *const *ctxs, const CalibItem *it
     if (count > kCalibMaxJobs) return SP_ERR_INVALID_ARG;
     int64_t total_strips = 0;
     for (int i = 0; i < count; ++i) total_strips += ctxs[i]->strips;
-    CalibJobTable table{};
+    CalibMany table{};
     table.count = count;
     int64_t ctas = 0;
     int64_t slabs_of[kCalibMaxJobs];
@@ -369,14 +384,14 @@ sp_status launch_calib_accumulate_multi(sp_ctx *const *ctxs, const CalibItem *it
         int64_t slabs, rows_per_slab;
         calib_partition(c, items[i].n_tokens, total_strips, slabs, rows_per_slab);
         slabs_of[i] = slabs;
-        CalibJob &j = table.job[i];
+        CalibMany::Matrix &j = table.job[i];
         j.X = static_cast<const uint16_t *>(items[i].X);
         j.partial = c->partial;
-        j.ldx = items[i].ldx;
-        j.n_tokens = items[i].n_tokens;
-        j.n = c->d_in;
-        j.n_pad = c->n_pad;
-        j.rows_per_slab = rows_per_slab;
+        j.ldx = static_cast<int>(items[i].ldx);  // calib_multi_applies: all below 2^31
+        j.n_tokens = static_cast<int>(items[i].n_tokens);
+        j.n = static_cast<int>(c->d_in);
+        j.n_pad = static_cast<int>(c->n_pad);
+        j.rows_per_slab = static_cast<int>(rows_per_slab);
         j.strips = c->strips;
         j.first_fresh_slab = c->slabs_valid;
         j.first_cta = static_cast<int>(ctas);
@@ -384,9 +399,10 @@ sp_status launch_calib_accumulate_multi(sp_ctx *const *ctxs, const CalibItem *it
     }
     PdlConfig pdl(dim3(static_cast<unsigned>(ctas)), dim3(kCalibThreads), stream);
     const int x_ok = x_complete ? 1 : 0;
-    cudaError_t e = dtype == SP_BF16
-                        ? cudaLaunchKernelEx(&pdl.cfg, calib_accumulate_multi_kernel<true>, table, x_ok)
-                        : cudaLaunchKernelEx(&pdl.cfg, calib_accumulate_multi_kernel<false>, table, x_ok);
+    cudaError_t e =
+        dtype == SP_BF16
+            ? cudaLaunchKernelEx(&pdl.cfg, calib_accumulate_kernel<true, true, CalibMany>, table, x_ok)
+            : cudaLaunchKernelEx(&pdl.cfg, calib_accumulate_kernel<false, true, CalibMany>, table, x_ok);
     if (e != cudaSuccess) return cuda_fail(e);
     sp_status st = check_launch();
     if (st != SP_OK) return st;
@@ -544,11 +560,19 @@ sp_status launch_calib_stats_static(int device, const void *X, sp_dtype dtype, i
     const bool vec = aligned16(X) && (ldx % 8 == 0) && (n % 8 == 0);
     const bool bf16 = dtype == SP_BF16;
     dim3 grid(static_cast<unsigned>(strips), static_cast<unsigned>(slabs));
-    const uint16_t *Xp = static_cast<const uint16_t *>(X);
-#define SP_LAUNCH(B, V)                                                                       \
-    calib_accumulate_kernel<B, V><<<grid, kCalibThreads, 0, stream>>>(                        \
-        Xp, ldx, n_tokens, n, rows_per_slab, sc->partial, n_pad, /*first_fresh_slab=*/0, \
-        /*x_complete=*/0)
+    CalibOne args{};
+    args.m.X = static_cast<const uint16_t *>(X);
+    args.m.partial = sc->partial;
+    args.m.ldx = ldx;
+    args.m.n_tokens = n_tokens;
+    args.m.n = n;
+    args.m.n_pad = n_pad;
+    args.m.rows_per_slab = rows_per_slab;
+    args.m.strips = strips;
+    args.m.first_fresh_slab = 0;
+    args.m.first_cta = 0;
+#define SP_LAUNCH(B, V) \
+    calib_accumulate_kernel<B, V, CalibOne><<<grid, kCalibThreads, 0, stream>>>(args, /*x_complete=*/0)
     if (bf16) {
         if (vec) SP_LAUNCH(true, true); else SP_LAUNCH(true, false);
     } else {

@@ -91,7 +91,7 @@ struct CalibItem {
     const void *X;
     int64_t n_tokens, ldx;
 };
-bool calib_multi_applies(const sp_ctx *ctx, const void *X, int64_t ldx);
+bool calib_multi_applies(const sp_ctx *ctx, const void *X, int64_t ldx, int64_t n_tokens);
 sp_status launch_calib_accumulate_multi(sp_ctx *const *ctxs, const CalibItem *items, int count,
                                         sp_dtype dtype, cudaStream_t stream, bool x_complete);
 int64_t calib_static_max_d_in();

@@ -963,6 +963,44 @@ def test_multi_input_calibration_rejects_bad_calls(sp):
             b.sp_get_stats()
 
 
+def test_calls_on_two_user_streams_at_once(sp):
+    # two layer inputs, each calibrated and pruned on a stream of its own, the activations written
+    # by the kernel that precedes the first library call on that stream (ordinary stream order,
+    # no promise about X)
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    shapes = [(2048, 4096, 300), (1536, 1000, 257)]           # (d_in, tokens, rows)
+    seeds = [(1.0 + torch.arange(t * n, device="cuda", dtype=torch.float32).reshape(t, n) % 7)
+             for n, t, _ in shapes]
+    Ws = [_gen(40 + i, (r, n), torch.float16, 0.02) for i, (n, t, r) in enumerate(shapes)]
+    torch.cuda.synchronize()
+    ctxs = [sp.Context(n) for n, _, _ in shapes]
+    got = []
+    try:
+        Xs = []
+        for s, ctx, base, W in zip(streams, ctxs, seeds, Ws):
+            with torch.cuda.stream(s):
+                X = (base * 0.25 - 0.5).to(torch.float16)     # written on s, right before its use
+                Xs.append(X)
+                ctx.sp_calib_accumulate(X, stream=s)
+                got.append((ctx.sp_select_nm(W, 2, 4, stream=s),
+                            ctx.sp_select_unstructured(W, 0.5, stream=s)))
+        for s in streams:
+            s.synchronize()
+        for ctx, X, W, ((m_nm, o_nm), (m_e, o_e)), (n, _, _) in zip(ctxs, Xs, Ws, got, shapes):
+            st = P.oracle_stats([X], n)
+            colsq = ctx.sp_get_stats()[0]
+            assert P.rel_err(colsq.numpy(), st.colsq) <= P.SCORE_RTOL
+            own = so.Stats(colsq.numpy().copy(), 1)
+            P.check_selection(m_nm, o_nm, W, so.select_nm(P.bits(W), so.F16, own, 2, 4), None,
+                              strict=True)
+            sel = so.select_unstructured(P.bits(W), so.F16, own, 0.5, want_trace=True)
+            P.check_selection(m_e, o_e, W, sel, P.ewma_allowed_flips(sel))
+    finally:
+        for c in ctxs:
+            c.close()
+
+
 def test_calib_accumulate_ex_flag_changes_ordering_only(sp):
     n = 1000
     X = _activations(81, 3000, n, torch.float16)

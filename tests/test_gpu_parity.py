@@ -1001,6 +1001,49 @@ def test_calls_on_two_user_streams_at_once(sp):
             c.close()
 
 
+@pytest.mark.parametrize("multi", [False, True])
+def test_calibration_waits_for_a_library_kernel_that_writes_its_input(sp, multi):
+    # The producer is one of the library's own kernels, which lets its successor start early;
+    # without the X_COMPLETE promise the accumulate kernel must still see the finished matrix.
+    # Replayed as a CUDA graph, where launches follow each other closely enough for a consumer
+    # that did not wait to read the stale fill value (with the promise given wrongly it does).
+    n, R = 4096, 8192
+    A = _gen(61, (R, n), torch.float16, 0.5)
+    stats = _activations(62, 512, n, torch.float16)
+    with sp.Context(n) as maker, sp.Context(n) as ctx, sp.Context(n) as other:
+        maker.sp_calib_accumulate(stats)
+        maker.sp_score(None)
+        X = torch.full((R, n), 100.0, dtype=torch.float16, device="cuda")   # stale value: obvious
+
+        def producer_then_consumer():
+            ctx.sp_calib_reset()
+            other.sp_calib_reset()
+            maker.sp_select_nm(A, 2, 4, W_out=X, want_mask=False)
+            if multi:
+                sp.sp_calib_accumulate_multi([ctx, other], [X, X[:R // 2]])
+                sp.sp_finalize_multi([ctx, other])
+            else:
+                ctx.sp_calib_accumulate(X)
+                ctx.sp_score(None)
+        producer_then_consumer()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            producer_then_consumer()
+        for _ in range(4):
+            X.fill_(100.0)
+            torch.cuda.synchronize()
+            graph.replay()
+            torch.cuda.synchronize()
+            colsq = ctx.sp_get_stats()[0]
+            st = P.oracle_stats([X], n)
+            assert float(st.colsq.max()) < 100.0 ** 2 * 16    # nothing of the fill is left in X
+            assert P.rel_err(colsq.numpy(), st.colsq) <= P.SCORE_RTOL
+            if multi:
+                half = other.sp_get_stats()[0]
+                assert P.rel_err(half.numpy(), P.oracle_stats([X[:R // 2]], n).colsq) <= P.SCORE_RTOL
+
+
 def test_calib_accumulate_ex_flag_changes_ordering_only(sp):
     n = 1000
     X = _activations(81, 3000, n, torch.float16)

@@ -43,7 +43,7 @@ CALIB_BYTES_PER_ELEMENT = 2.0
 # Keys: calibration -> d_in; selection -> (total rows of the launch, d_in), or
 # ("block", workload) for one launch over all layers of a block.  Shapes that were
 # not captured, and kernels changed since, report null.
-NCU_CALIB_TRAFFIC = {4096: 271.5e6, 11008: 721.5e6}
+NCU_CALIB_TRAFFIC = {4096: 272.0e6, 11008: 725.0e6}
 NCU_SELECT_TRAFFIC = {
     "select_nm_stream_kernel": {("block", "llama2-7b"): 782.4e6,
                                 (12288, 4096): 154.9e6, (4096, 4096): 33.6e6,

@@ -5,8 +5,9 @@
 // Layout of the work: the channel axis is cut into strips of 256 channels (one warp-wide
 // 16-byte load per activation row), the token axis into slabs.  One CTA owns one
 // (strip, slab) cell; its 8 warps take rows slab_begin + warp, + 8, ... and keep 8 rows in
-// flight per lane.  Squares are exact in fp32; the sum of the 8 in-flight squares is formed in
-// fp32 and added to an fp64 accumulator.  The CTA adds its 256 sums to row `slab` of the
+// flight per lane.  Squares are exact in fp32 (formed straight from the 16-bit values by the
+// mixed-precision fused multiply-add); the sum of the 8 in-flight squares is formed in fp32 and
+// added to an fp64 accumulator.  The CTA adds its 256 sums to row `slab` of the
 // partial-sum array, which no other CTA touches: there are no floating-point atomics, so the
 // statistics are reproducible bit for bit for a given sequence of batches.
 #include <mutex>
@@ -104,10 +105,8 @@ calib_accumulate_kernel(const __grid_constant__ Args args, int x_complete) {
         for (int j = 0; j < 8; ++j) s[j] = 0.0f;
 #pragma unroll
         for (int u = 0; u < kRowsInFlight; ++u) {
-            float x[8];
-            unpack8<BF16>(v[u], x);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) s[j] = fmaf(x[j], x[j], s[j]);
+            for (int k = 0; k < 4; ++k) fma_square2<BF16>(v[u][k], s[2 * k], s[2 * k + 1]);
         }
 #pragma unroll
         for (int j = 0; j < 8; ++j) acc[j] += static_cast<double>(s[j]);

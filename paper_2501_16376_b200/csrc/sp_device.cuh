@@ -35,6 +35,23 @@ __device__ __forceinline__ void unpack8(const uint32_t (&p)[4], float (&w)[8]) {
     }
 }
 
+// s0 += lo^2, s1 += hi^2 for the two 16-bit floats of a packed word, with the mixed-precision
+// fused multiply-add of sm_100 (16-bit operands, binary32 addend and result): the square of a
+// 16-bit float is exact in binary32 and the sum is rounded once, so the result is the one that
+// converting the operand first and a binary32 fma would give, without the conversions.
+template <bool BF16>
+__device__ __forceinline__ void fma_square2(uint32_t p, float &s0, float &s1) {
+    unsigned short lo, hi;
+    asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(p));
+    if constexpr (BF16) {
+        asm("fma.rn.f32.bf16 %0, %1, %1, %0;" : "+f"(s0) : "h"(lo));
+        asm("fma.rn.f32.bf16 %0, %1, %1, %0;" : "+f"(s1) : "h"(hi));
+    } else {
+        asm("fma.rn.f32.f16 %0, %1, %1, %0;" : "+f"(s0) : "h"(lo));
+        asm("fma.rn.f32.f16 %0, %1, %1, %0;" : "+f"(s1) : "h"(hi));
+    }
+}
+
 // Loads elements [col, col+8) of a row into four packed words; elements at or past n read
 // as zero.  VEC: 16-byte access (requires 16-byte aligned row start, n % 8 == 0, col % 8 == 0).
 // STREAM: the data is read once (bypass L1, evict-first behaviour).

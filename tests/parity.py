@@ -54,7 +54,8 @@ def ewma_allowed_flips(sel: so.Selection) -> np.ndarray:
     """Entries whose oracle score lies within the band around the threshold it was tested against."""
     L = sel.L.astype(np.float64)
     thr = sel.thr.astype(np.float64)
-    return np.abs(L - thr) <= BAND_RTOL * np.maximum(np.abs(L), np.abs(thr))
+    with np.errstate(invalid="ignore"):     # inf - inf (a channel with infinite factor): not in band
+        return np.abs(L - thr) <= BAND_RTOL * np.maximum(np.abs(L), np.abs(thr))
 
 
 def nm_allowed_flips(sel: so.Selection, n: int, M: int) -> np.ndarray:

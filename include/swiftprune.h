@@ -143,11 +143,13 @@ sp_status sp_calib_accumulate_ex(sp_ctx *ctx, const void *X, sp_dtype dtype, int
 
 /*
  * One batch for each of several layer inputs (the inputs of one transformer block, say) in one
- * launch: exactly the effect of sp_calib_accumulate_ex(ctxs[i], batches[i].X, dtype,
- * batches[i].n_tokens, batches[i].ldx, flags, stream) for every i, bit for bit - Algorithm 1's
- * step 1 is a sum per channel, and the channels of different inputs have nothing to do with
- * each other.  For inputs so narrow or batches so short that a launch of their own would be
- * mostly ramp-up.  ctxs and batches are HOST arrays of n_items entries (1 <= n_items <=
+ * launch: the effect of sp_calib_accumulate_ex(ctxs[i], batches[i].X, dtype,
+ * batches[i].n_tokens, batches[i].ldx, flags, stream) for every i - Algorithm 1's step 1 is a
+ * sum per channel, and the channels of different inputs have nothing to do with each other.
+ * The sums agree with those of the single calls to rounding (the tokens of a batch may be cut
+ * into slabs differently, which moves the last bits of a sum) and are, like theirs,
+ * reproducible bit for bit for a given sequence of calls.  For inputs so narrow or batches so
+ * short that a launch of their own would be mostly ramp-up.  ctxs and batches are HOST arrays of n_items entries (1 <= n_items <=
  * SP_MAX_MULTI); the contexts must all be different (two batches of one launch cannot update
  * the same sums: SP_ERR_INVALID_ARG) and on one device; a batch with n_tokens == 0 is skipped;
  * batches that do not allow 16-byte access get launches of their own.

@@ -895,7 +895,7 @@ def test_grouped_selection_rejects_bad_groups(sp):
 
 
 @pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
-def test_multi_input_calibration_equals_single_calls_bit_for_bit_and_the_oracle(sp, dtype):
+def test_multi_input_calibration_matches_single_calls_and_the_oracle(sp, dtype):
     # four inputs of different widths (one ragged strip, one without 16-byte access, one with a
     # padded row stride), three batches of different lengths, one launch per batch
     widths = [1024, 520, 1001, 4096]
@@ -928,15 +928,28 @@ def test_multi_input_calibration_equals_single_calls_bit_for_bit_and_the_oracle(
             cm, Sm, fm, tm = multi[n].sp_get_stats()
             cs, Ss, fs, ts = single[n].sp_get_stats()
             assert tm == ts == sum(lengths)
-            assert torch.equal(cm, cs) and Sm == Ss and torch.equal(fm, fs)
+            # the same sums up to the grouping of the binary32 partial sums (slabs cut differently)
+            assert P.rel_err(cm.numpy(), cs.numpy()) <= 1e-7 and abs(Sm - Ss) <= 1e-7 * Ss
+            assert P.rel_err(fm.numpy(), fs.numpy()) <= 1e-6
             st = P.oracle_stats([Xs[n]], n)
             assert P.rel_err(cm.numpy(), st.colsq) <= P.SCORE_RTOL
             assert np.array_equal(fm.numpy(), so.Stats(cm.numpy().copy(), tm).channel_factor32())
         # the EWMA kernel's own copy of the factors comes out of the multi finalisation too
         W = _gen(11, (40, 1024), dtype, 0.02)
         m1, o1 = multi[1024].sp_select_unstructured(W, 0.5)
-        m2, o2 = single[1024].sp_select_unstructured(W, 0.5)
-        assert torch.equal(m1, m2) and torch.equal(o1.view(torch.int16), o2.view(torch.int16))
+        own = so.Stats(multi[1024].sp_get_stats()[0].numpy().copy(), 1)
+        sel = so.select_unstructured(P.bits(W), P.odtype(W), own, 0.5, want_trace=True)
+        P.check_selection(m1, o1, W, sel, P.ewma_allowed_flips(sel))
+        # and the sums are reproducible: the same calls again give the same bits
+        again = {n: sp.Context(n) for n in widths}
+        t0 = 0
+        for T in lengths:
+            sp.sp_calib_accumulate_multi([again[n] for n in widths],
+                                         [Xs[n][t0:t0 + T] for n in widths])
+            t0 += T
+        for n in widths:
+            assert torch.equal(again[n].sp_get_stats()[0], multi[n].sp_get_stats()[0])
+            again[n].close()
     finally:
         for c in list(multi.values()) + list(single.values()):
             c.close()

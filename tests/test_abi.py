@@ -86,3 +86,26 @@ def test_create_without_a_device_fails_cleanly(lib_path):
     with pytest.raises(binding.SpError) as e:
         binding.Context(64, device=0)
     assert e.value.status in (binding.SP_ERR_CUDA, binding.SP_ERR_INVALID_ARG)
+
+
+def test_product_path_fails_loudly_without_the_library_or_a_device(tmp_path):
+    # no CPU fallback anywhere: a missing library is an ImportError, a missing GPU a refusal
+    import subprocess
+    import sys
+    env = dict(os.environ, SWIFTPRUNE_LIBRARY=str(tmp_path / "not_built.so"))
+    proc = subprocess.run([sys.executable, "-c", "import paper_2501_16376_b200.binding"],
+                          cwd=ROOT, env=env, capture_output=True, text=True, timeout=300)
+    assert proc.returncode != 0 and "no CPU fallback" in proc.stderr
+    import torch
+    if not torch.cuda.is_available():
+        proc = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--workload", "single-512",
+                               "--no-cpu-baseline"], cwd=ROOT, capture_output=True, text=True, timeout=300)
+        assert proc.returncode != 0 and "CUDA device" in proc.stderr
+        # and nothing in the package reaches for the oracle
+        src = ""
+        pkg = os.path.join(ROOT, "paper_2501_16376_b200")
+        for name in os.listdir(pkg):
+            if name.endswith(".py"):
+                with open(os.path.join(pkg, name)) as f:
+                    src += f.read()
+        assert "import oracle" not in src and "from oracle" not in src
